@@ -1,0 +1,145 @@
+/*
+ * wcc.h -- C ABI of libwcc: the forward pass of one Wavelet Compressed Convolution (WCC) layer
+ * on an NVIDIA B200 (sm_100a).
+ *
+ *     WCC(K, x) = H^T T^T K_1x1 T H x                                   (Eq. 9, Alg. 1)
+ *
+ * H is the multi-level per-channel 2-D Haar transform (Eq. 3-6), T keeps the k wavelet-domain
+ * positions of largest feature norm across channels, the same positions for every channel
+ * (Eq. 7 and Sec. 4 "Joint hard shrinkage"), K_1x1 is the pointwise convolution applied to the kept
+ * columns only, T^T zero-fills and H^T is the inverse transform (Eq. 4).  The kept columns and the
+ * weights are quantized with the signed symmetric scheme of Eq. 1-2 (8 bits).
+ *
+ * Conventions, valid for every entry point unless it says otherwise:
+ *  - Every data pointer is a DEVICE pointer owned by the caller, 16-byte aligned.  The library
+ *    allocates no device memory; scratch space is passed in (`ws`, sized by wcc_workspace_bytes).
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only enqueue
+ *    work; they never synchronise and never throw.  Errors the host can see (bad shape, null or
+ *    misaligned pointer, small workspace) are returned before anything is launched.
+ *  - Tensors are dense, row-major: activations [N][C][H][Wd], weights [Cout][Cin].
+ *  - Wavelet-domain maps use the quadrant layout inside each H x Wd plane: level l works on the
+ *    top-left (H/2^(l-1)) x (Wd/2^(l-1)) corner and leaves y1 (low-pass) top-left, y2 (difference
+ *    along the width) top-right, y3 (difference along the height) bottom-left, y4 bottom-right.
+ *    A "position" p = row * Wd + col indexes this layout; P = H * Wd.
+ *  - levels is 1, 2 or 3 (the paper uses 3); H and Wd must be multiples of 2^levels.
+ *  - Cin <= 256 and Cout <= 256 for wcc_forward (one tensor-core tile along each).
+ *  - There is no CPU fallback: the library is built for sm_100a only.
+ */
+#ifndef WCC_H_
+#define WCC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    WCC_OK = 0,
+    WCC_ERR_NULL = 1,        /* a required pointer is NULL */
+    WCC_ERR_SHAPE = 2,       /* non-positive dims, H or Wd not a multiple of 2^levels, levels/channels out of range */
+    WCC_ERR_K = 3,           /* k < 1 or k > H*Wd */
+    WCC_ERR_BITS = 4,        /* bits not in {0, 2..8} */
+    WCC_ERR_DTYPE = 5,       /* unknown wcc_dtype */
+    WCC_ERR_ALIGN = 6,       /* a pointer is not 16-byte aligned */
+    WCC_ERR_WORKSPACE = 7,   /* ws_bytes smaller than wcc_workspace_bytes(...) */
+    WCC_ERR_CUDA = 8,        /* a CUDA runtime call or launch failed */
+    WCC_ERR_TIMEOUT = 9,     /* a bounded device-side wait ran out (reported by wcc_last_status) */
+    WCC_ERR_NONFINITE = 10   /* reserved */
+} wcc_status;
+
+typedef enum { WCC_F32 = 0, WCC_BF16 = 1 } wcc_dtype;   /* element type of activations x and y */
+
+/* Scratch bytes wcc_forward / wcc_forward_debug need for these arguments (0 on invalid arguments). */
+size_t wcc_workspace_bytes(int N, int Cin, int Cout, int H, int Wd, int levels, int k, int bits, wcc_dtype dt);
+
+/* Scratch bytes wcc_select_topk needs. */
+size_t wcc_select_workspace_bytes(int N, int P);
+
+/*
+ * Forward Haar transform, all levels, of every (n, c) plane (Eq. 3, 5, 6), and in the same pass the
+ * feature norm across channels of every position (Alg. 1, "vector norm along the channel dimension").
+ *   x     in : [N][C][H][Wd] of dt
+ *   coef  out: fp32 [N][C][H][Wd], quadrant layout.  Arithmetic is fp32: per 2x2 block a,b / c,d:
+ *              s0=a+b d0=a-b s1=c+d d1=c-d; y1=(s0+s1)/2 y2=(d0+d1)/2 y3=(s0-s1)/2 y4=(d0-d1)/2.
+ *   nrm2  out: fp32 [N][P] squared l2 norm over channels, one fused multiply-add per channel in
+ *              ascending channel order; NULL to skip.
+ */
+wcc_status wcc_haar_fwd(const void* x, int N, int C, int H, int Wd, int levels, wcc_dtype dt,
+                        float* coef, float* nrm2, void* stream);
+
+/*
+ * Inverse Haar transform (Eq. 4: the transposed convolution, coarsest level first).
+ *   coef  in : fp32 [N][C][H][Wd], quadrant layout
+ *   x_out out: [N][C][H][Wd] of dt (bf16: round to nearest even)
+ * Per quadruple: t0=y1+y3 t1=y1-y3 u0=y2+y4 u1=y2-y4; a=(t0+u0)/2 b=(t0-u0)/2 c=(t1+u1)/2 d=(t1-u1)/2.
+ */
+wcc_status wcc_haar_inv(const float* coef, int N, int C, int H, int Wd, int levels, wcc_dtype dt,
+                        void* x_out, void* stream);
+
+/*
+ * Joint shrinkage T (Eq. 7; Alg. 1 "top ceil(gamma n_w n_h) vectors by norm"): for each image the k
+ * positions of largest norm.  Ties at the k-th value go to the lowest position.  -0 ranks equal to +0;
+ * the order of NaNs is unspecified.
+ *   nrm2 in : fp32 [N][P]
+ *   idx  out: int32 [N][k], ascending within each image
+ *   tau  out: fp32 [N], the k-th largest norm of each image; NULL to skip
+ *   ws       : scratch of at least wcc_select_workspace_bytes(N, P) bytes
+ */
+wcc_status wcc_select_topk(const float* nrm2, int N, int P, int k, int32_t* idx, float* tau,
+                           void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * The whole layer (Eq. 9 in the order of Alg. 1).
+ *   x   in : [N][Cin][H][Wd] of dt          Wt in: fp32 [Cout][Cin] (no bias)
+ *   k      : kept positions per image (ceil(gamma * H * Wd))
+ *   bits   : 8 (or 2..7, a smaller grid on the same int8 path): kept columns quantized with one scale
+ *            for the whole call, scale_a = max|kept| / qmax, qmax = 2^(bits-1)-1, code =
+ *            clamp(rint(v * (qmax / max|kept|))); weights with one scale per output channel; int8 x int8
+ *            -> int32 contraction on tensor cores; y_wt = acc * (scale_a * scale_w[o]).
+ *            0: no quantization; columns and weights rounded to bf16, fp32 accumulation.
+ *   y   out: [N][Cout][H][Wd] of dt; must not overlap x
+ *   ws     : scratch of at least wcc_workspace_bytes(...) bytes; contents undefined afterwards
+ */
+wcc_status wcc_forward(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int Wd,
+                       int levels, int k, int bits, void* y, wcc_dtype dt,
+                       void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Intermediate results of wcc_forward for tests; any member may be NULL.  Row r = n * k + j is the
+ * j-th kept position of image n.  Rows of Xq / Xb are padded to kpad = wcc_kpad(Cin, bits) elements,
+ * the padding is zero.
+ */
+typedef struct wcc_taps {
+    float*   coef;      /* fp32 [N][Cin][P] */
+    float*   nrm2;      /* fp32 [N][P] */
+    int32_t* idx;       /* int32 [N][k] */
+    int8_t*  Xq;        /* int8 [N*k][kpad]           (bits >= 2) */
+    void*    Xb;        /* bf16 [N*k][kpad]           (bits == 0) */
+    float*   scale_a;   /* fp32 [1]                   (bits >= 2) */
+    int8_t*  Wq;        /* int8 [Cout][kpad]          (bits >= 2) */
+    float*   scale_w;   /* fp32 [Cout]                (bits >= 2) */
+    int32_t* acc;       /* int32 [N*k][Cout] (bits >= 2) or fp32 bit patterns of the products (bits == 0) */
+} wcc_taps;
+
+int wcc_kpad(int Cin, int bits);
+
+/* wcc_forward plus device-to-device copies of the requested intermediates (same kernels, same order). */
+wcc_status wcc_forward_debug(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int Wd,
+                             int levels, int k, int bits, void* y, wcc_dtype dt,
+                             void* ws, size_t ws_bytes, void* stream, const wcc_taps* taps);
+
+/*
+ * Synchronises `stream` and returns the device-side status word of the calling thread's current device:
+ * WCC_OK, or WCC_ERR_TIMEOUT if a bounded wait inside a kernel gave up (the output of that call is then
+ * undefined).  Reading clears the word.
+ */
+wcc_status wcc_last_status(void* stream);
+
+const char* wcc_status_str(wcc_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WCC_H_ */

@@ -1,0 +1,221 @@
+// libwcc: C-ABI entry points (see include/wcc.h).  One translation unit: the kernels live in the *.cuh files.
+#include "common.cuh"
+#include "haar.cuh"
+#include "select.cuh"
+#include "gather.cuh"
+#include "contract.cuh"
+
+namespace wcc {
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static wcc_status check_plane_args(int N, int C, int H, int W, int L, wcc_dtype dt)
+{
+    if (N <= 0 || C <= 0 || H <= 0 || W <= 0) return WCC_ERR_SHAPE;
+    if (L < 1 || L > 3) return WCC_ERR_SHAPE;
+    if ((H % (1 << L)) != 0 || (W % (1 << L)) != 0) return WCC_ERR_SHAPE;
+    if ((long long)N * C * H * W > (1LL << 40)) return WCC_ERR_SHAPE;
+    if ((long long)H * W > (1LL << 30)) return WCC_ERR_SHAPE;
+    if (dt != WCC_F32 && dt != WCC_BF16) return WCC_ERR_DTYPE;
+    return WCC_OK;
+}
+
+static wcc_status check_forward_args(int N, int Cin, int Cout, int H, int W, int L, int k, int bits, wcc_dtype dt)
+{
+    wcc_status s = check_plane_args(N, Cin, H, W, L, dt);
+    if (s != WCC_OK) return s;
+    if (Cout <= 0 || Cin > 256 || Cout > 256) return WCC_ERR_SHAPE;
+    if (k < 1 || (long long)k > (long long)H * W) return WCC_ERR_K;
+    if (!(bits == 0 || (bits >= 2 && bits <= 8))) return WCC_ERR_BITS;
+    if ((long long)N * k > (1LL << 30)) return WCC_ERR_SHAPE;
+    return WCC_OK;
+}
+
+struct FwdWs {
+    float* coef; float* nrm2; float* amaxpos; int32_t* rank; int32_t* idx; void* sel; size_t sel_bytes;
+    float* amax_kept; void* Xq; void* Wq; float* scale_w; int32_t* acc;
+    int kpad, ldc, es;
+    size_t total;
+};
+
+static FwdWs carve_forward_ws(void* ws, int N, int Cin, int Cout, int H, int W, int k, int bits)
+{
+    FwdWs f;
+    const size_t P = (size_t)H * W, M = (size_t)N * k;
+    f.kpad = wcc_kpad(Cin, bits);
+    f.es = (bits == 0) ? 2 : 1;
+    f.ldc = ceil_div(Cout, 4) * 4;
+    size_t off = 0;
+    char* b = static_cast<char*>(ws);
+    auto take = [&](size_t bytes) { char* p = b ? b + off : nullptr; off += align_up(bytes, 256); return p; };
+    f.coef = reinterpret_cast<float*>(take((size_t)N * Cin * P * 4));
+    f.nrm2 = reinterpret_cast<float*>(take((size_t)N * P * 4));
+    f.amaxpos = reinterpret_cast<float*>(take((size_t)N * P * 4));
+    f.rank = reinterpret_cast<int32_t*>(take((size_t)N * P * 4));
+    f.idx = reinterpret_cast<int32_t*>(take(M * 4));
+    f.sel_bytes = select_ws_bytes(N, (int)P);
+    f.sel = take(f.sel_bytes);
+    f.amax_kept = reinterpret_cast<float*>(take(256));
+    f.Xq = take(M * f.kpad * f.es);
+    f.Wq = take((size_t)Cout * f.kpad * f.es);
+    f.scale_w = reinterpret_cast<float*>(take((size_t)Cout * 4));
+    f.acc = reinterpret_cast<int32_t*>(take(M * f.ldc * 4));
+    f.total = off;
+    return f;
+}
+
+__global__ void scale_tap_kernel(const float* amax_kept, float qmax, float* out) { *out = __fdiv_rn(*amax_kept, qmax); }
+
+static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int W,
+                               int L, int k, int bits, void* y, wcc_dtype dt, void* ws, size_t ws_bytes,
+                               cudaStream_t st, const wcc_taps* taps)
+{
+    if (!x || !Wt || !y || !ws) return WCC_ERR_NULL;
+    wcc_status s = check_forward_args(N, Cin, Cout, H, W, L, k, bits, dt);
+    if (s != WCC_OK) return s;
+    if (!aligned16(x) || !aligned16(Wt) || !aligned16(y) || (reinterpret_cast<uintptr_t>(ws) & 255u)) return WCC_ERR_ALIGN;
+    const FwdWs f = carve_forward_ws(ws, N, Cin, Cout, H, W, k, bits);
+    if (ws_bytes < f.total) return WCC_ERR_WORKSPACE;
+    const int P = H * W, M = N * k;
+
+    // A: Haar transform + channel norms (and the per-position max |coef| the activation scale is taken from)
+    s = launch_haar_fwd(x, N, Cin, H, W, L, dt, f.coef, f.nrm2, f.amaxpos, st);
+    if (s != WCC_OK) return s;
+    // B: joint shrinkage: kept index list, rank map, max |kept|
+    s = launch_select(f.nrm2, N, P, k, f.idx, nullptr, f.rank, f.amaxpos, f.amax_kept, f.sel, f.sel_bytes, st);
+    if (s != WCC_OK) return s;
+    s = launch_weight_prep(Wt, Cout, Cin, f.kpad, bits, f.Wq, f.scale_w, st);
+    if (s != WCC_OK) return s;
+    s = launch_gather_quant(f.coef, f.idx, f.amax_kept, N, Cin, P, k, f.kpad, bits, f.Xq, st);
+    if (s != WCC_OK) return s;
+    // C: pointwise convolution on the compressed columns
+    s = launch_contract(f.Xq, f.Wq, M, Cout, f.kpad, bits, f.acc, f.ldc, st);
+    if (s != WCC_OK) return s;
+    // D + E: dequantize, zero-fill, inverse transform
+    s = launch_scatter_inv(f.acc, f.ldc, bits == 0, f.rank, f.amax_kept, bits, f.scale_w, N, Cout, H, W, L, k, dt, y, st);
+    if (s != WCC_OK) return s;
+
+    if (taps) {
+        const cudaMemcpyKind dd = cudaMemcpyDeviceToDevice;
+        if (taps->coef) WCC_CUDA_TRY(cudaMemcpyAsync(taps->coef, f.coef, (size_t)N * Cin * P * 4, dd, st));
+        if (taps->nrm2) WCC_CUDA_TRY(cudaMemcpyAsync(taps->nrm2, f.nrm2, (size_t)N * P * 4, dd, st));
+        if (taps->idx) WCC_CUDA_TRY(cudaMemcpyAsync(taps->idx, f.idx, (size_t)M * 4, dd, st));
+        if (bits >= 2) {
+            if (taps->Xq) WCC_CUDA_TRY(cudaMemcpyAsync(taps->Xq, f.Xq, (size_t)M * f.kpad, dd, st));
+            if (taps->Wq) WCC_CUDA_TRY(cudaMemcpyAsync(taps->Wq, f.Wq, (size_t)Cout * f.kpad, dd, st));
+            if (taps->scale_w) WCC_CUDA_TRY(cudaMemcpyAsync(taps->scale_w, f.scale_w, (size_t)Cout * 4, dd, st));
+            if (taps->scale_a) {
+                scale_tap_kernel<<<1, 1, 0, st>>>(f.amax_kept, (float)((1 << (bits - 1)) - 1), taps->scale_a);
+                WCC_LAUNCH_CHECK();
+            }
+        } else if (taps->Xb) {
+            WCC_CUDA_TRY(cudaMemcpyAsync(taps->Xb, f.Xq, (size_t)M * f.kpad * 2, dd, st));
+        }
+        if (taps->acc)
+            WCC_CUDA_TRY(cudaMemcpy2DAsync(taps->acc, (size_t)Cout * 4, f.acc, (size_t)f.ldc * 4, (size_t)Cout * 4, M, dd, st));
+    }
+    return WCC_OK;
+}
+
+}  // namespace wcc
+
+using namespace wcc;
+
+extern "C" {
+
+int wcc_kpad(int Cin, int bits)
+{
+    if (Cin <= 0) return 0;
+    return (bits == 0) ? ceil_div(Cin, 16) * 16 : ceil_div(Cin, 32) * 32;
+}
+
+size_t wcc_workspace_bytes(int N, int Cin, int Cout, int H, int Wd, int levels, int k, int bits, wcc_dtype dt)
+{
+    if (check_forward_args(N, Cin, Cout, H, Wd, levels, k, bits, dt) != WCC_OK) return 0;
+    return carve_forward_ws(nullptr, N, Cin, Cout, H, Wd, k, bits).total;
+}
+
+size_t wcc_select_workspace_bytes(int N, int P)
+{
+    if (N <= 0 || P <= 0) return 0;
+    return select_ws_bytes(N, P);
+}
+
+wcc_status wcc_haar_fwd(const void* x, int N, int C, int H, int Wd, int levels, wcc_dtype dt,
+                        float* coef, float* nrm2, void* stream)
+{
+    if (!x || !coef) return WCC_ERR_NULL;
+    wcc_status s = check_plane_args(N, C, H, Wd, levels, dt);
+    if (s != WCC_OK) return s;
+    if (!aligned16(x) || !aligned16(coef) || !aligned16(nrm2)) return WCC_ERR_ALIGN;
+    return launch_haar_fwd(x, N, C, H, Wd, levels, dt, coef, nrm2, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+wcc_status wcc_haar_inv(const float* coef, int N, int C, int H, int Wd, int levels, wcc_dtype dt,
+                        void* x_out, void* stream)
+{
+    if (!coef || !x_out) return WCC_ERR_NULL;
+    wcc_status s = check_plane_args(N, C, H, Wd, levels, dt);
+    if (s != WCC_OK) return s;
+    if (!aligned16(coef) || !aligned16(x_out)) return WCC_ERR_ALIGN;
+    return launch_haar_inv(coef, N, C, H, Wd, levels, dt, x_out, static_cast<cudaStream_t>(stream));
+}
+
+wcc_status wcc_select_topk(const float* nrm2, int N, int P, int k, int32_t* idx, float* tau,
+                           void* ws, size_t ws_bytes, void* stream)
+{
+    if (!nrm2 || !idx || !ws) return WCC_ERR_NULL;
+    if (N <= 0 || P <= 0 || N > 65535 || P > (1 << 30)) return WCC_ERR_SHAPE;
+    if (k < 1 || k > P) return WCC_ERR_K;
+    if (!aligned16(nrm2) || !aligned16(idx) || !aligned16(ws)) return WCC_ERR_ALIGN;
+    if (ws_bytes < select_ws_bytes(N, P)) return WCC_ERR_WORKSPACE;
+    return launch_select(nrm2, N, P, k, idx, tau, nullptr, nullptr, nullptr, ws, ws_bytes, static_cast<cudaStream_t>(stream));
+}
+
+wcc_status wcc_forward(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int Wd,
+                       int levels, int k, int bits, void* y, wcc_dtype dt,
+                       void* ws, size_t ws_bytes, void* stream)
+{
+    return forward_impl(x, Wt, N, Cin, Cout, H, Wd, levels, k, bits, y, dt, ws, ws_bytes,
+                        static_cast<cudaStream_t>(stream), nullptr);
+}
+
+wcc_status wcc_forward_debug(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int Wd,
+                             int levels, int k, int bits, void* y, wcc_dtype dt,
+                             void* ws, size_t ws_bytes, void* stream, const wcc_taps* taps)
+{
+    return forward_impl(x, Wt, N, Cin, Cout, H, Wd, levels, k, bits, y, dt, ws, ws_bytes,
+                        static_cast<cudaStream_t>(stream), taps);
+}
+
+wcc_status wcc_last_status(void* stream)
+{
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return WCC_ERR_CUDA;
+    int v = 0;
+    if (cudaMemcpyFromSymbol(&v, g_status, sizeof(int)) != cudaSuccess) return WCC_ERR_CUDA;
+    if (v != 0) {
+        const int zero = 0;
+        if (cudaMemcpyToSymbol(g_status, &zero, sizeof(int)) != cudaSuccess) return WCC_ERR_CUDA;
+    }
+    return static_cast<wcc_status>(v);
+}
+
+const char* wcc_status_str(wcc_status s)
+{
+    switch (s) {
+        case WCC_OK: return "ok";
+        case WCC_ERR_NULL: return "null pointer";
+        case WCC_ERR_SHAPE: return "bad shape";
+        case WCC_ERR_K: return "k out of range";
+        case WCC_ERR_BITS: return "bits not in {0, 2..8}";
+        case WCC_ERR_DTYPE: return "unknown dtype";
+        case WCC_ERR_ALIGN: return "misaligned pointer";
+        case WCC_ERR_WORKSPACE: return "workspace too small";
+        case WCC_ERR_CUDA: return "CUDA error";
+        case WCC_ERR_TIMEOUT: return "device wait timed out";
+        case WCC_ERR_NONFINITE: return "non-finite input";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

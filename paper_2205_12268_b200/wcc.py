@@ -1,0 +1,196 @@
+"""Thin binding over libwcc.so (the C ABI of include/wcc.h): argument marshalling only.
+
+Every step runs in the library's CUDA kernels; torch is used for device memory and the current stream.
+There is no fallback: if the library is missing, or a call returns an error code, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libwcc.so")
+
+F32, BF16 = 0, 1
+_STATUS = {0: "ok", 1: "null pointer", 2: "bad shape", 3: "k out of range", 4: "bad bits", 5: "bad dtype",
+           6: "misaligned pointer", 7: "workspace too small", 8: "CUDA error", 9: "device wait timed out",
+           10: "non-finite input"}
+
+EXPORTS = ("wcc_workspace_bytes", "wcc_select_workspace_bytes", "wcc_haar_fwd", "wcc_haar_inv", "wcc_select_topk",
+           "wcc_forward", "wcc_forward_debug", "wcc_kpad", "wcc_last_status", "wcc_status_str")
+
+
+class WccError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        super().__init__("%s: %s (status %d)" % (where, _STATUS.get(code, "?"), code))
+        self.code = code
+
+
+class Taps(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("coef", "nrm2", "idx", "Xq", "Xb", "scale_a", "Wq", "scale_w", "acc")]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """The loaded library; raises if it has not been built (``python -m paper_2205_12268_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError("libwcc.so is not built: run `python -m paper_2205_12268_b200.build` "
+                                    "(needs nvcc; there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        i, vp, sz = C.c_int, C.c_void_p, C.c_size_t
+        L.wcc_workspace_bytes.restype = sz
+        L.wcc_workspace_bytes.argtypes = [i] * 9
+        L.wcc_select_workspace_bytes.restype = sz
+        L.wcc_select_workspace_bytes.argtypes = [i, i]
+        L.wcc_kpad.restype = i
+        L.wcc_kpad.argtypes = [i, i]
+        L.wcc_haar_fwd.restype = i
+        L.wcc_haar_fwd.argtypes = [vp, i, i, i, i, i, i, vp, vp, vp]
+        L.wcc_haar_inv.restype = i
+        L.wcc_haar_inv.argtypes = [vp, i, i, i, i, i, i, vp, vp]
+        L.wcc_select_topk.restype = i
+        L.wcc_select_topk.argtypes = [vp, i, i, i, vp, vp, vp, sz, vp]
+        fwd = [vp, vp, i, i, i, i, i, i, i, i, vp, i, vp, sz, vp]
+        L.wcc_forward.restype = i
+        L.wcc_forward.argtypes = fwd
+        L.wcc_forward_debug.restype = i
+        L.wcc_forward_debug.argtypes = fwd + [C.POINTER(Taps)]
+        L.wcc_last_status.restype = i
+        L.wcc_last_status.argtypes = [vp]
+        L.wcc_status_str.restype = C.c_char_p
+        L.wcc_status_str.argtypes = [i]
+        _lib = L
+    return _lib
+
+
+def _check(code: int, where: str):
+    if code != 0:
+        raise WccError(code, where)
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError("activations must be float32 or bfloat16, got %s" % t.dtype)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def _dev(t: torch.Tensor, name: str):
+    if not (t.is_cuda and t.is_contiguous()):
+        raise ValueError("%s must be a contiguous CUDA tensor" % name)
+
+
+def workspace_bytes(N, Cin, Cout, H, W, levels, k, bits, dt) -> int:
+    return int(lib().wcc_workspace_bytes(N, Cin, Cout, H, W, levels, k, bits, dt))
+
+
+def kpad(Cin: int, bits: int) -> int:
+    return int(lib().wcc_kpad(Cin, bits))
+
+
+def haar_fwd(x: torch.Tensor, levels: int, want_norms: bool = True):
+    """x [N][C][H][W] -> (coef fp32 [N][C][H][W] quadrant layout, nrm2 fp32 [N][H*W] or None)."""
+    _dev(x, "x")
+    N, Cc, H, W = x.shape
+    coef = torch.empty((N, Cc, H, W), dtype=torch.float32, device=x.device)
+    nrm2 = torch.empty((N, H * W), dtype=torch.float32, device=x.device) if want_norms else None
+    _check(lib().wcc_haar_fwd(x.data_ptr(), N, Cc, H, W, levels, _dt(x), coef.data_ptr(), _ptr(nrm2), _stream()),
+           "wcc_haar_fwd")
+    return coef, nrm2
+
+
+def haar_inv(coef: torch.Tensor, levels: int, dtype: torch.dtype = torch.float32) -> torch.Tensor:
+    _dev(coef, "coef")
+    if coef.dtype != torch.float32:
+        raise TypeError("coef must be float32")
+    N, Cc, H, W = coef.shape
+    out = torch.empty((N, Cc, H, W), dtype=dtype, device=coef.device)
+    _check(lib().wcc_haar_inv(coef.data_ptr(), N, Cc, H, W, levels, _dt(out), out.data_ptr(), _stream()), "wcc_haar_inv")
+    return out
+
+
+def select_topk(nrm2: torch.Tensor, k: int):
+    """nrm2 fp32 [N][P] -> (idx int32 [N][k] ascending, tau fp32 [N])."""
+    _dev(nrm2, "nrm2")
+    if nrm2.dtype != torch.float32:
+        raise TypeError("nrm2 must be float32")
+    N, P = nrm2.shape
+    idx = torch.empty((N, max(k, 1)), dtype=torch.int32, device=nrm2.device)
+    tau = torch.empty((N,), dtype=torch.float32, device=nrm2.device)
+    nbytes = int(lib().wcc_select_workspace_bytes(N, P))
+    ws = torch.empty((max(nbytes, 256),), dtype=torch.uint8, device=nrm2.device)
+    _check(lib().wcc_select_topk(nrm2.data_ptr(), N, P, k, idx.data_ptr(), tau.data_ptr(), ws.data_ptr(), nbytes, _stream()),
+           "wcc_select_topk")
+    return idx, tau
+
+
+class Workspace:
+    """Caller-owned scratch for ``forward``; reuse it across calls of the same (or smaller) problem."""
+
+    def __init__(self, nbytes: int, device):
+        self.nbytes = int(nbytes)
+        self.buf = torch.empty((max(self.nbytes, 256),), dtype=torch.uint8, device=device)
+
+    @classmethod
+    def for_problem(cls, x: torch.Tensor, Cout: int, levels: int, k: int, bits: int):
+        N, Cin, H, W = x.shape
+        n = workspace_bytes(N, Cin, Cout, H, W, levels, k, bits, _dt(x))
+        if n == 0:
+            raise WccError(2, "wcc_workspace_bytes")
+        return cls(n, x.device)
+
+
+def forward(x: torch.Tensor, Wt: torch.Tensor, levels: int, k: int, bits: int = 8, y: torch.Tensor | None = None,
+            ws: Workspace | None = None, taps: bool = False):
+    """The WCC layer.  Returns y, or (y, dict of intermediate tensors) when ``taps`` is set."""
+    _dev(x, "x")
+    _dev(Wt, "Wt")
+    if Wt.dtype != torch.float32:
+        raise TypeError("Wt must be float32")
+    N, Cin, H, W = x.shape
+    Cout = Wt.shape[0]
+    if Wt.shape[1] != Cin:
+        raise ValueError("Wt must be [Cout][Cin]")
+    if y is None:
+        y = torch.empty((N, Cout, H, W), dtype=x.dtype, device=x.device)
+    if ws is None:
+        ws = Workspace.for_problem(x, Cout, levels, k, bits)
+    args = (x.data_ptr(), Wt.data_ptr(), N, Cin, Cout, H, W, levels, k, bits, y.data_ptr(), _dt(x),
+            ws.buf.data_ptr(), ws.nbytes, _stream())
+    if not taps:
+        _check(lib().wcc_forward(*args), "wcc_forward")
+        return y
+    P, M, kp = H * W, N * k, kpad(Cin, bits)
+    dev = x.device
+    t = dict(coef=torch.empty((N, Cin, P), dtype=torch.float32, device=dev),
+             nrm2=torch.empty((N, P), dtype=torch.float32, device=dev),
+             idx=torch.empty((N, k), dtype=torch.int32, device=dev),
+             acc=torch.empty((M, Cout), dtype=torch.int32, device=dev))
+    if bits >= 2:
+        t.update(Xq=torch.empty((M, kp), dtype=torch.int8, device=dev), scale_a=torch.empty((1,), dtype=torch.float32, device=dev),
+                 Wq=torch.empty((Cout, kp), dtype=torch.int8, device=dev), scale_w=torch.empty((Cout,), dtype=torch.float32, device=dev))
+    else:
+        t.update(Xb=torch.empty((M, kp), dtype=torch.bfloat16, device=dev))
+    s = Taps(**{name: _ptr(t.get(name)) for name, _ in Taps._fields_})
+    _check(lib().wcc_forward_debug(*args, C.byref(s)), "wcc_forward_debug")
+    return y, t
+
+
+def last_status() -> int:
+    """Synchronises the current stream and returns (and clears) the device status word."""
+    return int(lib().wcc_last_status(_stream()))
