@@ -139,6 +139,18 @@ wcc_status wcc_last_status(void* stream);
 
 const char* wcc_status_str(wcc_status s);
 
+/*
+ * Measurement helpers (no counterpart in the paper).  With profiling on, wcc_forward records CUDA events on its
+ * stream around each stage; wcc_profile_read waits for the last recorded call and writes, to the HOST array ms, the
+ * milliseconds of: 0 Haar transform + norms, 1 top-k select + compaction, 2 weight quantization, 3 gather + quantize,
+ * 4 tensor-core contraction, 5 dequantize + scatter + inverse Haar.  Off by default; not thread-safe.
+ */
+#define WCC_NUM_STAGES 6
+wcc_status wcc_profile_enable(int on);
+wcc_status wcc_profile_read(float* ms);
+/* Number of kernels this library has launched in this process so far (memset nodes not counted). */
+unsigned long long wcc_kernel_launches(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -22,8 +22,12 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
         if (e__ != cudaSuccess) return WCC_ERR_CUDA; \
     } while (0)
 
+// host-side count of kernel launches (reported by wcc_kernel_launches)
+static unsigned long long g_launches = 0;
+
 #define WCC_LAUNCH_CHECK()                                   \
     do {                                                     \
+        ++g_launches;                                        \
         if (cudaPeekAtLastError() != cudaSuccess) {          \
             (void)cudaGetLastError();                        \
             return WCC_ERR_CUDA;                             \

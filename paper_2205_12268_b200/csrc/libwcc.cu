@@ -64,6 +64,20 @@ static FwdWs carve_forward_ws(void* ws, int N, int Cin, int Cout, int H, int W, 
     return f;
 }
 
+// ---- optional stage timing ------------------------------------------------------------------
+static bool g_profile = false;
+static cudaEvent_t g_ev[WCC_NUM_STAGES + 1] = {nullptr};
+static bool g_ev_valid = false;
+
+static wcc_status profile_mark(int i, cudaStream_t st)
+{
+    if (!g_profile) return WCC_OK;
+    if (!g_ev[i]) WCC_CUDA_TRY(cudaEventCreate(&g_ev[i]));
+    WCC_CUDA_TRY(cudaEventRecord(g_ev[i], st));
+    if (i == WCC_NUM_STAGES) g_ev_valid = true;
+    return WCC_OK;
+}
+
 __global__ void scale_tap_kernel(const float* amax_kept, float qmax, float* out) { *out = __fdiv_rn(*amax_kept, qmax); }
 
 static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int W,
@@ -78,22 +92,29 @@ static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, i
     if (ws_bytes < f.total) return WCC_ERR_WORKSPACE;
     const int P = H * W, M = N * k;
 
+    if ((s = profile_mark(0, st)) != WCC_OK) return s;
     // A: Haar transform + channel norms (and the per-position max |coef| the activation scale is taken from)
     s = launch_haar_fwd(x, N, Cin, H, W, L, dt, f.coef, f.nrm2, f.amaxpos, st);
     if (s != WCC_OK) return s;
+    if ((s = profile_mark(1, st)) != WCC_OK) return s;
     // B: joint shrinkage: kept index list, rank map, max |kept|
     s = launch_select(f.nrm2, N, P, k, f.idx, nullptr, f.rank, f.amaxpos, f.amax_kept, f.sel, f.sel_bytes, st);
     if (s != WCC_OK) return s;
+    if ((s = profile_mark(2, st)) != WCC_OK) return s;
     s = launch_weight_prep(Wt, Cout, Cin, f.kpad, bits, f.Wq, f.scale_w, st);
     if (s != WCC_OK) return s;
+    if ((s = profile_mark(3, st)) != WCC_OK) return s;
     s = launch_gather_quant(f.coef, f.idx, f.amax_kept, N, Cin, P, k, f.kpad, bits, f.Xq, st);
     if (s != WCC_OK) return s;
+    if ((s = profile_mark(4, st)) != WCC_OK) return s;
     // C: pointwise convolution on the compressed columns
     s = launch_contract(f.Xq, f.Wq, M, Cout, f.kpad, bits, f.acc, f.ldc, st);
     if (s != WCC_OK) return s;
+    if ((s = profile_mark(5, st)) != WCC_OK) return s;
     // D + E: dequantize, zero-fill, inverse transform
     s = launch_scatter_inv(f.acc, f.ldc, bits == 0, f.rank, f.amax_kept, bits, f.scale_w, N, Cout, H, W, L, k, dt, y, st);
     if (s != WCC_OK) return s;
+    if ((s = profile_mark(6, st)) != WCC_OK) return s;
 
     if (taps) {
         const cudaMemcpyKind dd = cudaMemcpyDeviceToDevice;
@@ -199,6 +220,25 @@ wcc_status wcc_last_status(void* stream)
     }
     return static_cast<wcc_status>(v);
 }
+
+wcc_status wcc_profile_enable(int on)
+{
+    g_profile = on != 0;
+    if (!g_profile) g_ev_valid = false;
+    return WCC_OK;
+}
+
+wcc_status wcc_profile_read(float* ms)
+{
+    if (!ms) return WCC_ERR_NULL;
+    if (!g_ev_valid) return WCC_ERR_CUDA;
+    if (cudaEventSynchronize(g_ev[WCC_NUM_STAGES]) != cudaSuccess) return WCC_ERR_CUDA;
+    for (int i = 0; i < WCC_NUM_STAGES; ++i)
+        if (cudaEventElapsedTime(&ms[i], g_ev[i], g_ev[i + 1]) != cudaSuccess) return WCC_ERR_CUDA;
+    return WCC_OK;
+}
+
+unsigned long long wcc_kernel_launches(void) { return g_launches; }
 
 const char* wcc_status_str(wcc_status s)
 {

@@ -298,6 +298,7 @@ wcc_status launch_select(const float* nrm2, int N, int P, int k, int32_t* idx, f
     select_hist_kernel<3><<<grid, SEL_THREADS, 0, st>>>(nrm2, P, k, s.hist, s.state);
     select_count_kernel<<<grid, SEL_THREADS, 0, st>>>(nrm2, P, s.hist, s.state, s.chunkcnt, tau);
     select_compact_kernel<<<grid, SEL_THREADS, 0, st>>>(nrm2, P, k, s.state, s.chunkcnt, idx, rank, amaxpos, amax_kept);
+    g_launches += 4;
     WCC_LAUNCH_CHECK();
     return WCC_OK;
 }

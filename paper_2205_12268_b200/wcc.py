@@ -19,7 +19,9 @@ _STATUS = {0: "ok", 1: "null pointer", 2: "bad shape", 3: "k out of range", 4: "
            10: "non-finite input"}
 
 EXPORTS = ("wcc_workspace_bytes", "wcc_select_workspace_bytes", "wcc_haar_fwd", "wcc_haar_inv", "wcc_select_topk",
-           "wcc_forward", "wcc_forward_debug", "wcc_kpad", "wcc_last_status", "wcc_status_str")
+           "wcc_forward", "wcc_forward_debug", "wcc_kpad", "wcc_last_status", "wcc_status_str",
+           "wcc_profile_enable", "wcc_profile_read", "wcc_kernel_launches")
+STAGES = ("haar_fwd_norms", "select_topk", "weight_quant", "gather_quant", "contract", "scatter_inv")
 
 
 class WccError(RuntimeError):
@@ -63,6 +65,12 @@ def lib() -> C.CDLL:
         L.wcc_forward_debug.argtypes = fwd + [C.POINTER(Taps)]
         L.wcc_last_status.restype = i
         L.wcc_last_status.argtypes = [vp]
+        L.wcc_profile_enable.restype = i
+        L.wcc_profile_enable.argtypes = [i]
+        L.wcc_profile_read.restype = i
+        L.wcc_profile_read.argtypes = [C.POINTER(C.c_float)]
+        L.wcc_kernel_launches.restype = C.c_ulonglong
+        L.wcc_kernel_launches.argtypes = []
         L.wcc_status_str.restype = C.c_char_p
         L.wcc_status_str.argtypes = [i]
         _lib = L
@@ -194,3 +202,18 @@ def forward(x: torch.Tensor, Wt: torch.Tensor, levels: int, k: int, bits: int = 
 def last_status() -> int:
     """Synchronises the current stream and returns (and clears) the device status word."""
     return int(lib().wcc_last_status(_stream()))
+
+
+def profile_enable(on: bool):
+    _check(lib().wcc_profile_enable(int(on)), "wcc_profile_enable")
+
+
+def profile_read():
+    """Milliseconds of each stage (see ``STAGES``) of the last ``forward`` issued with profiling on."""
+    ms = (C.c_float * len(STAGES))()
+    _check(lib().wcc_profile_read(ms), "wcc_profile_read")
+    return [float(v) for v in ms]
+
+
+def kernel_launches() -> int:
+    return int(lib().wcc_kernel_launches())
