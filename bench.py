@@ -174,6 +174,27 @@ def _config_dict(w, args, **extra):
     return d
 
 
+# ------------------------------------------------------------------------------------------------ multi-rank helpers
+def rank_seed(rank: int) -> int:
+    """Rank r draws its own batch of the workload's shape: seed 0 on rank 0 (the named workload), r elsewhere."""
+    return rank
+
+
+def max_over_ranks(dist, ms: float, device) -> float:
+    """Device time of the slowest rank (the job is done when the last rank is)."""
+    if dist is None:
+        return ms
+    import torch
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gpix(world: int, pixels_per_rank: int, ms_per_step: float) -> float:
+    """Output pixels of all ranks per second, in Gpix/s (weak scaling: every rank processes pixels_per_rank)."""
+    return world * pixels_per_rank / (ms_per_step * 1e-3) / 1e9
+
+
 # ------------------------------------------------------------------------------------------------ our arm
 def run_ours(args):
     import numpy as np
@@ -201,7 +222,7 @@ def run_ours(args):
     wcc.lib()
 
     over = {"N": args.batch} if args.batch else {}
-    w = inputs.make(args.workload, seed=rank, **over)   # seed 0 on rank 0; other ranks draw their own batch
+    w = inputs.make(args.workload, seed=rank_seed(rank), **over)
     if w.dtype == "bf16":
         x_host = torch.from_numpy(w.x.view(np.int16)).view(torch.bfloat16).pin_memory()
     else:
@@ -272,13 +293,9 @@ def run_ours(args):
     t_wall = time.perf_counter() - t_wall0
     clocks = sampler.stop()
     assert wcc.last_status() == 0
-    total_ms = float(sum(ms))
-    if dist:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(dist, float(sum(ms)), dev)
     ms_per_step = total_ms / args.steps
-    value = world * pixels / (ms_per_step * 1e-3) / 1e9
+    value = whole_job_gpix(world, pixels, ms_per_step)
 
     if args.lean:                                       # profiling runs: the timed loop only
         if rank == 0:
@@ -299,12 +316,8 @@ def run_ours(args):
         e2e_step()
     torch.cuda.synchronize()
     e_ms = timed_loop(e2e_step, e2e_steps)
-    e_total = float(sum(e_ms))
-    if dist:
-        t = torch.tensor([e_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e_total = float(t.item())
-    e2e_val = world * pixels / (e_total / e2e_steps * 1e-3) / 1e9
+    e_total = max_over_ranks(dist, float(sum(e_ms)), dev)
+    e2e_val = whole_job_gpix(world, pixels, e_total / e2e_steps)
 
     # per-stage device times with CUDA events recorded inside the call, same launch configuration (eager)
     wcc.profile_enable(True)
