@@ -91,6 +91,25 @@ wcc_status wcc_select_topk(const float* nrm2, int N, int P, int k, int32_t* idx,
                            void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * wcc_select_topk without a scratch argument (the paper has no counterpart: this is a packaging variant).
+ * For callers that have no way to obtain scratch memory: code that runs where cudaMalloc must not be called
+ * (a latency-critical loop in which the allocator's implicit device synchronisation is unacceptable, or a host
+ * that has handed all device memory to a pool the caller cannot reach) and that receives only its input and
+ * output pointers.  The scratch is a fixed array inside the library's device image, WCC_STATIC_SCRATCH_BYTES
+ * large; every GPU that loads the library holds that much memory until the process exits.
+ *  - Same arguments, results and error codes as wcc_select_topk; additionally returns WCC_ERR_WORKSPACE when
+ *    wcc_select_workspace_bytes(N, P) exceeds WCC_STATIC_SCRATCH_BYTES (about 24 KB per image: N = 32 images do not fit).
+ *  - Calls no cudaMalloc / cudaFree and no allocating library routine.
+ *  - The first call on each device looks up the array's device address (with that device current); make that
+ *    first call before starting any stream capture.
+ *  - All calls on a device share the one array, and it keeps the previous call's contents; the entry point
+ *    clears the parts that must start at zero.  Two calls whose kernels overlap on the GPU (different streams
+ *    without ordering) race on it: order them.
+ */
+#define WCC_STATIC_SCRATCH_BYTES (512 * 1024)
+wcc_status wcc_select_topk_static(const float* nrm2, int N, int P, int k, int32_t* idx, float* tau, void* stream);
+
+/*
  * The whole layer (Eq. 9 in the order of Alg. 1).
  *   x   in : [N][Cin][H][Wd] of dt          Wt in: fp32 [Cout][Cin] (no bias)
  *   k      : kept positions per image (ceil(gamma * H * Wd))

@@ -64,6 +64,29 @@ static FwdWs carve_forward_ws(void* ws, int N, int Cin, int Cout, int H, int W, 
     return f;
 }
 
+// ---- scratch for wcc_select_topk_static ---------------------------------------------------------
+// Lives in the device image of this library on every GPU that loads it.  In host code the name below is only a
+// handle for the runtime; the device address is looked up once per device with cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char g_select_scratch[WCC_STATIC_SCRATCH_BYTES];
+
+static wcc_status static_scratch_ptr(void** out)
+{
+    static void* ptr_of_device[64] = {nullptr};
+    int dev = -1;
+    WCC_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return WCC_ERR_CUDA;
+    if (!ptr_of_device[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_select_scratch) != cudaSuccess || !p) {
+            (void)cudaGetLastError();
+            return WCC_ERR_CUDA;
+        }
+        ptr_of_device[dev] = p;
+    }
+    *out = ptr_of_device[dev];
+    return WCC_OK;
+}
+
 // ---- optional stage timing ------------------------------------------------------------------
 static bool g_profile = false;
 static cudaEvent_t g_ev[WCC_NUM_STAGES + 1] = {nullptr};
@@ -191,6 +214,21 @@ wcc_status wcc_select_topk(const float* nrm2, int N, int P, int k, int32_t* idx,
     if (!aligned16(nrm2) || !aligned16(idx) || !aligned16(ws)) return WCC_ERR_ALIGN;
     if (ws_bytes < select_ws_bytes(N, P)) return WCC_ERR_WORKSPACE;
     return launch_select(nrm2, N, P, k, idx, tau, nullptr, nullptr, nullptr, ws, ws_bytes, static_cast<cudaStream_t>(stream));
+}
+
+wcc_status wcc_select_topk_static(const float* nrm2, int N, int P, int k, int32_t* idx, float* tau, void* stream)
+{
+    if (!nrm2 || !idx) return WCC_ERR_NULL;
+    if (N <= 0 || P <= 0 || N > 65535 || P > (1 << 30)) return WCC_ERR_SHAPE;
+    if (k < 1 || k > P) return WCC_ERR_K;
+    if (!aligned16(nrm2) || !aligned16(idx)) return WCC_ERR_ALIGN;
+    const size_t need = select_ws_bytes(N, P);
+    if (need > (size_t)WCC_STATIC_SCRATCH_BYTES) return WCC_ERR_WORKSPACE;     // beyond the built-in scratch
+    void* scratch = nullptr;
+    wcc_status s = static_scratch_ptr(&scratch);                               // first call per device: address lookup
+    if (s != WCC_OK) return s;
+    // launch_select zeroes the histograms it accumulates into; everything else in the scratch is written before it is read
+    return launch_select(nrm2, N, P, k, idx, tau, nullptr, nullptr, nullptr, scratch, need, static_cast<cudaStream_t>(stream));
 }
 
 wcc_status wcc_forward(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int Wd,

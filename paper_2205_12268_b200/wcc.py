@@ -20,7 +20,8 @@ _STATUS = {0: "ok", 1: "null pointer", 2: "bad shape", 3: "k out of range", 4: "
 
 EXPORTS = ("wcc_workspace_bytes", "wcc_select_workspace_bytes", "wcc_haar_fwd", "wcc_haar_inv", "wcc_select_topk",
            "wcc_forward", "wcc_forward_debug", "wcc_kpad", "wcc_last_status", "wcc_status_str",
-           "wcc_profile_enable", "wcc_profile_read", "wcc_kernel_launches")
+           "wcc_profile_enable", "wcc_profile_read", "wcc_kernel_launches", "wcc_select_topk_static")
+STATIC_SCRATCH_BYTES = 512 * 1024
 STAGES = ("haar_fwd_norms", "select_topk", "weight_quant", "gather_quant", "contract", "scatter_inv")
 
 
@@ -58,6 +59,8 @@ def lib() -> C.CDLL:
         L.wcc_haar_inv.argtypes = [vp, i, i, i, i, i, i, vp, vp]
         L.wcc_select_topk.restype = i
         L.wcc_select_topk.argtypes = [vp, i, i, i, vp, vp, vp, sz, vp]
+        L.wcc_select_topk_static.restype = i
+        L.wcc_select_topk_static.argtypes = [vp, i, i, i, vp, vp, vp]
         fwd = [vp, vp, i, i, i, i, i, i, i, i, vp, i, vp, sz, vp]
         L.wcc_forward.restype = i
         L.wcc_forward.argtypes = fwd
@@ -144,6 +147,18 @@ def select_topk(nrm2: torch.Tensor, k: int):
     ws = torch.empty((max(nbytes, 256),), dtype=torch.uint8, device=nrm2.device)
     _check(lib().wcc_select_topk(nrm2.data_ptr(), N, P, k, idx.data_ptr(), tau.data_ptr(), ws.data_ptr(), nbytes, _stream()),
            "wcc_select_topk")
+    return idx, tau
+
+
+def select_topk_static(nrm2: torch.Tensor, k: int, idx: torch.Tensor, tau: torch.Tensor):
+    """``select_topk`` for callers that cannot provide scratch memory: the library's built-in scratch array is used
+    and nothing is allocated, here or in the library (the caller passes the output tensors).  Raises ``WccError``
+    with code 7 when N and P need more than ``STATIC_SCRATCH_BYTES``.  Calls on one device share the scratch, so
+    they must not overlap on the GPU."""
+    _dev(nrm2, "nrm2")
+    N, P = nrm2.shape
+    _check(lib().wcc_select_topk_static(nrm2.data_ptr(), N, P, k, idx.data_ptr(), tau.data_ptr(), _stream()),
+           "wcc_select_topk_static")
     return idx, tau
 
 
