@@ -57,6 +57,8 @@ def stage_bytes(w, stage: str) -> float:
     NP, Nk = w.N * w.P, w.N * w.k
     es = 2 if w.bits == 0 else 1
     return {
+        "haar_norms": NP * w.Cin * s + 8 * NP,                                  # x once; norms and per-position max out
+        "fused_pass2": NP * w.Cin * s + 4 * NP + s * NP * w.Cout,               # x again, rank map, y once
         "haar_fwd_norms": NP * w.Cin * (s + 4) + 4 * NP,
         "select_topk": 4 * NP + 4 * Nk,
         "weight_quant": w.Cout * w.Cin * (4 + es),
@@ -231,12 +233,12 @@ def run_ours(args):
     Wt = torch.from_numpy(w.Wt).to(dev)
     y = torch.empty((w.N, w.Cout, w.H, w.W), dtype=x.dtype, device=dev)
     y_host = torch.empty(y.shape, dtype=y.dtype).pin_memory()
-    ws = wcc.Workspace.for_problem(x, w.Cout, w.levels, w.k, w.bits)
+    ws = wcc.Workspace.for_problem(x, w.Cout, w.levels, w.k, w.bits, staged=args.staged)
     flush = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device=dev)
     pixels = w.N * w.H * w.W
 
     def step_eager():
-        wcc.forward(x, Wt, w.levels, w.k, w.bits, y=y, ws=ws)
+        wcc.forward(x, Wt, w.levels, w.k, w.bits, y=y, ws=ws, staged=args.staged)
 
     # one eager call first: sets kernel attributes, counts launches
     l0 = wcc.kernel_launches()
@@ -308,7 +310,7 @@ def run_ours(args):
     # end to end through the public call: host input -> device, layer, device -> host output, every step
     def e2e_step():
         x.copy_(x_host, non_blocking=True)
-        wcc.forward(x, Wt, w.levels, w.k, w.bits, y=y, ws=ws)
+        wcc.forward(x, Wt, w.levels, w.k, w.bits, y=y, ws=ws, staged=args.staged)
         y_host.copy_(y, non_blocking=True)
 
     e2e_steps = min(args.steps, 200)
@@ -322,6 +324,7 @@ def run_ours(args):
     # per-stage device times with CUDA events recorded inside the call, same launch configuration (eager)
     wcc.profile_enable(True)
     prof_steps = min(args.steps, 200)
+    names = wcc.STAGES if args.staged else wcc.FUSED_STAGES
     acc = [0.0] * len(wcc.STAGES)
     for _ in range(prof_steps):
         flush.fill_(1)
@@ -329,7 +332,7 @@ def run_ours(args):
         for i, v in enumerate(wcc.profile_read()):
             acc[i] += v
     wcc.profile_enable(False)
-    stage_ms = {n: acc[i] / prof_steps for i, n in enumerate(wcc.STAGES)}
+    stage_ms = {n: acc[i] / prof_steps for i, n in enumerate(names)}
     dom = max(stage_ms, key=stage_ms.get)
     peak, peak_kind = _peaks()
     achieved = stage_bytes(w, dom) / (stage_ms[dom] * 1e-3) / 1e9
@@ -379,7 +382,8 @@ def run_ours(args):
            "dtype": "f32 transform, int8 x int8 -> int32 contraction" if w.bits else "f32 transform, bf16 contraction",
            "data": "synthetic",
            "config": _config_dict(w, args, l2="flushed before every step by a %d MiB write outside the step's events" % (FLUSH_BYTES >> 20),
-                                  launch="CUDA graph replay of one wcc_forward" if graph is not None else "eager wcc_forward",
+                                  launch=("CUDA graph replay of one %s" if graph is not None else "eager %s") % (
+                                      "wcc_forward_staged" if args.staged else "wcc_forward"),
                                   wall_s_timed_region=t_wall),
            "clocks": clocks,
            "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": x_host.numel() * x_host.element_size(),
@@ -404,6 +408,7 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="time eager wcc_forward calls instead of a graph replay")
     ap.add_argument("--batch", type=int, default=0, help="override the number of images per GPU")
     ap.add_argument("--lean", action="store_true", help="timed loop only (for runs under a profiler)")
+    ap.add_argument("--staged", action="store_true", help="time wcc_forward_staged (every intermediate in memory)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

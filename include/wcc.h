@@ -53,6 +53,8 @@ typedef enum { WCC_F32 = 0, WCC_BF16 = 1 } wcc_dtype;   /* element type of activ
 
 /* Scratch bytes wcc_forward / wcc_forward_debug need for these arguments (0 on invalid arguments). */
 size_t wcc_workspace_bytes(int N, int Cin, int Cout, int H, int Wd, int levels, int k, int bits, wcc_dtype dt);
+/* Scratch bytes wcc_forward_staged needs (it materialises the coefficient map, the compressed matrix and the accumulators). */
+size_t wcc_staged_workspace_bytes(int N, int Cin, int Cout, int H, int Wd, int levels, int k, int bits, wcc_dtype dt);
 
 /* Scratch bytes wcc_select_topk needs. */
 size_t wcc_select_workspace_bytes(int N, int P);
@@ -119,7 +121,12 @@ wcc_status wcc_select_topk_static(const float* nrm2, int N, int P, int k, int32_
  *            -> int32 contraction on tensor cores; y_wt = acc * (scale_a * scale_w[o]).
  *            0: no quantization; columns and weights rounded to bf16, fp32 accumulation.
  *   y   out: [N][Cout][H][Wd] of dt; must not overlap x
- *   ws     : scratch of at least wcc_workspace_bytes(...) bytes; contents undefined afterwards
+ *   ws     : scratch of at least wcc_workspace_bytes(...) bytes, 256-byte aligned; contents undefined afterwards
+ * Execution: two passes over x around the selection.  Pass 1 transforms x in registers and keeps only the channel
+ * norms and the per-position max |coefficient|; the selection yields the index list, the rank of every position in
+ * it and max|kept|; pass 2 transforms x again, zeroes the dropped positions, quantizes into shared memory, runs the
+ * contraction on tensor cores, dequantizes, applies the inverse transform and stores y.  The results are those of
+ * the step-by-step definition above (same integers, same fp32 operation order).
  */
 wcc_status wcc_forward(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int Wd,
                        int levels, int k, int bits, void* y, wcc_dtype dt,
@@ -144,10 +151,24 @@ typedef struct wcc_taps {
 
 int wcc_kpad(int Cin, int bits);
 
-/* wcc_forward plus device-to-device copies of the requested intermediates (same kernels, same order). */
+/*
+ * wcc_forward with the requested intermediates written out by the same kernels (the transform kernel also stores
+ * the coefficient map, the fused kernel also stores the codes and accumulators of the kept rows).
+ * Tap pointers must be 16-byte aligned.
+ */
 wcc_status wcc_forward_debug(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int Wd,
                              int levels, int k, int bits, void* y, wcc_dtype dt,
                              void* ws, size_t ws_bytes, void* stream, const wcc_taps* taps);
+
+/*
+ * The same layer as wcc_forward computed stage by stage with every intermediate in memory (Alg. 1 literally):
+ * transform + norms -> select -> gather + quantize -> tensor-core contraction on the compressed matrix ->
+ * dequantize + scatter + inverse.  Same results as wcc_forward; used to measure the stages one by one and as a
+ * cross-check.  ws: at least wcc_staged_workspace_bytes(...) bytes.  taps may be NULL.
+ */
+wcc_status wcc_forward_staged(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int Wd,
+                              int levels, int k, int bits, void* y, wcc_dtype dt,
+                              void* ws, size_t ws_bytes, void* stream, const wcc_taps* taps);
 
 /*
  * Synchronises `stream` and returns the device-side status word of the calling thread's current device:
@@ -161,8 +182,10 @@ const char* wcc_status_str(wcc_status s);
 /*
  * Measurement helpers (no counterpart in the paper).  With profiling on, wcc_forward records CUDA events on its
  * stream around each stage; wcc_profile_read waits for the last recorded call and writes, to the HOST array ms, the
- * milliseconds of: 0 Haar transform + norms, 1 top-k select + compaction, 2 weight quantization, 3 gather + quantize,
- * 4 tensor-core contraction, 5 dequantize + scatter + inverse Haar.  Off by default; not thread-safe.
+ * milliseconds of, for wcc_forward_staged: 0 Haar transform + norms, 1 top-k select + compaction, 2 weight
+ * quantization, 3 gather + quantize, 4 tensor-core contraction, 5 dequantize + scatter + inverse Haar; for wcc_forward:
+ * 0 transform + norms (pass 1), 1 select, 2 weight quantization, 3 fused pass 2, 4 and 5 zero.  Off by default; not
+ * thread-safe.
  */
 #define WCC_NUM_STAGES 6
 wcc_status wcc_profile_enable(int on);

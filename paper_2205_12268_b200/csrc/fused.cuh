@@ -1,0 +1,298 @@
+// Second pass of the fused layer: for one warp tile of one image, recompute the Haar transform from x, keep the
+// selected positions (zero the others), quantize, run the pointwise convolution on tensor cores, dequantize,
+// apply the inverse transform and store y (steps A, C, D, E of the WCC workflow, Eq. 9 / Alg. 1, with the index
+// set and the activation scale of step B already known).  Neither the coefficient map, nor the compressed matrix,
+// nor the accumulators, nor the zero-filled map ever reach HBM.
+//
+// One CTA = 4 warps = one warp tile (32 lanes x 8 slots = 256 wavelet-domain positions, see haar.cuh).
+//  phase 1  the four warps split the input channels in units of 8; every lane transforms its 2x4 patch of each
+//           channel in registers and writes the eight quantized (or bf16) slot values into the A operand in shared
+//           memory.  Row of a position in A: slot * 32 + lane, so one MMA block of 128 rows is four slots.
+//           Dropped positions are written as zeros: their accumulators are zero, which is the zero-filled map.
+//  phase 2  one thread issues tcgen05.mma (kind::i8, int32 accumulate; or kind::f16 on bf16, fp32 accumulate):
+//           D[256 x Cout] = A[256 x Cin] * Wq[Cout x Cin]^T, two M blocks, output channels in chunks of <= 64.
+//  phase 3  warp w reads TMEM lane quarter w (slots w and w+4 of all lanes) with tcgen05.ld, dequantizes and
+//           transposes through shared memory so that every lane gets its own eight slots back; inverse transform
+//           by warp shuffles, stores of y.
+// Operands use the no-swizzle K-major core-matrix layout (8 rows x 16 bytes contiguous): element (row, 16-byte
+// K chunk j) at j * rows * 16 + row * 16, i.e. leading (K) offset rows*16 bytes, stride (M/N) offset 128 bytes.
+// The single mbarrier wait is bounded and reports WCC_ERR_TIMEOUT.
+#pragma once
+
+#include "common.cuh"
+#include "contract.cuh"
+#include "haar.cuh"
+
+namespace wcc {
+namespace fz {
+
+constexpr int ROWS = 256;            // positions per CTA
+constexpr int SUB = 8;               // output channels per transpose round
+constexpr float MAGIC = 12582912.0f; // 1.5 * 2^23: adding it rounds to the nearest integer, ties to even
+
+__device__ __forceinline__ uint64_t smem_desc_plain(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    const uint32_t lo = ((addr & 0x3FFFFu) >> 4) | ((lbo_bytes >> 4) << 16);
+    const uint32_t hi = (sbo_bytes >> 4) | (1u << 14);      // version 1, layout type 0 (no swizzle)
+    return ((uint64_t)hi << 32) | lo;
+}
+
+__device__ __forceinline__ void tmem_ld8_nowait(uint32_t taddr, uint32_t (&r)[8])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr));
+}
+
+struct Ctl {
+    uint64_t mma_done;
+    uint32_t tmem_base;
+    int pad;
+};
+
+template <typename T, int L, bool VEC, bool I8>
+__global__ void __launch_bounds__(128, 4)
+fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, const int32_t* __restrict__ rank,
+                   const float* __restrict__ amax_kept, float qmax, const float* __restrict__ scale_w,
+                   int N, int Cin, int Cout, int H, int W, int k, int kpad, int npad, int nchunk, int tmem_cols,
+                   T* __restrict__ y, uint8_t* __restrict__ xq_tap, int32_t* __restrict__ acc_tap, int* __restrict__ status)
+{
+    using TT = HaarTile<L>;
+    constexpr int ES = I8 ? 1 : 2;                    // operand element size
+    constexpr int UNIT_BYTES = 8 * ES;                // 8 channels of one position
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = tc::smem_u32(smem_raw);
+    const uint32_t base = (raw + 127u) & ~127u;
+    uint8_t* sm = smem_raw + (base - raw);
+    const int krow = kpad * ES;                       // bytes of K per row
+    const int kchunks = krow / 16;
+    uint8_t* sA = sm;                                                   // [kchunks][256][16]
+    uint8_t* sB = sA + (size_t)kchunks * ROWS * 16;                     // [kchunks][npad][16]
+    float* stage = reinterpret_cast<float*>(sB + (size_t)kchunks * npad * 16);   // [SUB][8][32]
+    int32_t* srank = reinterpret_cast<int32_t*>(stage + SUB * 8 * 32);  // [8][32]
+    Ctl* ctl = reinterpret_cast<Ctl*>(srank + 8 * 32);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tiles_x = (W + TT::TW - 1) / TT::TW, tiles_y = H / TT::TH;
+    int n, ty, tx;
+    tile_coords(blockIdx.x, tiles_x, tiles_y, n, ty, tx);
+    const LanePos lp = lane_positions<L>(H, W, ty, tx, lane);
+    const size_t P = (size_t)H * W;
+
+    // ---- phase 0: barrier, TMEM, ranks, weights ---------------------------------------------------
+    if (threadIdx.x == 0) {
+        tc::mbar_init(tc::smem_u32(&ctl->mma_done), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(tc::smem_u32(&ctl->tmem_base)), "r"((uint32_t)tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    int rk[8];
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+        rk[s] = slot_ok<L>(lp, s) ? rank[(size_t)n * P + lp.pos[s]] : -1;
+        if (warp == 0) srank[s * 32 + lane] = rk[s];
+    }
+    for (int i = threadIdx.x; i < npad * kchunks; i += 128) {
+        const int row = i / kchunks, j = i - row * kchunks;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (row < Cout) v = *reinterpret_cast<const uint4*>(Wq + (size_t)row * krow + j * 16);
+        *reinterpret_cast<uint4*>(sB + ((size_t)j * npad + row) * 16) = v;
+    }
+    float inv = 0.0f, scale_a = 1.0f;
+    if (I8) {
+        const float amax = *amax_kept;
+        inv = (amax > 0.0f) ? __fdiv_rn(qmax, amax) : 0.0f;
+        scale_a = __fdiv_rn(amax, qmax);
+    } else {
+        inv = 1.0f;
+    }
+    float mul[8];                      // per slot: the quantization factor, or 0 for a dropped position
+#pragma unroll
+    for (int s = 0; s < 8; ++s) mul[s] = (rk[s] >= 0) ? inv : 0.0f;
+
+    // ---- phase 1: transform + quantize into the A operand --------------------------------------------
+    const T* xin = x + (size_t)n * Cin * P;
+    const int units = kpad / 8;
+    for (int u = warp; u < units; u += 4) {
+        RawPatch rawp[8];
+#pragma unroll
+        for (int d = 0; d < 8; ++d) {
+            const int c = u * 8 + d;
+            if (c < Cin) load_patch<T, VEC>(xin + (size_t)c * P, W, lp, rawp[d]);
+        }
+        uint32_t packed[8][4];         // per slot: 8 int8 codes (2 words) or 8 bf16 values (4 words)
+        float prev[8];
+#pragma unroll
+        for (int d = 0; d < 8; ++d) {
+            const int c = u * 8 + d;
+            float o[8];
+            if (c < Cin) {             // warp-uniform
+                float p[2][4];
+                unpack_patch<T>(rawp[d], p);
+                haar_fwd_lane<L>(p, o, lane);
+            } else {
+#pragma unroll
+                for (int s = 0; s < 8; ++s) o[s] = 0.0f;
+            }
+#pragma unroll
+            for (int s = 0; s < 8; ++s) {
+                const float t = __fmul_rn(o[s], mul[s]);
+                if (I8) {
+                    // low byte of (t + 1.5*2^23) is the two's complement code of rint(t); |t| <= qmax by construction
+                    const uint32_t code = __float_as_uint(__fadd_rn(t, MAGIC));
+                    if ((d & 3) == 0) packed[s][d >> 2] = code & 0xFFu;
+                    else packed[s][d >> 2] |= (code & 0xFFu) << (8 * (d & 3));
+                } else {
+                    if ((d & 1) == 0) prev[s] = t;
+                    else packed[s][d >> 1] = pack_bf16x2(prev[s], t);
+                }
+            }
+        }
+        const int j = (u * UNIT_BYTES) >> 4;               // 16-byte K chunk
+        const int off = (u * UNIT_BYTES) & 15;             // 0 or 8 (int8); always 0 (bf16)
+#pragma unroll
+        for (int s = 0; s < 8; ++s) {
+            uint8_t* dst = sA + ((size_t)j * ROWS + s * 32 + lane) * 16 + off;
+            if (I8) *reinterpret_cast<uint2*>(dst) = make_uint2(packed[s][0], packed[s][1]);
+            else *reinterpret_cast<uint4*>(dst) = make_uint4(packed[s][0], packed[s][1], packed[s][2], packed[s][3]);
+            if (xq_tap && rk[s] >= 0) {
+                uint8_t* g = xq_tap + ((size_t)n * k + rk[s]) * krow + (size_t)u * UNIT_BYTES;
+                if (I8) *reinterpret_cast<uint2*>(g) = make_uint2(packed[s][0], packed[s][1]);
+                else *reinterpret_cast<uint4*>(g) = make_uint4(packed[s][0], packed[s][1], packed[s][2], packed[s][3]);
+            }
+        }
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic-proxy writes -> visible to the tensor core
+    tc::fence_before();
+    __syncthreads();
+    tc::fence_after();
+    const uint32_t tmem = ctl->tmem_base;
+
+    // ---- phases 2 + 3, per chunk of output channels -------------------------------------------------
+    const int ksteps = krow / 32;
+    const uint32_t a_addr = tc::smem_u32(sA), b_addr = tc::smem_u32(sB);
+    volatile int no_abort = 0;
+    int chunk = 0;
+    bool ok = true;
+    for (int n0 = 0; n0 < npad; n0 += nchunk, ++chunk) {
+        const int cur = min(nchunk, npad - n0);
+        if (threadIdx.x == 0) {
+            const uint32_t idesc = (I8 ? (2u << 4) : (1u << 4)) | (1u << 7) | (1u << 10) |
+                                   ((uint32_t)(cur >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+            for (int b = 0; b < 2; ++b) {
+                for (int kk = 0; kk < ksteps; ++kk) {
+                    const uint64_t ad = smem_desc_plain(a_addr + (uint32_t)(kk * 2 * ROWS * 16 + b * 128 * 16), ROWS * 16, 128);
+                    const uint64_t bd = smem_desc_plain(b_addr + (uint32_t)(kk * 2 * npad * 16 + n0 * 16), (uint32_t)npad * 16, 128);
+                    tc::mma_ss<I8>(tmem + (uint32_t)(b * nchunk), ad, bd, idesc, kk > 0 ? 1u : 0u);
+                }
+            }
+            tc::mma_commit(tc::smem_u32(&ctl->mma_done));
+        }
+        ok = tc::mbar_wait(tc::smem_u32(&ctl->mma_done), (uint32_t)chunk & 1u, &no_abort);
+        ok = __syncthreads_and(ok ? 1 : 0) != 0;
+        if (!ok) break;
+        tc::fence_after();
+
+        for (int s0 = 0; s0 < cur; s0 += SUB) {
+            uint32_t r0[8], r1[8];
+            const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)s0;
+            tmem_ld8_nowait(taddr, r0);                              // slot `warp`
+            tmem_ld8_nowait(taddr + (uint32_t)nchunk, r1);           // slot `warp + 4`
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            const int rka = srank[warp * 32 + lane], rkb = srank[(warp + 4) * 32 + lane];
+#pragma unroll
+            for (int j = 0; j < SUB; ++j) {
+                const int o = n0 + s0 + j;
+                float fa, fb;
+                if (I8) {
+                    const float sc = (o < Cout) ? __fmul_rn(scale_a, scale_w[o]) : 0.0f;
+                    // exact int -> float for |acc| < 2^22: bits(1.5*2^23) + acc, minus 1.5*2^23
+                    fa = __fmul_rn(__fsub_rn(__uint_as_float(0x4B400000u + r0[j]), MAGIC), sc);
+                    fb = __fmul_rn(__fsub_rn(__uint_as_float(0x4B400000u + r1[j]), MAGIC), sc);
+                } else {
+                    fa = __uint_as_float(r0[j]);
+                    fb = __uint_as_float(r1[j]);
+                }
+                stage[(j * 8 + warp) * 32 + lane] = fa;
+                stage[(j * 8 + warp + 4) * 32 + lane] = fb;
+                if (acc_tap && o < Cout) {
+                    if (rka >= 0) acc_tap[((size_t)n * k + rka) * Cout + o] = (int32_t)r0[j];
+                    if (rkb >= 0) acc_tap[((size_t)n * k + rkb) * Cout + o] = (int32_t)r1[j];
+                }
+            }
+            __syncthreads();
+#pragma unroll
+            for (int jj = 0; jj < SUB / 4; ++jj) {
+                const int j = warp + 4 * jj;
+                const int o = n0 + s0 + j;
+                if (o < Cout) {                                      // warp-uniform
+                    float sl[8], p[2][4];
+#pragma unroll
+                    for (int s = 0; s < 8; ++s) sl[s] = stage[(j * 8 + s) * 32 + lane];
+                    haar_inv_lane<L>(sl, p, lane);
+                    store_patch<T, VEC>(y + ((size_t)n * Cout + o) * P, W, lp, p);
+                }
+            }
+            __syncthreads();
+        }
+        tc::fence_before();
+        __syncthreads();
+    }
+    if (!ok && threadIdx.x == 0) atomicExch(status, (int)WCC_ERR_TIMEOUT);
+    tc::fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc::fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)tmem_cols) : "memory");
+    }
+}
+
+}  // namespace fz
+
+template <typename T, int L, bool VEC>
+static wcc_status fused_pass2_dispatch(const void* x, const void* Wq, const int32_t* rank, const float* amax_kept, int bits,
+                                       const float* scale_w, int N, int Cin, int Cout, int H, int W, int k, int kpad,
+                                       void* y, void* xq_tap, int32_t* acc_tap, cudaStream_t st)
+{
+    using TT = HaarTile<L>;
+    const bool i8 = bits >= 2;
+    const int es = i8 ? 1 : 2;
+    const int npad = ceil_div(Cout, 16) * 16;
+    const int nchunk = npad < 64 ? npad : 64;
+    int tmem_cols = 32;
+    while (tmem_cols < 2 * nchunk) tmem_cols <<= 1;
+    const int kchunks = kpad * es / 16;
+    const size_t smem = 128 + (size_t)kchunks * fz::ROWS * 16 + (size_t)kchunks * npad * 16 + fz::SUB * 8 * 32 * 4 +
+                        8 * 32 * 4 + sizeof(fz::Ctl) + 16;
+    if (smem > 200 * 1024 || (kpad * es) % 32 != 0) return WCC_ERR_SHAPE;
+    const float qmax = i8 ? (float)((1 << (bits - 1)) - 1) : 1.0f;
+    int* status = nullptr;
+    WCC_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_status));
+    const long long ctas = (long long)N * ceil_div(W, TT::TW) * (H / TT::TH);
+    if (ctas > 0x7FFFFFFFLL) return WCC_ERR_SHAPE;
+    auto launch = [&](auto kern) -> wcc_status {
+        WCC_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+        kern<<<(unsigned)ctas, 128, smem, st>>>(static_cast<const T*>(x), static_cast<const uint8_t*>(Wq), rank, amax_kept, qmax,
+                                                scale_w, N, Cin, Cout, H, W, k, kpad, npad, nchunk, tmem_cols,
+                                                static_cast<T*>(y), static_cast<uint8_t*>(xq_tap), acc_tap, status);
+        WCC_LAUNCH_CHECK();
+        return WCC_OK;
+    };
+    if (i8) return launch(fz::fused_pass2_kernel<T, L, VEC, true>);
+    return launch(fz::fused_pass2_kernel<T, L, VEC, false>);
+}
+
+// Fused second pass.  xq_tap ([N*k][kpad] of int8 or bf16) and acc_tap (int32 [N*k][Cout]) may be NULL.
+wcc_status launch_fused_pass2(const void* x, const void* Wq, const int32_t* rank, const float* amax_kept, int bits,
+                              const float* scale_w, int N, int Cin, int Cout, int H, int W, int L, int k, int kpad,
+                              wcc_dtype dt, void* y, void* xq_tap, int32_t* acc_tap, cudaStream_t st)
+{
+    const bool vec = (W % 4) == 0;
+    WCC_DISPATCH_TLV(fused_pass2_dispatch, dt, L, vec, x, Wq, rank, amax_kept, bits, scale_w, N, Cin, Cout, H, W, k, kpad,
+                     y, xq_tap, acc_tap, st);
+}
+
+}  // namespace wcc

@@ -4,6 +4,7 @@
 #include "select.cuh"
 #include "gather.cuh"
 #include "contract.cuh"
+#include "fused.cuh"
 
 namespace wcc {
 
@@ -103,7 +104,7 @@ static wcc_status profile_mark(int i, cudaStream_t st)
 
 __global__ void scale_tap_kernel(const float* amax_kept, float qmax, float* out) { *out = __fdiv_rn(*amax_kept, qmax); }
 
-static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int W,
+static wcc_status staged_impl(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int W,
                                int L, int k, int bits, void* y, wcc_dtype dt, void* ws, size_t ws_bytes,
                                cudaStream_t st, const wcc_taps* taps)
 {
@@ -161,6 +162,87 @@ static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, i
     return WCC_OK;
 }
 
+// ---- fused path ----------------------------------------------------------------------------------
+struct FusedWs {
+    float* nrm2; float* amaxpos; int32_t* rank; int32_t* idx; void* sel; size_t sel_bytes;
+    float* amax_kept; void* Wq; float* scale_w;
+    int kpad, es;
+    size_t total;
+};
+
+static FusedWs carve_fused_ws(void* ws, int N, int Cin, int Cout, int H, int W, int k, int bits)
+{
+    FusedWs f;
+    const size_t P = (size_t)H * W, M = (size_t)N * k;
+    f.kpad = wcc_kpad(Cin, bits);
+    f.es = (bits == 0) ? 2 : 1;
+    size_t off = 0;
+    char* b = static_cast<char*>(ws);
+    auto take = [&](size_t bytes) { char* p = b ? b + off : nullptr; off += align_up(bytes, 256); return p; };
+    f.nrm2 = reinterpret_cast<float*>(take((size_t)N * P * 4));
+    f.amaxpos = reinterpret_cast<float*>(take((size_t)N * P * 4));
+    f.rank = reinterpret_cast<int32_t*>(take((size_t)N * P * 4));
+    f.idx = reinterpret_cast<int32_t*>(take(M * 4));
+    f.sel_bytes = select_ws_bytes(N, (int)P);
+    f.sel = take(f.sel_bytes);
+    f.amax_kept = reinterpret_cast<float*>(take(256));
+    f.Wq = take((size_t)Cout * f.kpad * f.es);
+    f.scale_w = reinterpret_cast<float*>(take((size_t)Cout * 4));
+    f.total = off;
+    return f;
+}
+
+static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int W,
+                               int L, int k, int bits, void* y, wcc_dtype dt, void* ws, size_t ws_bytes,
+                               cudaStream_t st, const wcc_taps* taps)
+{
+    if (!x || !Wt || !y || !ws) return WCC_ERR_NULL;
+    wcc_status s = check_forward_args(N, Cin, Cout, H, W, L, k, bits, dt);
+    if (s != WCC_OK) return s;
+    if (!aligned16(x) || !aligned16(Wt) || !aligned16(y) || (reinterpret_cast<uintptr_t>(ws) & 255u)) return WCC_ERR_ALIGN;
+    if (taps && (!aligned16(taps->coef) || !aligned16(taps->Xq) || !aligned16(taps->Xb) || !aligned16(taps->acc)))
+        return WCC_ERR_ALIGN;
+    const FusedWs f = carve_fused_ws(ws, N, Cin, Cout, H, W, k, bits);
+    if (ws_bytes < f.total) return WCC_ERR_WORKSPACE;
+    const int P = H * W, M = N * k;
+
+    if ((s = profile_mark(0, st)) != WCC_OK) return s;
+    // first pass over x: transform in registers, keep only the channel norms and the per-position max |coef|
+    // (the coefficient map is written only when a test asks for it)
+    s = launch_haar_fwd(x, N, Cin, H, W, L, dt, taps ? taps->coef : nullptr, f.nrm2, f.amaxpos, st);
+    if (s != WCC_OK) return s;
+    if ((s = profile_mark(1, st)) != WCC_OK) return s;
+    // joint shrinkage: index list, rank map, max |kept|
+    s = launch_select(f.nrm2, N, P, k, f.idx, nullptr, f.rank, f.amaxpos, f.amax_kept, f.sel, f.sel_bytes, st);
+    if (s != WCC_OK) return s;
+    if ((s = profile_mark(2, st)) != WCC_OK) return s;
+    s = launch_weight_prep(Wt, Cout, Cin, f.kpad, bits, f.Wq, f.scale_w, st);
+    if (s != WCC_OK) return s;
+    if ((s = profile_mark(3, st)) != WCC_OK) return s;
+    // second pass over x: transform, mask + quantize, tensor-core contraction, dequantize, inverse, store
+    void* xq_tap = taps ? (bits >= 2 ? static_cast<void*>(taps->Xq) : taps->Xb) : nullptr;
+    s = launch_fused_pass2(x, f.Wq, f.rank, f.amax_kept, bits, f.scale_w, N, Cin, Cout, H, W, L, k, f.kpad, dt, y,
+                           xq_tap, taps ? taps->acc : nullptr, st);
+    if (s != WCC_OK) return s;
+    for (int i = 4; i <= WCC_NUM_STAGES; ++i)
+        if ((s = profile_mark(i, st)) != WCC_OK) return s;
+
+    if (taps) {
+        const cudaMemcpyKind dd = cudaMemcpyDeviceToDevice;
+        if (taps->nrm2) WCC_CUDA_TRY(cudaMemcpyAsync(taps->nrm2, f.nrm2, (size_t)N * P * 4, dd, st));
+        if (taps->idx) WCC_CUDA_TRY(cudaMemcpyAsync(taps->idx, f.idx, (size_t)M * 4, dd, st));
+        if (bits >= 2) {
+            if (taps->Wq) WCC_CUDA_TRY(cudaMemcpyAsync(taps->Wq, f.Wq, (size_t)Cout * f.kpad, dd, st));
+            if (taps->scale_w) WCC_CUDA_TRY(cudaMemcpyAsync(taps->scale_w, f.scale_w, (size_t)Cout * 4, dd, st));
+            if (taps->scale_a) {
+                scale_tap_kernel<<<1, 1, 0, st>>>(f.amax_kept, (float)((1 << (bits - 1)) - 1), taps->scale_a);
+                WCC_LAUNCH_CHECK();
+            }
+        }
+    }
+    return WCC_OK;
+}
+
 }  // namespace wcc
 
 using namespace wcc;
@@ -174,6 +256,12 @@ int wcc_kpad(int Cin, int bits)
 }
 
 size_t wcc_workspace_bytes(int N, int Cin, int Cout, int H, int Wd, int levels, int k, int bits, wcc_dtype dt)
+{
+    if (check_forward_args(N, Cin, Cout, H, Wd, levels, k, bits, dt) != WCC_OK) return 0;
+    return carve_fused_ws(nullptr, N, Cin, Cout, H, Wd, k, bits).total;
+}
+
+size_t wcc_staged_workspace_bytes(int N, int Cin, int Cout, int H, int Wd, int levels, int k, int bits, wcc_dtype dt)
 {
     if (check_forward_args(N, Cin, Cout, H, Wd, levels, k, bits, dt) != WCC_OK) return 0;
     return carve_forward_ws(nullptr, N, Cin, Cout, H, Wd, k, bits).total;
@@ -237,6 +325,14 @@ wcc_status wcc_forward(const void* x, const float* Wt, int N, int Cin, int Cout,
 {
     return forward_impl(x, Wt, N, Cin, Cout, H, Wd, levels, k, bits, y, dt, ws, ws_bytes,
                         static_cast<cudaStream_t>(stream), nullptr);
+}
+
+wcc_status wcc_forward_staged(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int Wd,
+                              int levels, int k, int bits, void* y, wcc_dtype dt,
+                              void* ws, size_t ws_bytes, void* stream, const wcc_taps* taps)
+{
+    return staged_impl(x, Wt, N, Cin, Cout, H, Wd, levels, k, bits, y, dt, ws, ws_bytes,
+                       static_cast<cudaStream_t>(stream), taps);
 }
 
 wcc_status wcc_forward_debug(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int Wd,

@@ -18,11 +18,12 @@ _STATUS = {0: "ok", 1: "null pointer", 2: "bad shape", 3: "k out of range", 4: "
            6: "misaligned pointer", 7: "workspace too small", 8: "CUDA error", 9: "device wait timed out",
            10: "non-finite input"}
 
-EXPORTS = ("wcc_workspace_bytes", "wcc_select_workspace_bytes", "wcc_haar_fwd", "wcc_haar_inv", "wcc_select_topk",
+EXPORTS = ("wcc_staged_workspace_bytes", "wcc_forward_staged", "wcc_workspace_bytes", "wcc_select_workspace_bytes", "wcc_haar_fwd", "wcc_haar_inv", "wcc_select_topk",
            "wcc_forward", "wcc_forward_debug", "wcc_kpad", "wcc_last_status", "wcc_status_str",
            "wcc_profile_enable", "wcc_profile_read", "wcc_kernel_launches", "wcc_select_topk_static")
 STATIC_SCRATCH_BYTES = 512 * 1024
-STAGES = ("haar_fwd_norms", "select_topk", "weight_quant", "gather_quant", "contract", "scatter_inv")
+STAGES = ("haar_fwd_norms", "select_topk", "weight_quant", "gather_quant", "contract", "scatter_inv")   # wcc_forward_staged
+FUSED_STAGES = ("haar_norms", "select_topk", "weight_quant", "fused_pass2")                               # wcc_forward
 
 
 class WccError(RuntimeError):
@@ -49,6 +50,8 @@ def lib() -> C.CDLL:
         i, vp, sz = C.c_int, C.c_void_p, C.c_size_t
         L.wcc_workspace_bytes.restype = sz
         L.wcc_workspace_bytes.argtypes = [i] * 9
+        L.wcc_staged_workspace_bytes.restype = sz
+        L.wcc_staged_workspace_bytes.argtypes = [i] * 9
         L.wcc_select_workspace_bytes.restype = sz
         L.wcc_select_workspace_bytes.argtypes = [i, i]
         L.wcc_kpad.restype = i
@@ -66,6 +69,8 @@ def lib() -> C.CDLL:
         L.wcc_forward.argtypes = fwd
         L.wcc_forward_debug.restype = i
         L.wcc_forward_debug.argtypes = fwd + [C.POINTER(Taps)]
+        L.wcc_forward_staged.restype = i
+        L.wcc_forward_staged.argtypes = fwd + [C.POINTER(Taps)]
         L.wcc_last_status.restype = i
         L.wcc_last_status.argtypes = [vp]
         L.wcc_profile_enable.restype = i
@@ -170,17 +175,19 @@ class Workspace:
         self.buf = torch.empty((max(self.nbytes, 256),), dtype=torch.uint8, device=device)
 
     @classmethod
-    def for_problem(cls, x: torch.Tensor, Cout: int, levels: int, k: int, bits: int):
+    def for_problem(cls, x: torch.Tensor, Cout: int, levels: int, k: int, bits: int, staged: bool = False):
         N, Cin, H, W = x.shape
-        n = workspace_bytes(N, Cin, Cout, H, W, levels, k, bits, _dt(x))
+        fn = lib().wcc_staged_workspace_bytes if staged else lib().wcc_workspace_bytes
+        n = int(fn(N, Cin, Cout, H, W, levels, k, bits, _dt(x)))
         if n == 0:
             raise WccError(2, "wcc_workspace_bytes")
         return cls(n, x.device)
 
 
 def forward(x: torch.Tensor, Wt: torch.Tensor, levels: int, k: int, bits: int = 8, y: torch.Tensor | None = None,
-            ws: Workspace | None = None, taps: bool = False):
-    """The WCC layer.  Returns y, or (y, dict of intermediate tensors) when ``taps`` is set."""
+            ws: Workspace | None = None, taps: bool = False, staged: bool = False):
+    """The WCC layer.  Returns y, or (y, dict of intermediate tensors) when ``taps`` is set.
+    ``staged`` selects wcc_forward_staged (every intermediate in memory) instead of the fused wcc_forward."""
     _dev(x, "x")
     _dev(Wt, "Wt")
     if Wt.dtype != torch.float32:
@@ -192,11 +199,14 @@ def forward(x: torch.Tensor, Wt: torch.Tensor, levels: int, k: int, bits: int = 
     if y is None:
         y = torch.empty((N, Cout, H, W), dtype=x.dtype, device=x.device)
     if ws is None:
-        ws = Workspace.for_problem(x, Cout, levels, k, bits)
+        ws = Workspace.for_problem(x, Cout, levels, k, bits, staged=staged)
     args = (x.data_ptr(), Wt.data_ptr(), N, Cin, Cout, H, W, levels, k, bits, y.data_ptr(), _dt(x),
             ws.buf.data_ptr(), ws.nbytes, _stream())
     if not taps:
-        _check(lib().wcc_forward(*args), "wcc_forward")
+        if staged:
+            _check(lib().wcc_forward_staged(*args, None), "wcc_forward_staged")
+        else:
+            _check(lib().wcc_forward(*args), "wcc_forward")
         return y
     P, M, kp = H * W, N * k, kpad(Cin, bits)
     dev = x.device
@@ -209,8 +219,14 @@ def forward(x: torch.Tensor, Wt: torch.Tensor, levels: int, k: int, bits: int = 
                  Wq=torch.empty((Cout, kp), dtype=torch.int8, device=dev), scale_w=torch.empty((Cout,), dtype=torch.float32, device=dev))
     else:
         t.update(Xb=torch.empty((M, kp), dtype=torch.bfloat16, device=dev))
+    for name in ("Xq", "Xb", "acc"):          # every row is a kept position and gets written; start from zeros anyway
+        if name in t:
+            t[name].zero_()
     s = Taps(**{name: _ptr(t.get(name)) for name, _ in Taps._fields_})
-    _check(lib().wcc_forward_debug(*args, C.byref(s)), "wcc_forward_debug")
+    if staged:
+        _check(lib().wcc_forward_staged(*args, C.byref(s)), "wcc_forward_staged")
+    else:
+        _check(lib().wcc_forward_debug(*args, C.byref(s)), "wcc_forward_debug")
     return y, t
 
 

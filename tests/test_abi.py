@@ -44,8 +44,11 @@ def test_kpad(L):
 
 def test_workspace_query(L):
     n = L.wcc_workspace_bytes(1, 32, 32, 64, 64, 2, 1024, 8, 0)
-    assert n > 1 * 32 * 4096 * 4            # holds at least the coefficient map
+    assert n >= 3 * 4096 * 4                # norms, per-position max, rank map
     assert n % 256 == 0
+    m = L.wcc_staged_workspace_bytes(1, 32, 32, 64, 64, 2, 1024, 8, 0)
+    assert m > 1 * 32 * 4096 * 4 and m > n  # also holds the coefficient map
+    assert L.wcc_staged_workspace_bytes(1, 32, 32, 60, 64, 3, 10, 8, 0) == 0
     assert L.wcc_workspace_bytes(1, 32, 32, 64, 64, 2, 1024, 8, 0) == n
     # invalid arguments give 0
     assert L.wcc_workspace_bytes(1, 32, 32, 60, 64, 3, 10, 8, 0) == 0     # 60 % 8 != 0

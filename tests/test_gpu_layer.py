@@ -29,12 +29,12 @@ def _x_dev(w):
     return torch.from_numpy(w.x).cuda()
 
 
-def _run_and_compare(wcc, w, full_taps=True):
+def _run_and_compare(wcc, w, staged=False):
     x = _x_dev(w)
     Wt = torch.from_numpy(w.Wt).cuda()
-    ws = wcc.Workspace.for_problem(x, w.Cout, w.levels, w.k, w.bits)
+    ws = wcc.Workspace.for_problem(x, w.Cout, w.levels, w.k, w.bits, staged=staged)
     ws.buf.fill_(0xFF)                                        # poison: nothing may depend on old contents
-    y, t = wcc.forward(x, Wt, w.levels, w.k, w.bits, ws=ws, taps=True)
+    y, t = wcc.forward(x, Wt, w.levels, w.k, w.bits, ws=ws, taps=True, staged=staged)
     assert wcc.last_status() == 0
     want, o = oracle.forward(w.x_f32(), w.Wt, w.levels, w.k, w.bits, out_bf16=(w.dtype == "bf16"), taps=True)
 
@@ -69,9 +69,10 @@ def _run_and_compare(wcc, w, full_taps=True):
         # same integers and the same fp32 operation order: identical up to the final rounding to the output type
         assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
     # plain wcc_forward gives the same bytes as the debug entry point, and does so again (determinism)
-    y2 = wcc.forward(x, Wt, w.levels, w.k, w.bits, ws=ws)
-    y3 = wcc.forward(x, Wt, w.levels, w.k, w.bits)
+    y2 = wcc.forward(x, Wt, w.levels, w.k, w.bits, ws=ws, staged=staged)
+    y3 = wcc.forward(x, Wt, w.levels, w.k, w.bits, staged=staged)
     assert torch.equal(y, y2) and torch.equal(y, y3)
+    assert wcc.last_status() == 0
     return got, want
 
 
@@ -93,11 +94,12 @@ SMALL = [  # N, Cin, Cout, H, W, dtype, levels, gamma, bits
 ]
 
 
+@pytest.mark.parametrize("staged", [False, True], ids=["fused", "staged"])
 @pytest.mark.parametrize("cfg", SMALL, ids=lambda c: "N%d_%dto%d_%dx%d_%s_L%d_g%s_b%d" % c)
-def test_layer_small(wcc, cfg):
+def test_layer_small(wcc, cfg, staged):
     N, Cin, Cout, H, W, dtype, L, gamma, bits = cfg
     w = inputs.custom("small", 3, N, Cin, Cout, H, W, dtype, L, gamma, bits, n_sin=4, fmax=3.0)
-    _run_and_compare(wcc, w)
+    _run_and_compare(wcc, w, staged=staged)
 
 
 def test_layer_k_equals_one_and_all(wcc):
@@ -120,10 +122,11 @@ def test_keep_everything_unquantized_is_the_dense_conv(wcc):
     assert np.abs(y - ref).max() <= 2e-2 * np.abs(ref).max()
 
 
+@pytest.mark.parametrize("staged", [False, True], ids=["fused", "staged"])
 @pytest.mark.parametrize("name", ["C1", "C2", "C3", "C3u", "C4", "C4b", "C5a", "C5b"])
-def test_layer_named_workloads_full_size(wcc, name):
+def test_layer_named_workloads_full_size(wcc, name, staged):
     """The five benchmark workloads at full size, in the launch configuration the bench times."""
-    _run_and_compare(wcc, inputs.make(name))
+    _run_and_compare(wcc, inputs.make(name), staged=staged)
 
 
 def test_chain_of_layers_with_relu(wcc):
