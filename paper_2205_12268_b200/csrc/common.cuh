@@ -78,7 +78,7 @@ wcc_status launch_scatter_inv(const int32_t* acc, int ldc, bool acc_is_float, co
 // kept positions of amaxpos, as float bits, must be zeroed by this call) are optional.
 size_t select_ws_bytes(int N, int P);
 wcc_status launch_select(const float* nrm2, int N, int P, int k, int32_t* idx, float* tau,
-                         int32_t* rank, const float* amaxpos, float* amax_kept,
+                         int32_t* rank, const float* amaxpos, bool want_amax,
                          void* ws, size_t ws_bytes, cudaStream_t st);
 
 // Weight quantization (bits >= 2: int8 codes + per-row scale; bits == 0: bf16 copy), rows padded to kpad.

@@ -28,6 +28,7 @@ namespace fz {
 
 constexpr int ROWS = 256;            // positions per CTA
 constexpr int SUB = 8;               // output channels per transpose round
+constexpr int RING2 = 3;             // cp.async stages per warp in phase 1
 constexpr float MAGIC = 12582912.0f; // 1.5 * 2^23: adding it rounds to the nearest integer, ties to even
 
 __device__ __forceinline__ uint64_t smem_desc_plain(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
@@ -66,11 +67,13 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
     uint8_t* sm = smem_raw + (base - raw);
     const int krow = kpad * ES;                       // bytes of K per row
     const int kchunks = krow / 16;
+    using Ring = PatchRing<T>;
     uint8_t* sA = sm;                                                   // [kchunks][256][16]
     uint8_t* sB = sA + (size_t)kchunks * ROWS * 16;                     // [kchunks][npad][16]
-    float* stage = reinterpret_cast<float*>(sB + (size_t)kchunks * npad * 16);   // [SUB][8][32]
-    int32_t* srank = reinterpret_cast<int32_t*>(stage + SUB * 8 * 32);  // [8][32]
+    int32_t* srank = reinterpret_cast<int32_t*>(sB + (size_t)kchunks * npad * 16);      // [8][32]
     Ctl* ctl = reinterpret_cast<Ctl*>(srank + 8 * 32);
+    uint8_t* shared_region = reinterpret_cast<uint8_t*>(ctl + 1);       // phase 1: input rings; phase 3: transpose buffer
+    float* stage = reinterpret_cast<float*>(shared_region);             // [SUB][8][32]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tiles_x = (W + TT::TW - 1) / TT::TW, tiles_y = H / TT::TH;
@@ -114,40 +117,68 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
     for (int s = 0; s < 8; ++s) mul[s] = (rk[s] >= 0) ? inv : 0.0f;
 
     // ---- phase 1: transform + quantize into the A operand --------------------------------------------
+    // Warp w takes the 8-channel units w, w+4, ...; inputs arrive LU channels at a time through its cp.async ring.
     const T* xin = x + (size_t)n * Cin * P;
     const int units = kpad / 8;
-    for (int u = warp; u < units; u += 4) {
-        RawPatch rawp[8];
+    const int my_units = (units - warp + 3) / 4;
+    constexpr int LU = Ring::LU, SUBS = 8 / LU;
+    uint8_t* my_ring = shared_region + (VEC ? warp * RING2 * Ring::STAGE_BYTES : 0);
+    const uint32_t my_ring_s = tc::smem_u32(my_ring);
+    const int nq = my_units * SUBS;                    // ring stages this warp will consume
+    auto chan0 = [&](int q) { return (warp + 4 * (q / SUBS)) * 8 + (q % SUBS) * LU; };
+    if (VEC) {
 #pragma unroll
-        for (int d = 0; d < 8; ++d) {
-            const int c = u * 8 + d;
-            if (c < Cin) load_patch<T, VEC>(xin + (size_t)c * P, W, lp, rawp[d]);
-        }
+        for (int q = 0; q < RING2 - 1; ++q) Ring::issue(my_ring_s, q, xin, P, W, q < nq ? Cin : 0, chan0(q), lp, lane);
+    }
+    for (int ui = 0; ui < my_units; ++ui) {
+        const int u = warp + 4 * ui;
         uint32_t packed[8][4];         // per slot: 8 int8 codes (2 words) or 8 bf16 values (4 words)
-        float prev[8];
 #pragma unroll
-        for (int d = 0; d < 8; ++d) {
-            const int c = u * 8 + d;
-            float o[8];
-            if (c < Cin) {             // warp-uniform
-                float p[2][4];
-                unpack_patch<T>(rawp[d], p);
-                haar_fwd_lane<L>(p, o, lane);
-            } else {
+        for (int g = 0; g < 2; ++g) {                      // two groups of 4 channels
+            uint32_t code[4][8];                           // int8: float bits whose low byte is the code; bf16: value bits
 #pragma unroll
-                for (int s = 0; s < 8; ++s) o[s] = 0.0f;
+            for (int dd4 = 0; dd4 < 4; ++dd4) {
+                const int d = g * 4 + dd4;                 // channel within the unit
+                const int sub = d / LU, dd = d % LU;       // ring stage within the unit, channel within the stage
+                const int q = ui * SUBS + sub;
+                if (VEC && dd == 0) {
+                    const int qn = q + RING2 - 1;
+                    Ring::issue(my_ring_s, qn % RING2, xin, P, W, qn < nq ? Cin : 0, chan0(qn), lp, lane);
+                    Ring::template wait<RING2 - 1>();
+                }
+                const int c = u * 8 + d;
+                float o[8];
+                if (c < Cin) {             // warp-uniform
+                    RawPatch rawp;
+                    if (VEC) Ring::read(my_ring, q % RING2, dd, lane, rawp);
+                    else load_patch<T, VEC>(xin + (size_t)c * P, W, lp, rawp);
+                    float p[2][4];
+                    unpack_patch<T>(rawp, p);
+                    haar_fwd_lane<L>(p, o, lane);
+                } else {
+#pragma unroll
+                    for (int s = 0; s < 8; ++s) o[s] = 0.0f;
+                }
+#pragma unroll
+                for (int s = 0; s < 8; s += 2) {
+                    float2 t = mul2(make_float2(o[s], o[s + 1]), make_float2(mul[s], mul[s + 1]));
+                    // int8: the low byte of (t + 1.5*2^23) is the two's complement code of rint(t); |t| <= qmax by construction
+                    // scalar adds on purpose: a packed add right after the packed product gets contracted into one
+                    // fused operation, which rounds once and changes codes that sit on a half-way point
+                    if (I8) t = make_float2(__fadd_rn(t.x, MAGIC), __fadd_rn(t.y, MAGIC));
+                    code[dd4][s] = __float_as_uint(t.x);
+                    code[dd4][s + 1] = __float_as_uint(t.y);
+                }
             }
 #pragma unroll
             for (int s = 0; s < 8; ++s) {
-                const float t = __fmul_rn(o[s], mul[s]);
                 if (I8) {
-                    // low byte of (t + 1.5*2^23) is the two's complement code of rint(t); |t| <= qmax by construction
-                    const uint32_t code = __float_as_uint(__fadd_rn(t, MAGIC));
-                    if ((d & 3) == 0) packed[s][d >> 2] = code & 0xFFu;
-                    else packed[s][d >> 2] |= (code & 0xFFu) << (8 * (d & 3));
+                    const uint32_t lo = __byte_perm(code[0][s], code[1][s], 0x0040);
+                    const uint32_t hi = __byte_perm(code[2][s], code[3][s], 0x0040);
+                    packed[s][g] = __byte_perm(lo, hi, 0x5410);
                 } else {
-                    if ((d & 1) == 0) prev[s] = t;
-                    else packed[s][d >> 1] = pack_bf16x2(prev[s], t);
+                    packed[s][2 * g] = pack_bf16x2(__uint_as_float(code[0][s]), __uint_as_float(code[1][s]));
+                    packed[s][2 * g + 1] = pack_bf16x2(__uint_as_float(code[2][s]), __uint_as_float(code[3][s]));
                 }
             }
         }
@@ -165,6 +196,7 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
             }
         }
     }
+    if (VEC) Ring::template wait<0>();
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic-proxy writes -> visible to the tensor core
     tc::fence_before();
     __syncthreads();
@@ -252,6 +284,8 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
 
 }  // namespace fz
 
+static inline size_t vmax(size_t a, size_t b) { return a > b ? a : b; }
+
 template <typename T, int L, bool VEC>
 static wcc_status fused_pass2_dispatch(const void* x, const void* Wq, const int32_t* rank, const float* amax_kept, int bits,
                                        const float* scale_w, int N, int Cin, int Cout, int H, int W, int k, int kpad,
@@ -265,8 +299,9 @@ static wcc_status fused_pass2_dispatch(const void* x, const void* Wq, const int3
     int tmem_cols = 32;
     while (tmem_cols < 2 * nchunk) tmem_cols <<= 1;
     const int kchunks = kpad * es / 16;
-    const size_t smem = 128 + (size_t)kchunks * fz::ROWS * 16 + (size_t)kchunks * npad * 16 + fz::SUB * 8 * 32 * 4 +
-                        8 * 32 * 4 + sizeof(fz::Ctl) + 16;
+    const size_t region = vmax((size_t)fz::SUB * 8 * 32 * 4, (size_t)4 * fz::RING2 * PatchRing<T>::STAGE_BYTES);
+    const size_t smem = 128 + (size_t)kchunks * fz::ROWS * 16 + (size_t)kchunks * npad * 16 + 8 * 32 * 4 + sizeof(fz::Ctl) +
+                        region + 16;
     if (smem > 200 * 1024 || (kpad * es) % 32 != 0) return WCC_ERR_SHAPE;
     const float qmax = i8 ? (float)((1 << (bits - 1)) - 1) : 1.0f;
     int* status = nullptr;

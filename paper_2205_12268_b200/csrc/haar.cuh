@@ -8,7 +8,7 @@
 // transform every lane owns exactly eight wavelet-domain positions ("slots"):
 //   0,1  y2 of level 1 (two quads)      2,3  y3 of level 1       4,5  y4 of level 1
 //   6,7  L=1: y1 of level 1 (two quads)
-//        L>=2, rp even: slot 6 = y2 of level 2, slot 7 = y1 of level 2 (L=2) or one of y1..y4 of level 3,
+//        L>=2, rp even: slot 7 = y2 of level 2, slot 6 = y1 of level 2 (L=2) or one of y1..y4 of level 3,
 //                       by (rp & 2, cg & 1): (0,0) y1, (0,1) y2, (2,0) y3, (2,1) y4
 //        L>=2, rp odd : slot 6 = y3 of level 2, slot 7 = y4 of level 2
 // so the per-position norm accumulators live in registers across the whole channel loop, which keeps the
@@ -58,13 +58,13 @@ __device__ __forceinline__ LanePos lane_positions(int H, int W, int tile_y, int 
     } else {
         const int i2 = i1 >> 1, j2 = j1 >> 1, h2 = H >> 2, w2 = W >> 2;
         if ((rp & 1) == 0) {
-            lp.pos[6] = i2 * W + w2 + j2;
+            lp.pos[7] = i2 * W + w2 + j2;
             if (L == 2) {
-                lp.pos[7] = i2 * W + j2;
+                lp.pos[6] = i2 * W + j2;
             } else {
                 const int i3 = i2 >> 1, j3 = j2 >> 1, h3 = H >> 3, w3 = W >> 3;
                 const bool top = (rp & 2) == 0, left = (cg & 1) == 0;
-                lp.pos[7] = (top ? i3 : h3 + i3) * W + (left ? j3 : w3 + j3);
+                lp.pos[6] = (top ? i3 : h3 + i3) * W + (left ? j3 : w3 + j3);
             }
         } else {
             lp.pos[6] = (h2 + i2) * W + j2;
@@ -83,54 +83,69 @@ __device__ __forceinline__ bool slot_ok(const LanePos& lp, int s)
     return lp.ok0;
 }
 
-// Forward transform of the lane's patch p[row][col] into its eight slots.
+// Packed fp32 pairs (Blackwell f32x2 pipe): each operation rounds both halves once, to nearest even, exactly like
+// the scalar operation.  a - b is written fma(b, -1, a): one rounding of the exact difference.
+// add2 / mul2 are written in PTX with an explicit rounding modifier so that a product followed by a sum is never
+// contracted into one fused operation (that would round once instead of twice and change quantization codes).
+__device__ __forceinline__ float2 add2(float2 a, float2 b)
+{
+    float2 r;
+    asm("{\n .reg .b64 ra, rb, rc;\n mov.b64 ra, {%2, %3};\n mov.b64 rb, {%4, %5};\n add.rn.f32x2 rc, ra, rb;\n mov.b64 {%0, %1}, rc;\n}\n"
+        : "=f"(r.x), "=f"(r.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+    return r;
+}
+__device__ __forceinline__ float2 mul2(float2 a, float2 b)
+{
+    float2 r;
+    asm("{\n .reg .b64 ra, rb, rc;\n mov.b64 ra, {%2, %3};\n mov.b64 rb, {%4, %5};\n mul.rn.f32x2 rc, ra, rb;\n mov.b64 {%0, %1}, rc;\n}\n"
+        : "=f"(r.x), "=f"(r.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+    return r;
+}
+__device__ __forceinline__ float2 sub2(float2 a, float2 b) { return __ffma2_rn(b, make_float2(-1.0f, -1.0f), a); }
+__device__ __forceinline__ float2 half2x(float2 a) { return mul2(a, make_float2(0.5f, 0.5f)); }
+
+// Forward transform of the lane's patch p[row][col] into its eight slots.  The two quads of the patch are processed
+// side by side in packed pairs: (quad 0, quad 1).
 template <int L>
 __device__ __forceinline__ void haar_fwd_lane(const float (&p)[2][4], float (&o)[8], int lane)
 {
     using T = HaarTile<L>;
-    float ll[2];
-#pragma unroll
-    for (int q = 0; q < 2; ++q) {
-        const float a = p[0][2 * q], b = p[0][2 * q + 1], c = p[1][2 * q], d = p[1][2 * q + 1];
-        const float s0 = __fadd_rn(a, b), d0 = __fsub_rn(a, b), s1 = __fadd_rn(c, d), d1 = __fsub_rn(c, d);
-        ll[q] = __fmul_rn(__fadd_rn(s0, s1), 0.5f);
-        o[0 + q] = __fmul_rn(__fadd_rn(d0, d1), 0.5f);
-        o[2 + q] = __fmul_rn(__fsub_rn(s0, s1), 0.5f);
-        o[4 + q] = __fmul_rn(__fsub_rn(d0, d1), 0.5f);
-    }
+    const float2 a = make_float2(p[0][0], p[0][2]), b = make_float2(p[0][1], p[0][3]);
+    const float2 c = make_float2(p[1][0], p[1][2]), d = make_float2(p[1][1], p[1][3]);
+    const float2 s0 = add2(a, b), d0 = sub2(a, b), s1 = add2(c, d), d1 = sub2(c, d);
+    const float2 ll = half2x(add2(s0, s1));            // y1 of both quads
+    const float2 y2 = half2x(add2(d0, d1));
+    const float2 y3 = half2x(sub2(s0, s1));
+    const float2 y4 = half2x(sub2(d0, d1));
+    o[0] = y2.x; o[1] = y2.y; o[2] = y3.x; o[3] = y3.y; o[4] = y4.x; o[5] = y4.y;
     if (L == 1) {
-        o[6] = ll[0];
-        o[7] = ll[1];
+        o[6] = ll.x;
+        o[7] = ll.y;
         return;
     }
+    // Level 2: the lane pair (rp, rp^1) holds the 2x2 block of level-1 low-pass values, one row each.  With
+    // sg = +1 on the upper (even) lane and -1 on the lower one, fma(own, sg, other) is own+other on the upper lane
+    // (s0+s1, d0+d1 -> y1, y2) and other-own on the lower lane (s0-s1, d0-d1 -> y3, y4): one rounding, as an add.
     const int rp = lane / T::CG, cg = lane % T::CG;
     const bool even = (rp & 1) == 0;
-    const float s = __fadd_rn(ll[0], ll[1]), d = __fsub_rn(ll[0], ll[1]);
+    const float sg = even ? 1.0f : -1.0f;
+    const float s = __fadd_rn(ll.x, ll.y), dd = __fsub_rn(ll.x, ll.y);
     const float ps = __shfl_xor_sync(0xFFFFFFFFu, s, T::CG);
-    const float pd = __shfl_xor_sync(0xFFFFFFFFu, d, T::CG);
-    float ll2 = 0.0f;
-    if (even) {
-        ll2 = __fmul_rn(__fadd_rn(s, ps), 0.5f);       // y1 = (s0 + s1) / 2
-        o[6] = __fmul_rn(__fadd_rn(d, pd), 0.5f);      // y2 = (d0 + d1) / 2
-        o[7] = ll2;
-    } else {
-        o[6] = __fmul_rn(__fsub_rn(ps, s), 0.5f);      // y3 = (s0 - s1) / 2, s0 from the even lane
-        o[7] = __fmul_rn(__fsub_rn(pd, d), 0.5f);      // y4 = (d0 - d1) / 2
-    }
+    const float pd = __shfl_xor_sync(0xFFFFFFFFu, dd, T::CG);
+    const float2 l2 = half2x(__ffma2_rn(make_float2(s, dd), make_float2(sg, sg), make_float2(ps, pd)));
+    o[6] = l2.x;                                       // even: y1, odd: y3
+    o[7] = l2.y;                                       // even: y2, odd: y4
     if (L == 3) {
-        const float v = ll2;
+        // Level 3: the four even lanes {rp, rp^2} x {cg, cg^1} hold a, b / c, d.  Horizontal step: left lane a+b (c+d),
+        // right lane a-b (c-d); vertical step: top lanes sum (y1, y2), bottom lanes difference (y3, y4).
+        const float sgh = (cg & 1) == 0 ? 1.0f : -1.0f;
+        const float sgv = (rp & 2) == 0 ? 1.0f : -1.0f;
+        const float v = o[6];
         const float h = __shfl_xor_sync(0xFFFFFFFFu, v, 1);
-        const float v2 = __shfl_xor_sync(0xFFFFFFFFu, v, 2 * T::CG);
-        const float h2 = __shfl_xor_sync(0xFFFFFFFFu, h, 2 * T::CG);
-        const bool top = (rp & 2) == 0, left = (cg & 1) == 0;
-        const float a = top ? (left ? v : h) : (left ? v2 : h2);
-        const float b = top ? (left ? h : v) : (left ? h2 : v2);
-        const float c = top ? (left ? v2 : h2) : (left ? v : h);
-        const float dd = top ? (left ? h2 : v2) : (left ? h : v);
-        const float s0 = __fadd_rn(a, b), d0 = __fsub_rn(a, b), s1 = __fadd_rn(c, dd), d1 = __fsub_rn(c, dd);
-        const float r = top ? (left ? __fadd_rn(s0, s1) : __fadd_rn(d0, d1))
-                            : (left ? __fsub_rn(s0, s1) : __fsub_rn(d0, d1));
-        if (even) o[7] = __fmul_rn(r, 0.5f);
+        const float t = __fmaf_rn(v, sgh, h);
+        const float q = __shfl_xor_sync(0xFFFFFFFFu, t, 2 * T::CG);
+        const float r = __fmul_rn(__fmaf_rn(t, sgv, q), 0.5f);
+        if (even) o[6] = r;
     }
 }
 
@@ -139,52 +154,38 @@ template <int L>
 __device__ __forceinline__ void haar_inv_lane(const float (&o)[8], float (&p)[2][4], int lane)
 {
     using T = HaarTile<L>;
-    float ll[2];
+    float2 ll;
     if (L == 1) {
-        ll[0] = o[6];
-        ll[1] = o[7];
+        ll = make_float2(o[6], o[7]);
     } else {
         const int rp = lane / T::CG, cg = lane % T::CG;
-        const bool even = (rp & 1) == 0;
-        float ll2 = o[7];
+        const float sg = (rp & 1) == 0 ? 1.0f : -1.0f;
+        float m0 = o[6];
         if (L == 3) {
-            const float v = o[7];
-            const float h = __shfl_xor_sync(0xFFFFFFFFu, v, 1);
-            const float v2 = __shfl_xor_sync(0xFFFFFFFFu, v, 2 * T::CG);
-            const float h2 = __shfl_xor_sync(0xFFFFFFFFu, h, 2 * T::CG);
-            const bool top = (rp & 2) == 0, left = (cg & 1) == 0;
-            const float y1 = top ? (left ? v : h) : (left ? v2 : h2);
-            const float y2 = top ? (left ? h : v) : (left ? h2 : v2);
-            const float y3 = top ? (left ? v2 : h2) : (left ? v : h);
-            const float y4 = top ? (left ? h2 : v2) : (left ? h : v);
-            const float t0 = __fadd_rn(y1, y3), t1 = __fsub_rn(y1, y3), u0 = __fadd_rn(y2, y4), u1 = __fsub_rn(y2, y4);
-            const float r = top ? (left ? __fadd_rn(t0, u0) : __fsub_rn(t0, u0))
-                                : (left ? __fadd_rn(t1, u1) : __fsub_rn(t1, u1));
-            ll2 = __fmul_rn(r, 0.5f);
+            // vertical step: top lanes y1+y3 (y2+y4), bottom lanes y1-y3 (y2-y4); horizontal step: left lanes sum
+            // (a, c), right lanes difference (b, d)
+            const float sgh = (cg & 1) == 0 ? 1.0f : -1.0f;
+            const float sgv = (rp & 2) == 0 ? 1.0f : -1.0f;
+            const float pv = __shfl_xor_sync(0xFFFFFFFFu, m0, 2 * T::CG);
+            const float w = __fmaf_rn(m0, sgv, pv);
+            const float q = __shfl_xor_sync(0xFFFFFFFFu, w, 1);
+            const float r = __fmul_rn(__fmaf_rn(w, sgh, q), 0.5f);
+            if ((rp & 1) == 0) m0 = r;
         }
-        const float m0 = even ? ll2 : o[6];
-        const float m1 = even ? o[6] : o[7];
+        // level 2: upper lane holds (y1, y2), lower lane (y3, y4)
+        const float m1 = o[7];
         const float p0 = __shfl_xor_sync(0xFFFFFFFFu, m0, T::CG);
         const float p1 = __shfl_xor_sync(0xFFFFFFFFu, m1, T::CG);
-        if (even) {       // y1 = m0, y2 = m1, y3 = p0, y4 = p1 -> first row of the 2x2 output
-            const float t0 = __fadd_rn(m0, p0), u0 = __fadd_rn(m1, p1);
-            ll[0] = __fmul_rn(__fadd_rn(t0, u0), 0.5f);
-            ll[1] = __fmul_rn(__fsub_rn(t0, u0), 0.5f);
-        } else {          // y1 = p0, y2 = p1, y3 = m0, y4 = m1 -> second row
-            const float t1 = __fsub_rn(p0, m0), u1 = __fsub_rn(p1, m1);
-            ll[0] = __fmul_rn(__fadd_rn(t1, u1), 0.5f);
-            ll[1] = __fmul_rn(__fsub_rn(t1, u1), 0.5f);
-        }
+        // upper: (t0, u0) = (y1 + y3, y2 + y4); lower: (t1, u1) = (y1 - y3, y2 - y4)
+        const float2 tu = __ffma2_rn(make_float2(m0, m1), make_float2(sg, sg), make_float2(p0, p1));
+        ll = make_float2(__fmul_rn(__fadd_rn(tu.x, tu.y), 0.5f), __fmul_rn(__fsub_rn(tu.x, tu.y), 0.5f));
     }
-#pragma unroll
-    for (int q = 0; q < 2; ++q) {
-        const float y1 = ll[q], y2 = o[0 + q], y3 = o[2 + q], y4 = o[4 + q];
-        const float t0 = __fadd_rn(y1, y3), t1 = __fsub_rn(y1, y3), u0 = __fadd_rn(y2, y4), u1 = __fsub_rn(y2, y4);
-        p[0][2 * q] = __fmul_rn(__fadd_rn(t0, u0), 0.5f);
-        p[0][2 * q + 1] = __fmul_rn(__fsub_rn(t0, u0), 0.5f);
-        p[1][2 * q] = __fmul_rn(__fadd_rn(t1, u1), 0.5f);
-        p[1][2 * q + 1] = __fmul_rn(__fsub_rn(t1, u1), 0.5f);
-    }
+    const float2 y2 = make_float2(o[0], o[1]), y3 = make_float2(o[2], o[3]), y4 = make_float2(o[4], o[5]);
+    const float2 t0 = add2(ll, y3), t1 = sub2(ll, y3), u0 = add2(y2, y4), u1 = sub2(y2, y4);
+    const float2 a = half2x(add2(t0, u0)), b = half2x(sub2(t0, u0));
+    const float2 c = half2x(add2(t1, u1)), d = half2x(sub2(t1, u1));
+    p[0][0] = a.x; p[0][1] = b.x; p[0][2] = a.y; p[0][3] = b.y;
+    p[1][0] = c.x; p[1][1] = d.x; p[1][2] = c.y; p[1][3] = d.y;
 }
 
 // ---- patch load / store ------------------------------------------------------------------------
@@ -369,6 +370,156 @@ haar_fwd_kernel(const T* __restrict__ x, int N, int C, int H, int W,
     if (amaxpos) store_slots<L, VEC>(amaxpos + (size_t)n * P, lp, amax);
 }
 
+
+// ---- per-warp asynchronous patch ring ------------------------------------------------------------
+// Each lane copies its own 2 x 4 patch of a few channels ahead of use with cp.async (global -> shared, no
+// registers held while the copy flies) and later reads back exactly the bytes it copied, so no barrier is needed:
+// only the thread's own cp.async groups are waited for.  A stage holds LU channels; slot of (stage, channel d,
+// row r, lane) = ((stage * LU + d) * 2 + r) * 32 + lane, ROWB bytes each (conflict-free: lanes are contiguous).
+template <typename T>
+struct PatchRing {
+    static constexpr int ROWB = 4 * (int)sizeof(T);              // bytes of one patch row: 8 (bf16) or 16 (fp32)
+    static constexpr int LU = (sizeof(T) == 2) ? 4 : 2;          // channels per stage: 2 KB per warp and stage
+    static constexpr int STAGE_BYTES = LU * 2 * 32 * ROWB;
+
+    // start the copies of channels [c0, c0 + LU) of one image into `stage`; always commits one group
+    static __device__ __forceinline__ void issue(uint32_t ring, int stage, const T* __restrict__ xin, size_t P, int W,
+                                                 int C, int c0, const LanePos& lp, int lane)
+    {
+#pragma unroll
+        for (int d = 0; d < LU; ++d) {
+            const int c = c0 + d;
+            const bool valid = (c < C) && lp.ok0;
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                const T* src = valid ? xin + (size_t)c * P + (size_t)(lp.r0 + r) * W + lp.c0 : xin;
+                const uint32_t dst = ring + (uint32_t)((((stage * LU + d) * 2 + r) * 32 + lane) * ROWB);
+                const int nbytes = valid ? ROWB : 0;              // 0: the slot is zero-filled
+                if (ROWB == 16)
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(nbytes) : "memory");
+                else
+                    asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dst), "l"(src), "r"(nbytes) : "memory");
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+
+    template <int PENDING>
+    static __device__ __forceinline__ void wait() { asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory"); }
+
+    static __device__ __forceinline__ void read(const uint8_t* ring, int stage, int d, int lane, RawPatch& raw)
+    {
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            const uint8_t* src = ring + (size_t)((((stage * LU + d) * 2 + r) * 32 + lane) * ROWB);
+            if (ROWB == 16) {
+                const uint4 v = *reinterpret_cast<const uint4*>(src);
+                raw.w[4 * r + 0] = v.x; raw.w[4 * r + 1] = v.y; raw.w[4 * r + 2] = v.z; raw.w[4 * r + 3] = v.w;
+            } else {
+                const uint2 v = *reinterpret_cast<const uint2*>(src);
+                raw.w[4 * r + 0] = v.x; raw.w[4 * r + 1] = v.y;
+            }
+        }
+    }
+};
+
+// ---- first pass of the fused layer: norms only -------------------------------------------------
+// One CTA of 4 warps per (image, tile).  The warps split the channels: in every round of 4 * LU channels warp w
+// transforms channels [w * LU, (w + 1) * LU) of the round in registers and hands the slot values over through shared
+// memory; then the 128 threads run the fused multiply-add chain of two positions each (warp w: slots 2w and 2w+1
+// of every lane) over the round's channels in ascending order, so the sum is the same sequential chain a single
+// thread would build.  Inputs arrive through the per-warp cp.async ring (RING stages ahead).  Nothing but the
+// norms and the per-position max |coef| is written.
+template <typename T, int L, bool VEC>
+__global__ void __launch_bounds__(128)
+haar_norms_kernel(const T* __restrict__ x, int N, int C, int H, int W,
+                  float* __restrict__ nrm2, float* __restrict__ amaxpos)
+{
+    using TT = HaarTile<L>;
+    using Ring = PatchRing<T>;
+    constexpr int LU = Ring::LU, RC = 4 * LU;          // channels per warp and per round
+    constexpr int RING = 4;                            // stages per warp
+    __shared__ float2 buf[RC][4][32];                  // [channel of the round][slot pair][lane]
+    __shared__ __align__(16) uint8_t ring_mem[VEC ? 4 * RING * Ring::STAGE_BYTES : 16];
+    const int tiles_x = (W + TT::TW - 1) / TT::TW, tiles_y = H / TT::TH;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int n, ty, tx;
+    tile_coords(blockIdx.x, tiles_x, tiles_y, n, ty, tx);
+    const LanePos lp = lane_positions<L>(H, W, ty, tx, lane);
+    const size_t P = (size_t)H * W;
+    const T* xin = x + (size_t)n * C * P;
+    uint8_t* my_ring = ring_mem + (VEC ? warp * RING * Ring::STAGE_BYTES : 0);
+    const uint32_t my_ring_s = (uint32_t)__cvta_generic_to_shared(my_ring);
+
+    float2 nn = make_float2(0.0f, 0.0f);
+    float a0 = 0.0f, a1 = 0.0f;
+    const int rounds = (C + RC - 1) / RC;
+    if (VEC) {
+#pragma unroll
+        for (int r = 0; r < RING - 1; ++r) Ring::issue(my_ring_s, r, xin, P, W, C, r * RC + warp * LU, lp, lane);
+    }
+    for (int r = 0; r < rounds; ++r) {
+        if (VEC) {
+            Ring::issue(my_ring_s, (r + RING - 1) % RING, xin, P, W, C, (r + RING - 1) * RC + warp * LU, lp, lane);
+            Ring::template wait<RING - 1>();
+        }
+#pragma unroll
+        for (int d = 0; d < LU; ++d) {
+            const int c = r * RC + warp * LU + d;
+            if (c < C) {                               // warp-uniform
+                RawPatch raw;
+                if (VEC) Ring::read(my_ring, r % RING, d, lane, raw);
+                else load_patch<T, VEC>(xin + (size_t)c * P, W, lp, raw);
+                float p[2][4], o[8];
+                unpack_patch<T>(raw, p);
+                haar_fwd_lane<L>(p, o, lane);
+#pragma unroll
+                for (int s = 0; s < 8; s += 2) buf[warp * LU + d][s >> 1][lane] = make_float2(o[s], o[s + 1]);
+            }
+        }
+        __syncthreads();
+        const int cnt = min(RC, C - r * RC);
+#pragma unroll
+        for (int c = 0; c < RC; ++c) {
+            if (c < cnt) {
+                const float2 v = buf[c][warp][lane];
+                nn = __ffma2_rn(v, v, nn);
+                a0 = fmaxf(a0, fabsf(v.x));
+                a1 = fmaxf(a1, fabsf(v.y));
+            }
+        }
+        __syncthreads();
+    }
+    if (VEC) Ring::template wait<0>();
+    const float n0 = nn.x, n1 = nn.y;
+    int p0 = 0, p1 = 0;
+    bool ok0 = false, ok1 = false;
+#pragma unroll
+    for (int s = 0; s < 8; s += 2) {
+        if (s == 2 * warp) {
+            p0 = lp.pos[s]; p1 = lp.pos[s + 1];
+            ok0 = slot_ok<L>(lp, s); ok1 = slot_ok<L>(lp, s + 1);
+        }
+    }
+    const bool pair = VEC && (L == 1 || warp < 3);     // adjacent, 8-byte aligned positions
+    float* nr = nrm2 + (size_t)n * P;
+    if (pair) {
+        if (ok0) *reinterpret_cast<float2*>(nr + p0) = make_float2(n0, n1);
+    } else {
+        if (ok0) nr[p0] = n0;
+        if (ok1) nr[p1] = n1;
+    }
+    if (amaxpos) {
+        float* am = amaxpos + (size_t)n * P;
+        if (pair) {
+            if (ok0) *reinterpret_cast<float2*>(am + p0) = make_float2(a0, a1);
+        } else {
+            if (ok0) am[p0] = a0;
+            if (ok1) am[p1] = a1;
+        }
+    }
+}
+
 // ---- plain inverse -------------------------------------------------------------------------------
 // One warp per (plane, tile).
 template <typename T, int L, bool VEC>
@@ -456,6 +607,11 @@ static wcc_status haar_fwd_dispatch(const void* x, int N, int C, int H, int W, f
     using TT = HaarTile<L>;
     constexpr int D = (sizeof(T) == 4) ? 4 : 8;
     const long long warps = (long long)N * ceil_div(W, TT::TW) * (H / TT::TH);
+    if (!coef && nrm2) {          // norms only: four warps per tile
+        haar_norms_kernel<T, L, VEC><<<(unsigned)warps, 128, 0, st>>>(static_cast<const T*>(x), N, C, H, W, nrm2, amaxpos);
+        WCC_LAUNCH_CHECK();
+        return WCC_OK;
+    }
     const int blocks = (int)((warps + 3) / 4);
     haar_fwd_kernel<T, L, VEC, D><<<blocks, 128, 0, st>>>(static_cast<const T*>(x), N, C, H, W, coef, nrm2, amaxpos);
     WCC_LAUNCH_CHECK();

@@ -56,7 +56,7 @@ static FwdWs carve_forward_ws(void* ws, int N, int Cin, int Cout, int H, int W, 
     f.idx = reinterpret_cast<int32_t*>(take(M * 4));
     f.sel_bytes = select_ws_bytes(N, (int)P);
     f.sel = take(f.sel_bytes);
-    f.amax_kept = reinterpret_cast<float*>(take(256));
+    f.amax_kept = b ? carve_select_ws(f.sel, N, (int)P).amax : nullptr;
     f.Xq = take(M * f.kpad * f.es);
     f.Wq = take((size_t)Cout * f.kpad * f.es);
     f.scale_w = reinterpret_cast<float*>(take((size_t)Cout * 4));
@@ -122,7 +122,7 @@ static wcc_status staged_impl(const void* x, const float* Wt, int N, int Cin, in
     if (s != WCC_OK) return s;
     if ((s = profile_mark(1, st)) != WCC_OK) return s;
     // B: joint shrinkage: kept index list, rank map, max |kept|
-    s = launch_select(f.nrm2, N, P, k, f.idx, nullptr, f.rank, f.amaxpos, f.amax_kept, f.sel, f.sel_bytes, st);
+    s = launch_select(f.nrm2, N, P, k, f.idx, nullptr, f.rank, f.amaxpos, true, f.sel, f.sel_bytes, st);
     if (s != WCC_OK) return s;
     if ((s = profile_mark(2, st)) != WCC_OK) return s;
     s = launch_weight_prep(Wt, Cout, Cin, f.kpad, bits, f.Wq, f.scale_w, st);
@@ -185,7 +185,7 @@ static FusedWs carve_fused_ws(void* ws, int N, int Cin, int Cout, int H, int W, 
     f.idx = reinterpret_cast<int32_t*>(take(M * 4));
     f.sel_bytes = select_ws_bytes(N, (int)P);
     f.sel = take(f.sel_bytes);
-    f.amax_kept = reinterpret_cast<float*>(take(256));
+    f.amax_kept = b ? carve_select_ws(f.sel, N, (int)P).amax : nullptr;
     f.Wq = take((size_t)Cout * f.kpad * f.es);
     f.scale_w = reinterpret_cast<float*>(take((size_t)Cout * 4));
     f.total = off;
@@ -213,7 +213,7 @@ static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, i
     if (s != WCC_OK) return s;
     if ((s = profile_mark(1, st)) != WCC_OK) return s;
     // joint shrinkage: index list, rank map, max |kept|
-    s = launch_select(f.nrm2, N, P, k, f.idx, nullptr, f.rank, f.amaxpos, f.amax_kept, f.sel, f.sel_bytes, st);
+    s = launch_select(f.nrm2, N, P, k, f.idx, nullptr, f.rank, f.amaxpos, true, f.sel, f.sel_bytes, st);
     if (s != WCC_OK) return s;
     if ((s = profile_mark(2, st)) != WCC_OK) return s;
     s = launch_weight_prep(Wt, Cout, Cin, f.kpad, bits, f.Wq, f.scale_w, st);
@@ -301,7 +301,7 @@ wcc_status wcc_select_topk(const float* nrm2, int N, int P, int k, int32_t* idx,
     if (k < 1 || k > P) return WCC_ERR_K;
     if (!aligned16(nrm2) || !aligned16(idx) || !aligned16(ws)) return WCC_ERR_ALIGN;
     if (ws_bytes < select_ws_bytes(N, P)) return WCC_ERR_WORKSPACE;
-    return launch_select(nrm2, N, P, k, idx, tau, nullptr, nullptr, nullptr, ws, ws_bytes, static_cast<cudaStream_t>(stream));
+    return launch_select(nrm2, N, P, k, idx, tau, nullptr, nullptr, false, ws, ws_bytes, static_cast<cudaStream_t>(stream));
 }
 
 wcc_status wcc_select_topk_static(const float* nrm2, int N, int P, int k, int32_t* idx, float* tau, void* stream)
@@ -316,7 +316,7 @@ wcc_status wcc_select_topk_static(const float* nrm2, int N, int P, int k, int32_
     wcc_status s = static_scratch_ptr(&scratch);                               // first call per device: address lookup
     if (s != WCC_OK) return s;
     // launch_select zeroes the histograms it accumulates into; everything else in the scratch is written before it is read
-    return launch_select(nrm2, N, P, k, idx, tau, nullptr, nullptr, nullptr, scratch, need, static_cast<cudaStream_t>(stream));
+    return launch_select(nrm2, N, P, k, idx, tau, nullptr, nullptr, false, scratch, need, static_cast<cudaStream_t>(stream));
 }
 
 wcc_status wcc_forward(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int Wd,
