@@ -55,7 +55,7 @@ template <typename T, int L, bool VEC, bool I8>
 __global__ void __launch_bounds__(128, 4)
 fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, const int32_t* __restrict__ rank,
                    const float* __restrict__ amax_kept, float qmax, const float* __restrict__ scale_w,
-                   int N, int Cin, int Cout, int H, int W, int k, int kpad, int npad, int nchunk, int tmem_cols,
+                   int N, int Cin, int Cout, int H, int W, int k, int kpad, int npad, int nchunk, int tmem_cols, int a_ksteps,
                    T* __restrict__ y, uint8_t* __restrict__ xq_tap, int32_t* __restrict__ acc_tap, int* __restrict__ status)
 {
     using TT = HaarTile<L>;
@@ -68,8 +68,8 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
     const int krow = kpad * ES;                       // bytes of K per row
     const int kchunks = krow / 16;
     using Ring = PatchRing<T>;
-    uint8_t* sA = sm;                                                   // [kchunks][256][16]
-    uint8_t* sB = sA + (size_t)kchunks * ROWS * 16;                     // [kchunks][npad][16]
+    uint8_t* sA = sm;                                                   // [2 * a_ksteps][256][16]
+    uint8_t* sB = sA + (size_t)a_ksteps * 2 * ROWS * 16;                // [kchunks][npad][16]
     int32_t* srank = reinterpret_cast<int32_t*>(sB + (size_t)kchunks * npad * 16);      // [8][32]
     Ctl* ctl = reinterpret_cast<Ctl*>(srank + 8 * 32);
     uint8_t* shared_region = reinterpret_cast<uint8_t*>(ctl + 1);       // phase 1: input rings; phase 3: transpose buffer
@@ -116,114 +116,136 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
 #pragma unroll
     for (int s = 0; s < 8; ++s) mul[s] = (rk[s] >= 0) ? inv : 0.0f;
 
-    // ---- phase 1: transform + quantize into the A operand --------------------------------------------
-    // Warp w takes the 8-channel units w, w+4, ...; inputs arrive LU channels at a time through its cp.async ring.
+    // ---- phases 1 + 2: transform + quantize into the A operand, tensor-core contraction ----------------
+    // A holds a_ksteps K steps (32 bytes of K each).  When the input channels need more than that (and there is a
+    // single chunk of output channels) the K range is done in two halves that accumulate into the same TMEM tile, so
+    // that A stays small enough for four CTAs per SM.
+    // Warp w takes the 8-channel units w, w+4, ... of a half; inputs arrive LU channels at a time through its ring.
     const T* xin = x + (size_t)n * Cin * P;
-    const int units = kpad / 8;
-    const int my_units = (units - warp + 3) / 4;
     constexpr int LU = Ring::LU, SUBS = 8 / LU;
+    constexpr int UPK = 32 / UNIT_BYTES;               // units per K step
+    const int ksteps = krow / 32;
+    const int halves = (a_ksteps < ksteps) ? 2 : 1;
     uint8_t* my_ring = shared_region + (VEC ? warp * RING2 * Ring::STAGE_BYTES : 0);
     const uint32_t my_ring_s = tc::smem_u32(my_ring);
-    const int nq = my_units * SUBS;                    // ring stages this warp will consume
-    auto chan0 = [&](int q) { return (warp + 4 * (q / SUBS)) * 8 + (q % SUBS) * LU; };
-    if (VEC) {
-#pragma unroll
-        for (int q = 0; q < RING2 - 1; ++q) Ring::issue(my_ring_s, q, xin, P, W, q < nq ? Cin : 0, chan0(q), lp, lane);
-    }
-    for (int ui = 0; ui < my_units; ++ui) {
-        const int u = warp + 4 * ui;
-        uint32_t packed[8][4];         // per slot: 8 int8 codes (2 words) or 8 bf16 values (4 words)
-#pragma unroll
-        for (int g = 0; g < 2; ++g) {                      // two groups of 4 channels
-            uint32_t code[4][8];                           // int8: float bits whose low byte is the code; bf16: value bits
-#pragma unroll
-            for (int dd4 = 0; dd4 < 4; ++dd4) {
-                const int d = g * 4 + dd4;                 // channel within the unit
-                const int sub = d / LU, dd = d % LU;       // ring stage within the unit, channel within the stage
-                const int q = ui * SUBS + sub;
-                if (VEC && dd == 0) {
-                    const int qn = q + RING2 - 1;
-                    Ring::issue(my_ring_s, qn % RING2, xin, P, W, qn < nq ? Cin : 0, chan0(qn), lp, lane);
-                    Ring::template wait<RING2 - 1>();
-                }
-                const int c = u * 8 + d;
-                float o[8];
-                if (c < Cin) {             // warp-uniform
-                    RawPatch rawp;
-                    if (VEC) Ring::read(my_ring, q % RING2, dd, lane, rawp);
-                    else load_patch<T, VEC>(xin + (size_t)c * P, W, lp, rawp);
-                    float p[2][4];
-                    unpack_patch<T>(rawp, p);
-                    haar_fwd_lane<L>(p, o, lane);
-                } else {
-#pragma unroll
-                    for (int s = 0; s < 8; ++s) o[s] = 0.0f;
-                }
-#pragma unroll
-                for (int s = 0; s < 8; s += 2) {
-                    float2 t = mul2(make_float2(o[s], o[s + 1]), make_float2(mul[s], mul[s + 1]));
-                    // int8: the low byte of (t + 1.5*2^23) is the two's complement code of rint(t); |t| <= qmax by construction
-                    // scalar adds on purpose: a packed add right after the packed product gets contracted into one
-                    // fused operation, which rounds once and changes codes that sit on a half-way point
-                    if (I8) t = make_float2(__fadd_rn(t.x, MAGIC), __fadd_rn(t.y, MAGIC));
-                    code[dd4][s] = __float_as_uint(t.x);
-                    code[dd4][s + 1] = __float_as_uint(t.y);
-                }
-            }
-#pragma unroll
-            for (int s = 0; s < 8; ++s) {
-                if (I8) {
-                    const uint32_t lo = __byte_perm(code[0][s], code[1][s], 0x0040);
-                    const uint32_t hi = __byte_perm(code[2][s], code[3][s], 0x0040);
-                    packed[s][g] = __byte_perm(lo, hi, 0x5410);
-                } else {
-                    packed[s][2 * g] = pack_bf16x2(__uint_as_float(code[0][s]), __uint_as_float(code[1][s]));
-                    packed[s][2 * g + 1] = pack_bf16x2(__uint_as_float(code[2][s]), __uint_as_float(code[3][s]));
-                }
-            }
-        }
-        const int j = (u * UNIT_BYTES) >> 4;               // 16-byte K chunk
-        const int off = (u * UNIT_BYTES) & 15;             // 0 or 8 (int8); always 0 (bf16)
-#pragma unroll
-        for (int s = 0; s < 8; ++s) {
-            uint8_t* dst = sA + ((size_t)j * ROWS + s * 32 + lane) * 16 + off;
-            if (I8) *reinterpret_cast<uint2*>(dst) = make_uint2(packed[s][0], packed[s][1]);
-            else *reinterpret_cast<uint4*>(dst) = make_uint4(packed[s][0], packed[s][1], packed[s][2], packed[s][3]);
-            if (xq_tap && rk[s] >= 0) {
-                uint8_t* g = xq_tap + ((size_t)n * k + rk[s]) * krow + (size_t)u * UNIT_BYTES;
-                if (I8) *reinterpret_cast<uint2*>(g) = make_uint2(packed[s][0], packed[s][1]);
-                else *reinterpret_cast<uint4*>(g) = make_uint4(packed[s][0], packed[s][1], packed[s][2], packed[s][3]);
-            }
-        }
-    }
-    if (VEC) Ring::template wait<0>();
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic-proxy writes -> visible to the tensor core
-    tc::fence_before();
-    __syncthreads();
-    tc::fence_after();
-    const uint32_t tmem = ctl->tmem_base;
-
-    // ---- phases 2 + 3, per chunk of output channels -------------------------------------------------
-    const int ksteps = krow / 32;
     const uint32_t a_addr = tc::smem_u32(sA), b_addr = tc::smem_u32(sB);
     volatile int no_abort = 0;
-    int chunk = 0;
+    uint32_t commits = 0;                              // MMA batches committed so far (same value in every thread)
+    uint32_t tmem = 0;
     bool ok = true;
-    for (int n0 = 0; n0 < npad; n0 += nchunk, ++chunk) {
-        const int cur = min(nchunk, npad - n0);
-        if (threadIdx.x == 0) {
-            const uint32_t idesc = (I8 ? (2u << 4) : (1u << 4)) | (1u << 7) | (1u << 10) |
-                                   ((uint32_t)(cur >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-            for (int b = 0; b < 2; ++b) {
-                for (int kk = 0; kk < ksteps; ++kk) {
-                    const uint64_t ad = smem_desc_plain(a_addr + (uint32_t)(kk * 2 * ROWS * 16 + b * 128 * 16), ROWS * 16, 128);
-                    const uint64_t bd = smem_desc_plain(b_addr + (uint32_t)(kk * 2 * npad * 16 + n0 * 16), (uint32_t)npad * 16, 128);
-                    tc::mma_ss<I8>(tmem + (uint32_t)(b * nchunk), ad, bd, idesc, kk > 0 ? 1u : 0u);
+    auto issue_mmas = [&](int ks0, int ks1, int ks_base, int n0, int cur) {   // thread 0 only
+        const uint32_t idesc = (I8 ? (2u << 4) : (1u << 4)) | (1u << 7) | (1u << 10) |
+                               ((uint32_t)(cur >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+        for (int b = 0; b < 2; ++b) {
+            for (int ks = ks0; ks < ks1; ++ks) {
+                const uint64_t ad = smem_desc_plain(a_addr + (uint32_t)((ks - ks_base) * 2 * ROWS * 16 + b * 128 * 16), ROWS * 16, 128);
+                const uint64_t bd = smem_desc_plain(b_addr + (uint32_t)(ks * 2 * npad * 16 + n0 * 16), (uint32_t)npad * 16, 128);
+                tc::mma_ss<I8>(tmem + (uint32_t)(b * nchunk), ad, bd, idesc, ks > 0 ? 1u : 0u);
+            }
+        }
+        tc::mma_commit(tc::smem_u32(&ctl->mma_done));
+    };
+
+    for (int h = 0; h < halves; ++h) {
+        const int ks0 = h * a_ksteps, ks1 = min(ksteps, ks0 + a_ksteps);
+        const int u0 = ks0 * UPK, u1 = ks1 * UPK;
+        if (h > 0) {                                   // the tensor core still reads A: wait for the first half
+            ok = tc::mbar_wait(tc::smem_u32(&ctl->mma_done), (commits - 1u) & 1u, &no_abort);
+            ok = __syncthreads_and(ok ? 1 : 0) != 0;
+            if (!ok) break;
+            tc::fence_after();
+        }
+        const int my_units = (u1 - u0 - warp + 3) / 4;
+        const int nq = my_units * SUBS;                // ring stages this warp will consume in this half
+        auto chan0 = [&](int q) { return (u0 + warp + 4 * (q / SUBS)) * 8 + (q % SUBS) * LU; };
+        if (VEC) {
+#pragma unroll
+            for (int q = 0; q < RING2 - 1; ++q) Ring::issue(my_ring_s, q, xin, P, W, q < nq ? Cin : 0, chan0(q), lp, lane);
+        }
+        for (int ui = 0; ui < my_units; ++ui) {
+            const int u = u0 + warp + 4 * ui;
+            uint32_t packed[8][4];     // per slot: 8 int8 codes (2 words) or 8 bf16 values (4 words)
+#pragma unroll
+            for (int g = 0; g < 2; ++g) {                  // two groups of 4 channels
+                uint32_t code[4][8];                       // int8: float bits whose low byte is the code; bf16: value bits
+#pragma unroll
+                for (int dd4 = 0; dd4 < 4; ++dd4) {
+                    const int d = g * 4 + dd4;             // channel within the unit
+                    const int sub = d / LU, dd = d % LU;   // ring stage within the unit, channel within the stage
+                    const int q = ui * SUBS + sub;
+                    if (VEC && dd == 0) {
+                        const int qn = q + RING2 - 1;
+                        Ring::issue(my_ring_s, qn % RING2, xin, P, W, qn < nq ? Cin : 0, chan0(qn), lp, lane);
+                        Ring::template wait<RING2 - 1>();
+                    }
+                    const int c = u * 8 + d;
+                    RawPatch rawp;
+                    if (VEC) {
+                        Ring::read(my_ring, q % RING2, dd, lane, rawp);      // channels beyond Cin arrive as zeros
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) rawp.w[i] = 0u;
+                        if (c < Cin) load_patch<T, VEC>(xin + (size_t)c * P, W, lp, rawp);
+                    }
+                    float p[2][4], o[8];
+                    unpack_patch<T>(rawp, p);
+                    haar_fwd_lane<L>(p, o, lane);
+#pragma unroll
+                    for (int s = 0; s < 8; s += 2) {
+                        float2 t = mul2(make_float2(o[s], o[s + 1]), make_float2(mul[s], mul[s + 1]));
+                        // int8: the low byte of (t + 1.5*2^23) is the two's complement code of rint(t); |t| <= qmax by
+                        // construction.  Scalar adds on purpose: a packed add right after the packed product gets
+                        // contracted into one fused operation, which rounds once and changes half-way codes.
+                        if (I8) t = make_float2(__fadd_rn(t.x, MAGIC), __fadd_rn(t.y, MAGIC));
+                        code[dd4][s] = __float_as_uint(t.x);
+                        code[dd4][s + 1] = __float_as_uint(t.y);
+                    }
+                }
+#pragma unroll
+                for (int s = 0; s < 8; ++s) {
+                    if (I8) {
+                        const uint32_t lo = __byte_perm(code[0][s], code[1][s], 0x0040);
+                        const uint32_t hi = __byte_perm(code[2][s], code[3][s], 0x0040);
+                        packed[s][g] = __byte_perm(lo, hi, 0x5410);
+                    } else {
+                        packed[s][2 * g] = pack_bf16x2(__uint_as_float(code[0][s]), __uint_as_float(code[1][s]));
+                        packed[s][2 * g + 1] = pack_bf16x2(__uint_as_float(code[2][s]), __uint_as_float(code[3][s]));
+                    }
                 }
             }
-            tc::mma_commit(tc::smem_u32(&ctl->mma_done));
+            const int j = ((u - u0) * UNIT_BYTES) >> 4;    // 16-byte K chunk inside this half's A
+            const int off = (u * UNIT_BYTES) & 15;         // 0 or 8 (int8); always 0 (bf16)
+#pragma unroll
+            for (int s = 0; s < 8; ++s) {
+                uint8_t* dst = sA + ((size_t)j * ROWS + s * 32 + lane) * 16 + off;
+                if (I8) *reinterpret_cast<uint2*>(dst) = make_uint2(packed[s][0], packed[s][1]);
+                else *reinterpret_cast<uint4*>(dst) = make_uint4(packed[s][0], packed[s][1], packed[s][2], packed[s][3]);
+                if (xq_tap && rk[s] >= 0) {
+                    uint8_t* g = xq_tap + ((size_t)n * k + rk[s]) * krow + (size_t)u * UNIT_BYTES;
+                    if (I8) *reinterpret_cast<uint2*>(g) = make_uint2(packed[s][0], packed[s][1]);
+                    else *reinterpret_cast<uint4*>(g) = make_uint4(packed[s][0], packed[s][1], packed[s][2], packed[s][3]);
+                }
+            }
         }
-        ok = tc::mbar_wait(tc::smem_u32(&ctl->mma_done), (uint32_t)chunk & 1u, &no_abort);
+        if (VEC) Ring::template wait<0>();
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic-proxy writes -> visible to the tensor core
+        tc::fence_before();
+        __syncthreads();
+        tc::fence_after();
+        tmem = ctl->tmem_base;
+        if (h + 1 < halves) {                          // first half of K: start accumulating now (single chunk of N)
+            if (threadIdx.x == 0) issue_mmas(ks0, ks1, ks0, 0, npad);
+            ++commits;
+        }
+    }
+
+    // ---- phases 2 (last K range) + 3, per chunk of output channels -----------------------------------
+    const int ks_last = (halves - 1) * a_ksteps;
+    for (int n0 = 0; ok && n0 < npad; n0 += nchunk) {
+        const int cur = min(nchunk, npad - n0);
+        if (threadIdx.x == 0) issue_mmas(ks_last, ksteps, ks_last, n0, cur);
+        ++commits;
+        ok = tc::mbar_wait(tc::smem_u32(&ctl->mma_done), (commits - 1u) & 1u, &no_abort);
         ok = __syncthreads_and(ok ? 1 : 0) != 0;
         if (!ok) break;
         tc::fence_after();
@@ -278,6 +300,7 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
     __syncthreads();
     if (warp == 0) {
         tc::fence_after();
+        tmem = ctl->tmem_base;
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)tmem_cols) : "memory");
     }
 }
@@ -299,8 +322,11 @@ static wcc_status fused_pass2_dispatch(const void* x, const void* Wq, const int3
     int tmem_cols = 32;
     while (tmem_cols < 2 * nchunk) tmem_cols <<= 1;
     const int kchunks = kpad * es / 16;
+    const int ksteps = kpad * es / 32;
+    // two K halves when that brings A down enough for a fourth CTA per SM (single chunk of output channels only)
+    const int a_ksteps = (npad <= nchunk && ksteps >= 4) ? (ksteps + 1) / 2 : ksteps;
     const size_t region = vmax((size_t)fz::SUB * 8 * 32 * 4, (size_t)4 * fz::RING2 * PatchRing<T>::STAGE_BYTES);
-    const size_t smem = 128 + (size_t)kchunks * fz::ROWS * 16 + (size_t)kchunks * npad * 16 + 8 * 32 * 4 + sizeof(fz::Ctl) +
+    const size_t smem = 128 + (size_t)a_ksteps * 2 * fz::ROWS * 16 + (size_t)kchunks * npad * 16 + 8 * 32 * 4 + sizeof(fz::Ctl) +
                         region + 16;
     if (smem > 200 * 1024 || (kpad * es) % 32 != 0) return WCC_ERR_SHAPE;
     const float qmax = i8 ? (float)((1 << (bits - 1)) - 1) : 1.0f;
@@ -311,7 +337,7 @@ static wcc_status fused_pass2_dispatch(const void* x, const void* Wq, const int3
     auto launch = [&](auto kern) -> wcc_status {
         WCC_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
         kern<<<(unsigned)ctas, 128, smem, st>>>(static_cast<const T*>(x), static_cast<const uint8_t*>(Wq), rank, amax_kept, qmax,
-                                                scale_w, N, Cin, Cout, H, W, k, kpad, npad, nchunk, tmem_cols,
+                                                scale_w, N, Cin, Cout, H, W, k, kpad, npad, nchunk, tmem_cols, a_ksteps,
                                                 static_cast<T*>(y), static_cast<uint8_t*>(xq_tap), acc_tap, status);
         WCC_LAUNCH_CHECK();
         return WCC_OK;

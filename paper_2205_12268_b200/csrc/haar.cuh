@@ -466,27 +466,28 @@ haar_norms_kernel(const T* __restrict__ x, int N, int C, int H, int W,
 #pragma unroll
         for (int d = 0; d < LU; ++d) {
             const int c = r * RC + warp * LU + d;
-            if (c < C) {                               // warp-uniform
-                RawPatch raw;
-                if (VEC) Ring::read(my_ring, r % RING, d, lane, raw);
-                else load_patch<T, VEC>(xin + (size_t)c * P, W, lp, raw);
-                float p[2][4], o[8];
-                unpack_patch<T>(raw, p);
-                haar_fwd_lane<L>(p, o, lane);
+            RawPatch raw;
+            if (VEC) {
+                Ring::read(my_ring, r % RING, d, lane, raw);          // channels beyond C arrive as zeros
+            } else {
 #pragma unroll
-                for (int s = 0; s < 8; s += 2) buf[warp * LU + d][s >> 1][lane] = make_float2(o[s], o[s + 1]);
+                for (int i = 0; i < 8; ++i) raw.w[i] = 0u;
+                if (c < C) load_patch<T, VEC>(xin + (size_t)c * P, W, lp, raw);
             }
+            float p[2][4], o[8];
+            unpack_patch<T>(raw, p);
+            haar_fwd_lane<L>(p, o, lane);
+#pragma unroll
+            for (int s = 0; s < 8; s += 2) buf[warp * LU + d][s >> 1][lane] = make_float2(o[s], o[s + 1]);
         }
         __syncthreads();
-        const int cnt = min(RC, C - r * RC);
+        // channels beyond C contribute fma(0, 0, acc) = acc and max(acc, 0) = acc: no special case needed
 #pragma unroll
         for (int c = 0; c < RC; ++c) {
-            if (c < cnt) {
-                const float2 v = buf[c][warp][lane];
-                nn = __ffma2_rn(v, v, nn);
-                a0 = fmaxf(a0, fabsf(v.x));
-                a1 = fmaxf(a1, fabsf(v.y));
-            }
+            const float2 v = buf[c][warp][lane];
+            nn = __ffma2_rn(v, v, nn);
+            a0 = fmaxf(a0, fabsf(v.x));
+            a1 = fmaxf(a1, fabsf(v.y));
         }
         __syncthreads();
     }
