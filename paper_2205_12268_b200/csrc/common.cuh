@@ -56,6 +56,18 @@ __device__ __forceinline__ float key_float(uint32_t k)
     return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
 }
 
+// Histogram increment with warp aggregation: lanes of a warp that hit the same bin elect one lane that adds their
+// count, so a bin that attracts most keys (typical for the leading digit of the norms) costs one shared-memory
+// atomic per warp instead of up to 32 serialized ones.  Must be reached by all 32 lanes (pred selects the ones that count).
+__device__ __forceinline__ void hist_add(uint32_t* h, uint32_t bin, bool pred)
+{
+    const unsigned active = __ballot_sync(0xFFFFFFFFu, pred);
+    if (pred) {
+        const unsigned peers = __match_any_sync(active, bin);
+        if ((int)(threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&h[bin], (uint32_t)__popc(peers));
+    }
+}
+
 // ---- geometry of one call -------------------------------------------------------------------
 struct Geom {
     int N, C, H, W, L;
@@ -79,7 +91,7 @@ wcc_status launch_scatter_inv(const int32_t* acc, int ldc, bool acc_is_float, co
 size_t select_ws_bytes(int N, int P);
 wcc_status launch_select(const float* nrm2, int N, int P, int k, int32_t* idx, float* tau,
                          int32_t* rank, const float* amaxpos, bool want_amax,
-                         void* ws, size_t ws_bytes, cudaStream_t st);
+                         void* ws, size_t ws_bytes, cudaStream_t st, bool hist1_ready = false);
 
 // Weight quantization (bits >= 2: int8 codes + per-row scale; bits == 0: bf16 copy), rows padded to kpad.
 wcc_status launch_weight_prep(const float* Wt, int Cout, int Cin, int kpad, int bits,

@@ -13,14 +13,11 @@ __device__ __forceinline__ int quant_code(float v, float inv, float qmax)
     return (int)r;
 }
 
-// One warp per output channel.  bits >= 2: Wq int8 [Cout][kpad] (zero padded) and scale_w[o] = max|w| / qmax.
+// One warp per output channel o.  bits >= 2: Wq int8 [Cout][kpad] (zero padded) and scale_w[o] = max|w| / qmax.
 // bits == 0: bf16 copy of the row, zero padded.
-__global__ void __launch_bounds__(128)
-weight_prep_kernel(const float* __restrict__ Wt, int Cout, int Cin, int kpad, int bits,
-                   void* __restrict__ Wq, float* __restrict__ scale_w)
+__device__ __forceinline__ void weight_prep_row(const float* __restrict__ Wt, int o, int Cin, int kpad, int bits,
+                                                void* __restrict__ Wq, float* __restrict__ scale_w)
 {
-    const int o = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (o >= Cout) return;
     const int lane = threadIdx.x & 31;
     const float* w = Wt + (size_t)o * Cin;
     if (bits == 0) {
@@ -37,6 +34,14 @@ weight_prep_kernel(const float* __restrict__ Wt, int Cout, int Cin, int kpad, in
     int8_t* dst = static_cast<int8_t*>(Wq) + (size_t)o * kpad;
     for (int c = lane; c < kpad; c += 32) dst[c] = (c < Cin) ? (int8_t)quant_code(w[c], inv, qmax) : (int8_t)0;
     if (lane == 0) scale_w[o] = __fdiv_rn(m, qmax);
+}
+
+__global__ void __launch_bounds__(128)
+weight_prep_kernel(const float* __restrict__ Wt, int Cout, int Cin, int kpad, int bits,
+                   void* __restrict__ Wq, float* __restrict__ scale_w)
+{
+    const int o = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (o < Cout) weight_prep_row(Wt, o, Cin, kpad, bits, Wq, scale_w);
 }
 
 // One thread per kept position (row r = n*k + j of the compressed matrix): reads coef[n][c][idx[n][j]] for every

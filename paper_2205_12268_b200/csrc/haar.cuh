@@ -428,13 +428,30 @@ struct PatchRing {
 // transforms channels [w * LU, (w + 1) * LU) of the round in registers and hands the slot values over through shared
 // memory; then the 128 threads run the fused multiply-add chain of two positions each (warp w: slots 2w and 2w+1
 // of every lane) over the round's channels in ascending order, so the sum is the same sequential chain a single
-// thread would build.  Inputs arrive through the per-warp cp.async ring (RING stages ahead).  Nothing but the
-// norms and the per-position max |coef| is written.
+// thread would build.  Inputs arrive through the per-warp cp.async ring (RING stages ahead).  Only the norms and
+// the per-position max |coef| are written, plus on request (NormsExtra): the coefficient map (tests), round 1 of
+// the select's histogram (top 11 bits of the order-preserving key of every norm), and, in extra CTAs appended to
+// the grid, the quantized weights (one warp per output channel), which saves a launch of its own.
+struct NormsExtra {
+    float* coef;          // fp32 [N][C][P] or NULL
+    uint32_t* hist1;      // [N][3][2048] (round 1 first), zeroed by the caller, or NULL
+    const float* Wt;      // weights to prepare in the extra CTAs, or NULL
+    void* Wq;
+    float* scale_w;
+    int Cout, kpad, bits;
+    int tiles;            // CTAs that transform; CTAs beyond prepare weights
+};
+
 template <typename T, int L, bool VEC>
 __global__ void __launch_bounds__(128)
 haar_norms_kernel(const T* __restrict__ x, int N, int C, int H, int W,
-                  float* __restrict__ nrm2, float* __restrict__ amaxpos)
+                  float* __restrict__ nrm2, float* __restrict__ amaxpos, const NormsExtra ex)
 {
+    if ((int)blockIdx.x >= ex.tiles) {                 // weight preparation CTAs
+        const int o = ((int)blockIdx.x - ex.tiles) * 4 + (int)(threadIdx.x >> 5);
+        if (o < ex.Cout) weight_prep_row(ex.Wt, o, C, ex.kpad, ex.bits, ex.Wq, ex.scale_w);
+        return;
+    }
     using TT = HaarTile<L>;
     using Ring = PatchRing<T>;
     constexpr int LU = Ring::LU, RC = 4 * LU;          // channels per warp and per round
@@ -479,6 +496,7 @@ haar_norms_kernel(const T* __restrict__ x, int N, int C, int H, int W,
             haar_fwd_lane<L>(p, o, lane);
 #pragma unroll
             for (int s = 0; s < 8; s += 2) buf[warp * LU + d][s >> 1][lane] = make_float2(o[s], o[s + 1]);
+            if (ex.coef && c < C) store_slots<L, VEC>(ex.coef + ((size_t)n * C + c) * P, lp, o);
         }
         __syncthreads();
         // channels beyond C contribute fma(0, 0, acc) = acc and max(acc, 0) = acc: no special case needed
@@ -518,6 +536,11 @@ haar_norms_kernel(const T* __restrict__ x, int N, int C, int H, int W,
             if (ok0) am[p0] = a0;
             if (ok1) am[p1] = a1;
         }
+    }
+    if (ex.hist1) {                                    // norms are >= +0: key = bits | sign bit, digit = top 11 bits
+        uint32_t* h = ex.hist1 + (size_t)n * 3 * 2048;
+        hist_add(h, float_key(n0) >> 21, ok0);
+        hist_add(h, float_key(n1) >> 21, ok1);
     }
 }
 
@@ -609,7 +632,9 @@ static wcc_status haar_fwd_dispatch(const void* x, int N, int C, int H, int W, f
     constexpr int D = (sizeof(T) == 4) ? 4 : 8;
     const long long warps = (long long)N * ceil_div(W, TT::TW) * (H / TT::TH);
     if (!coef && nrm2) {          // norms only: four warps per tile
-        haar_norms_kernel<T, L, VEC><<<(unsigned)warps, 128, 0, st>>>(static_cast<const T*>(x), N, C, H, W, nrm2, amaxpos);
+        NormsExtra ex = {};
+        ex.tiles = (int)warps;
+        haar_norms_kernel<T, L, VEC><<<(unsigned)warps, 128, 0, st>>>(static_cast<const T*>(x), N, C, H, W, nrm2, amaxpos, ex);
         WCC_LAUNCH_CHECK();
         return WCC_OK;
     }
@@ -631,6 +656,27 @@ static wcc_status haar_fwd_dispatch(const void* x, int N, int C, int H, int W, f
             return FN<__nv_bfloat16, 3, true>(__VA_ARGS__);                                          \
         }                                                                                            \
     } while (0)
+
+template <typename T, int L, bool VEC>
+static wcc_status haar_norms_dispatch(const void* x, int N, int C, int H, int W, float* nrm2, float* amaxpos,
+                                      NormsExtra ex, cudaStream_t st)
+{
+    using TT = HaarTile<L>;
+    const long long tiles = (long long)N * ceil_div(W, TT::TW) * (H / TT::TH);
+    ex.tiles = (int)tiles;
+    const long long grid = tiles + (ex.Wt ? ceil_div(ex.Cout, 4) : 0);
+    haar_norms_kernel<T, L, VEC><<<(unsigned)grid, 128, 0, st>>>(static_cast<const T*>(x), N, C, H, W, nrm2, amaxpos, ex);
+    WCC_LAUNCH_CHECK();
+    return WCC_OK;
+}
+
+// First pass of the fused layer (see haar_norms_kernel); ex.tiles is filled in here.
+wcc_status launch_haar_norms(const void* x, int N, int C, int H, int W, int L, wcc_dtype dt,
+                             float* nrm2, float* amaxpos, const NormsExtra& ex, cudaStream_t st)
+{
+    const bool vec = (W % 4) == 0;
+    WCC_DISPATCH_TLV(haar_norms_dispatch, dt, L, vec, x, N, C, H, W, nrm2, amaxpos, ex, st);
+}
 
 wcc_status launch_haar_fwd(const void* x, int N, int C, int H, int W, int L, wcc_dtype dt,
                            float* coef, float* nrm2, float* amaxpos, cudaStream_t st)

@@ -1,8 +1,8 @@
 // libwcc: C-ABI entry points (see include/wcc.h).  One translation unit: the kernels live in the *.cuh files.
 #include "common.cuh"
+#include "gather.cuh"
 #include "haar.cuh"
 #include "select.cuh"
-#include "gather.cuh"
 #include "contract.cuh"
 #include "fused.cuh"
 
@@ -207,17 +207,22 @@ static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, i
     const int P = H * W, M = N * k;
 
     if ((s = profile_mark(0, st)) != WCC_OK) return s;
-    // first pass over x: transform in registers, keep only the channel norms and the per-position max |coef|
-    // (the coefficient map is written only when a test asks for it)
-    s = launch_haar_fwd(x, N, Cin, H, W, L, dt, taps ? taps->coef : nullptr, f.nrm2, f.amaxpos, st);
+    // first pass over x: transform in registers, keep only the channel norms and the per-position max |coef| (the
+    // coefficient map is written only when a test asks for it).  The same launch fills round 1 of the select's
+    // histogram and quantizes the weights in a few extra CTAs.
+    const SelectWs sw = carve_select_ws(f.sel, N, P);
+    WCC_CUDA_TRY(cudaMemsetAsync(sw.hist, 0, sw.zero_bytes, st));          // histograms, max |kept|, barrier counters
+    NormsExtra ex = {};
+    ex.coef = taps ? taps->coef : nullptr;
+    ex.hist1 = sw.hist;
+    ex.Wt = Wt; ex.Wq = f.Wq; ex.scale_w = f.scale_w; ex.Cout = Cout; ex.kpad = f.kpad; ex.bits = bits;
+    s = launch_haar_norms(x, N, Cin, H, W, L, dt, f.nrm2, f.amaxpos, ex, st);
     if (s != WCC_OK) return s;
     if ((s = profile_mark(1, st)) != WCC_OK) return s;
     // joint shrinkage: index list, rank map, max |kept|
-    s = launch_select(f.nrm2, N, P, k, f.idx, nullptr, f.rank, f.amaxpos, true, f.sel, f.sel_bytes, st);
+    s = launch_select(f.nrm2, N, P, k, f.idx, nullptr, f.rank, f.amaxpos, true, f.sel, f.sel_bytes, st, true);
     if (s != WCC_OK) return s;
     if ((s = profile_mark(2, st)) != WCC_OK) return s;
-    s = launch_weight_prep(Wt, Cout, Cin, f.kpad, bits, f.Wq, f.scale_w, st);
-    if (s != WCC_OK) return s;
     if ((s = profile_mark(3, st)) != WCC_OK) return s;
     // second pass over x: transform, mask + quantize, tensor-core contraction, dequantize, inverse, store
     void* xq_tap = taps ? (bits >= 2 ? static_cast<void*>(taps->Xq) : taps->Xb) : nullptr;

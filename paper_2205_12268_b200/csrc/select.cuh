@@ -10,9 +10,12 @@
 // in which atomics land.
 #pragma once
 
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 
 namespace wcc {
+namespace cg = cooperative_groups;
 
 constexpr int SEL_THREADS = 256;
 constexpr int SEL_KPT = 8;                           // keys per thread
@@ -164,10 +167,9 @@ select_hist_kernel(const float* __restrict__ nrm2, int P, int k, uint32_t* __res
     load_keys(nrm2 + (size_t)n * P, P, blockIdx.x * SEL_CHUNK + threadIdx.x * SEL_KPT, key, ok);
 #pragma unroll
     for (int i = 0; i < SEL_KPT; ++i) {
-        if (!ok[i]) continue;
-        if (R == 1) atomicAdd(&sh[key[i] >> 21], 1u);
-        if (R == 2 && (key[i] >> 21) == prefix) atomicAdd(&sh[(key[i] >> 10) & 0x7FFu], 1u);
-        if (R == 3 && (key[i] >> 10) == prefix) atomicAdd(&sh[key[i] & 0x3FFu], 1u);
+        if (R == 1) hist_add(sh, key[i] >> 21, ok[i]);
+        if (R == 2) hist_add(sh, (key[i] >> 10) & 0x7FFu, ok[i] && (key[i] >> 21) == prefix);
+        if (R == 3) hist_add(sh, key[i] & 0x3FFu, ok[i] && (key[i] >> 10) == prefix);
     }
     __syncthreads();
     uint32_t* out = hn + (R - 1) * SEL_BINS;
@@ -353,8 +355,7 @@ select_coop_kernel(const float* __restrict__ nrm2, int P, int k, uint32_t* __res
 
     // round 1
 #pragma unroll
-    for (int i = 0; i < SEL_KPT; ++i)
-        if (okk[i]) atomicAdd(&sh[key[i] >> 21], 1u);
+    for (int i = 0; i < SEL_KPT; ++i) hist_add(sh, key[i] >> 21, okk[i]);
     flush_hist<SEL_BINS>(sh, hn);
     bool good = image_barrier(barn, chunks);
     // round 2
@@ -362,8 +363,7 @@ select_coop_kernel(const float* __restrict__ nrm2, int P, int k, uint32_t* __res
     find_bin<SEL_BINS>(hn, (uint32_t)k, sh_scan, sh_res, b1, above);
     const uint32_t k1 = (uint32_t)k - above;
 #pragma unroll
-    for (int i = 0; i < SEL_KPT; ++i)
-        if (okk[i] && (key[i] >> 21) == b1) atomicAdd(&sh[(key[i] >> 10) & 0x7FFu], 1u);
+    for (int i = 0; i < SEL_KPT; ++i) hist_add(sh, (key[i] >> 10) & 0x7FFu, okk[i] && (key[i] >> 21) == b1);
     flush_hist<SEL_BINS>(sh, hn + SEL_BINS);
     good = image_barrier(barn, 2 * chunks) && good;
     // round 3
@@ -372,8 +372,7 @@ select_coop_kernel(const float* __restrict__ nrm2, int P, int k, uint32_t* __res
     const uint32_t k2 = k1 - above;
     const uint32_t prefix = (b1 << 11) | b2;
 #pragma unroll
-    for (int i = 0; i < SEL_KPT; ++i)
-        if (okk[i] && (key[i] >> 10) == prefix) atomicAdd(&sh[key[i] & 0x3FFu], 1u);
+    for (int i = 0; i < SEL_KPT; ++i) hist_add(sh, key[i] & 0x3FFu, okk[i] && (key[i] >> 10) == prefix);
     flush_hist<1024>(sh, hn + 2 * SEL_BINS);
     good = image_barrier(barn, 3 * chunks) && good;
     // threshold, chunk counts
@@ -435,13 +434,274 @@ select_coop_kernel(const float* __restrict__ nrm2, int P, int k, uint32_t* __res
     if (!good && threadIdx.x == 0) atomicExch(status, (int)WCC_ERR_TIMEOUT);
 }
 
+// ---- the select as one thread-block cluster per image -------------------------------------------------
+// Up to 8 CTAs of 1024 threads form one cluster per image (P <= 131072 keys, at most 16 per thread, held in
+// registers).  Each CTA histograms its keys in shared memory; the histograms are combined through distributed
+// shared memory (every CTA sums one slice of the bins over all CTAs, then all CTAs read the slice totals and the
+// slice that holds the k-th key), and the phases are separated by hardware cluster barriers: no global-memory
+// round trips, no spinning, no scratch memory.
+constexpr int CL_THREADS = 1024;
+constexpr int CL_MAXKPT = 16;
+constexpr int CL_MAXCS = 8;
+
+struct ClusterSmem {
+    uint32_t hist[SEL_BINS];
+    uint32_t slice[SEL_BINS];       // sums over all CTAs of this CTA's slice of bins
+    uint32_t warp_sums[CL_THREADS / 32 + 1];
+    uint32_t slice_total;
+    uint32_t cnt[2];                // keys above / equal to the threshold in this CTA
+    uint32_t res[2];
+    uint32_t tot[CL_MAXCS];
+    uint32_t amax;
+};
+
+// exclusive scan over the threads of the block (256, 512 or 1024); every thread also gets the total
+__device__ __forceinline__ uint32_t block_scan_1024(uint32_t v, uint32_t* warp_sums, uint32_t* total)
+{
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    uint32_t inc = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+        if (lane >= d) inc += t;
+    }
+    if (lane == 31) warp_sums[w] = inc;
+    __syncthreads();
+    if (w == 0) {
+        const uint32_t s = (lane < nw) ? warp_sums[lane] : 0u;
+        uint32_t si = s;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, si, d);
+            if (lane >= d) si += t;
+        }
+        if (lane < nw) warp_sums[lane] = si - s;
+        if (lane == 31) warp_sums[32] = si;
+    }
+    __syncthreads();
+    const uint32_t res = warp_sums[w] + inc - v;
+    *total = warp_sums[32];
+    __syncthreads();
+    return res;
+}
+
+// After every CTA has filled sm.hist: find the bin holding the krem-th key from the top over the whole cluster.
+// nbins = 2048 or 1024.  Contains two cluster barriers.  Every thread of every CTA returns the same (bin, above).
+__device__ __forceinline__ void cluster_find_bin(cg::cluster_group& cluster, ClusterSmem& sm, int cs, int crank, int nbins,
+                                                 uint32_t krem, uint32_t& bin, uint32_t& above)
+{
+    const int B = nbins / cs;                        // bins per slice: 128 .. 2048
+    cluster.sync();                                  // all local histograms complete
+    uint32_t mine = 0;
+    for (int t = threadIdx.x; t < B; t += blockDim.x) {
+        uint32_t sum = 0;
+        for (int r = 0; r < cs; ++r) sum += cluster.map_shared_rank(sm.hist, r)[crank * B + t];
+        sm.slice[t] = sum;
+        mine += sum;
+    }
+    uint32_t total;
+    block_scan_1024(mine, sm.warp_sums, &total);
+    if (threadIdx.x == 0) sm.slice_total = total;
+    cluster.sync();                                  // all slices and slice totals complete
+    if (threadIdx.x < cs) sm.tot[threadIdx.x] = *cluster.map_shared_rank(&sm.slice_total, threadIdx.x);
+    __syncthreads();
+    uint32_t above_slices = 0;
+    int target = 0;
+    for (int r = cs - 1; r >= 0; --r) {              // slices from the top bins downwards
+        const uint32_t t = sm.tot[r];
+        if (krem <= above_slices + t) { target = r; break; }
+        above_slices += t;
+    }
+    const uint32_t kin = krem - above_slices;        // rank inside the target slice, from its top bin
+    const uint32_t* rs = cluster.map_shared_rank(sm.slice, target);
+    // thread t covers the `per` bins (B-1 - t*per) downwards of the slice (per <= 8)
+    const int per = (B + (int)blockDim.x - 1) / (int)blockDim.x;
+    const int top = B - 1 - (int)threadIdx.x * per;
+    uint32_t c[8], mysum = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        c[i] = (i < per && top - i >= 0) ? rs[top - i] : 0u;
+        mysum += c[i];
+    }
+    uint32_t tot2;
+    const uint32_t before = block_scan_1024(mysum, sm.warp_sums, &tot2);
+    if (before < kin && kin <= before + mysum) {
+        uint32_t a = before;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            if (a < kin && kin <= a + c[i]) { sm.res[0] = (uint32_t)(target * B + top - i); sm.res[1] = above_slices + a; }
+            a += c[i];
+        }
+    }
+    __syncthreads();
+    bin = sm.res[0];
+    above = sm.res[1];
+    __syncthreads();
+}
+
+
+// Find the bin of a complete 2048-bin histogram in global memory that holds the krem-th key from the top; block of
+// 256, 512 or 1024 threads, every thread returns the same values.
+__device__ __forceinline__ void block_find_bin_2048(const uint32_t* __restrict__ h, uint32_t krem, ClusterSmem& sm,
+                                                    uint32_t& bin, uint32_t& above)
+{
+    const int per = SEL_BINS / (int)blockDim.x;            // 8, 4 or 2
+    const int top = SEL_BINS - 1 - (int)threadIdx.x * per;
+    uint32_t c[8], mysum = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        c[i] = (i < per) ? __ldcg(&h[top - i]) : 0u;
+        mysum += c[i];
+    }
+    uint32_t tot;
+    const uint32_t before = block_scan_1024(mysum, sm.warp_sums, &tot);
+    if (before < krem && krem <= before + mysum) {
+        uint32_t a = before;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            if (a < krem && krem <= a + c[i]) { sm.res[0] = (uint32_t)(top - i); sm.res[1] = a; }
+            a += c[i];
+        }
+    }
+    __syncthreads();
+    bin = sm.res[0];
+    above = sm.res[1];
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(CL_THREADS, 1)
+select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int32_t* __restrict__ idx, float* __restrict__ tau,
+                      int32_t* __restrict__ rank, const float* __restrict__ amaxpos, float* __restrict__ amax_kept,
+                      const uint32_t* __restrict__ hist1)
+{
+    __shared__ ClusterSmem sm;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int cs = (int)cluster.num_blocks(), crank = (int)cluster.block_rank();
+    const int n = blockIdx.y;
+    const float* v = nrm2 + (size_t)n * P;
+    const int base = (crank * (int)blockDim.x + (int)threadIdx.x) * kpt;  // kpt consecutive keys per thread
+
+    uint32_t key[CL_MAXKPT];
+#pragma unroll
+    for (int i = 0; i < CL_MAXKPT; ++i) key[i] = (i < kpt && base + i < P) ? float_key(v[base + i]) : 0u;
+    auto valid = [&](int i) { return i < kpt && base + i < P; };
+
+    for (int i = threadIdx.x; i < SEL_BINS; i += blockDim.x) sm.hist[i] = 0u;
+    if (threadIdx.x == 0) sm.amax = 0u;
+    __syncthreads();
+    // round 1: top 11 bits.  When the producer of the norms already histogrammed them (hist1: [N][3][2048], round 1
+    // first), only the bin search is left.
+    uint32_t b1, above;
+    if (hist1) {
+        block_find_bin_2048(hist1 + (size_t)n * 3 * SEL_BINS, (uint32_t)k, sm, b1, above);
+    } else {
+#pragma unroll
+        for (int i = 0; i < CL_MAXKPT; ++i)
+            if (i < kpt) hist_add(sm.hist, key[i] >> 21, valid(i));
+        cluster_find_bin(cluster, sm, cs, crank, SEL_BINS, (uint32_t)k, b1, above);
+        for (int i = threadIdx.x; i < SEL_BINS; i += blockDim.x) sm.hist[i] = 0u;
+        __syncthreads();
+    }
+    const uint32_t k1 = (uint32_t)k - above;
+    // round 2: next 11 bits of the keys that match
+#pragma unroll
+    for (int i = 0; i < CL_MAXKPT; ++i)
+        if (i < kpt) hist_add(sm.hist, (key[i] >> 10) & 0x7FFu, valid(i) && (key[i] >> 21) == b1);
+    uint32_t b2;
+    cluster_find_bin(cluster, sm, cs, crank, SEL_BINS, k1, b2, above);
+    const uint32_t k2 = k1 - above;
+    const uint32_t prefix = (b1 << 11) | b2;
+    // round 3: last 10 bits
+    for (int i = threadIdx.x; i < SEL_BINS; i += blockDim.x) sm.hist[i] = 0u;
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < CL_MAXKPT; ++i)
+        if (i < kpt) hist_add(sm.hist, key[i] & 0x3FFu, valid(i) && (key[i] >> 10) == prefix);
+    uint32_t b3;
+    cluster_find_bin(cluster, sm, cs, crank, 1024, k2, b3, above);
+    const uint32_t tkey = (prefix << 10) | b3, need_eq = k2 - above;
+    if (tau && crank == 0 && threadIdx.x == 0) tau[n] = key_float(tkey);
+
+    // ordered compaction
+    uint32_t gt = 0, eq = 0;
+#pragma unroll
+    for (int i = 0; i < CL_MAXKPT; ++i) {
+        if (!valid(i)) continue;
+        gt += key[i] > tkey;
+        eq += key[i] == tkey;
+    }
+    uint32_t tot_gt, tot_eq;
+    uint32_t gt_before = block_scan_1024(gt, sm.warp_sums, &tot_gt);
+    uint32_t eq_before = block_scan_1024(eq, sm.warp_sums, &tot_eq);
+    if (threadIdx.x == 0) { sm.cnt[0] = tot_gt; sm.cnt[1] = tot_eq; }
+    cluster.sync();
+    for (int r = 0; r < crank; ++r) {
+        const uint32_t* c = cluster.map_shared_rank(sm.cnt, r);
+        gt_before += c[0];
+        eq_before += c[1];
+    }
+    float amax = 0.0f;
+#pragma unroll
+    for (int i = 0; i < CL_MAXKPT; ++i) {
+        if (!valid(i)) continue;
+        const bool is_gt = key[i] > tkey, is_eq = key[i] == tkey;
+        const bool keep = is_gt || (is_eq && eq_before < need_eq);
+        const uint32_t pos = gt_before + min(eq_before, need_eq);
+        if (keep) {
+            idx[(size_t)n * k + pos] = base + i;
+            if (amaxpos) amax = fmaxf(amax, amaxpos[(size_t)n * P + base + i]);
+        }
+        if (rank) rank[(size_t)n * P + base + i] = keep ? (int32_t)pos : -1;
+        gt_before += is_gt;
+        eq_before += is_eq;
+    }
+    if (amax_kept) {
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, d));
+        if ((threadIdx.x & 31) == 0) atomicMax(&sm.amax, __float_as_uint(amax));
+        __syncthreads();
+        if (threadIdx.x == 0 && sm.amax) atomicMax(reinterpret_cast<uint32_t*>(amax_kept), sm.amax);
+    }
+    cluster.sync();                                  // nobody leaves while a neighbour may still read its shared memory
+}
+
+// hist1_ready: the caller has already cleared the zero region of the workspace (carve_select_ws(...).hist,
+// zero_bytes) and filled round 1 of the histogram (top 11 key bits of every norm) before this call.
 wcc_status launch_select(const float* nrm2, int N, int P, int k, int32_t* idx, float* tau,
                          int32_t* rank, const float* amaxpos, bool want_amax,
-                         void* ws, size_t ws_bytes, cudaStream_t st)
+                         void* ws, size_t ws_bytes, cudaStream_t st, bool hist1_ready)
 {
     if (ws_bytes < select_ws_bytes(N, P)) return WCC_ERR_WORKSPACE;
     const SelectWs s = carve_select_ws(ws, N, P);
     float* amax_kept = want_amax ? s.amax : nullptr;
+    // one cluster per image while its keys fit in the registers of 8 x 1024 threads
+    if (P <= CL_MAXCS * CL_THREADS * CL_MAXKPT) {
+        // as many CTAs per image as useful, then as few threads as hold the keys (<= 16 each): the per-thread cost of
+        // the scans and barriers is fixed, so fewer, busier threads finish sooner
+        int cs = 1;
+        while (cs < CL_MAXCS && cs * 512 < P) cs <<= 1;
+        int threads = 256;
+        while (threads < CL_THREADS && (long long)cs * threads * CL_MAXKPT < P) threads <<= 1;
+        const int kpt = ceil_div(P, cs * threads);
+        if (amax_kept && !hist1_ready) WCC_CUDA_TRY(cudaMemsetAsync(amax_kept, 0, sizeof(float), st));
+        const uint32_t* hist1 = hist1_ready ? s.hist : nullptr;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(cs, N);
+        cfg.blockDim = dim3(threads);
+        cfg.dynamicSmemBytes = 0;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = cs;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        WCC_CUDA_TRY(cudaLaunchKernelEx(&cfg, select_cluster_kernel, nrm2, P, k, kpt, idx, tau, rank, amaxpos, amax_kept, hist1));
+        WCC_LAUNCH_CHECK();
+        return WCC_OK;
+    }
+    // (a round-1 histogram supplied by the caller is not used by these paths: they start from a clean slate)
     WCC_CUDA_TRY(cudaMemsetAsync(s.hist, 0, s.zero_bytes, st));
     const dim3 grid(s.chunks, N);
 

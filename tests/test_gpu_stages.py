@@ -90,6 +90,17 @@ def test_select_random(wcc, P):
         _check_select(wcc, nrm, k)
 
 
+@pytest.mark.parametrize("N,P", [(2, 200000), (10, 200000)])
+def test_select_large_images_other_code_paths(wcc, N, P):
+    """More keys per image than one cluster holds: the cooperative single kernel (few CTAs) and the one-kernel-per-phase
+    path (more CTAs than can be resident at once)."""
+    rng = np.random.default_rng(N)
+    nrm = (rng.random((N, P)) ** 3).astype(np.float32)
+    nrm[:, ::7] = nrm[:, 3:4]                                         # a long run of equal norms per image
+    for k in (1, 70000, P - 5):
+        _check_select(wcc, nrm, k)
+
+
 def test_select_ties_and_special_values(wcc):
     rng = np.random.default_rng(3)
     P = 6000
