@@ -376,10 +376,10 @@ haar_fwd_kernel(const T* __restrict__ x, int N, int C, int H, int W,
 // registers held while the copy flies) and later reads back exactly the bytes it copied, so no barrier is needed:
 // only the thread's own cp.async groups are waited for.  A stage holds LU channels; slot of (stage, channel d,
 // row r, lane) = ((stage * LU + d) * 2 + r) * 32 + lane, ROWB bytes each (conflict-free: lanes are contiguous).
-template <typename T>
+template <typename T, int LU_ = (sizeof(T) == 2) ? 4 : 2>
 struct PatchRing {
     static constexpr int ROWB = 4 * (int)sizeof(T);              // bytes of one patch row: 8 (bf16) or 16 (fp32)
-    static constexpr int LU = (sizeof(T) == 2) ? 4 : 2;          // channels per stage: 2 KB per warp and stage
+    static constexpr int LU = LU_;                               // channels per stage (default: 2 KB per warp and stage)
     static constexpr int STAGE_BYTES = LU * 2 * 32 * ROWB;
 
     // start the copies of channels [c0, c0 + LU) of one image into `stage`; always commits one group
@@ -442,22 +442,24 @@ struct NormsExtra {
     int tiles;            // CTAs that transform; CTAs beyond prepare weights
 };
 
+constexpr int NORMS_WARPS = 8;     // warps per CTA: the transform is issue-latency bound, more warps hide it
+
 template <typename T, int L, bool VEC>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(NORMS_WARPS * 32)
 haar_norms_kernel(const T* __restrict__ x, int N, int C, int H, int W,
                   float* __restrict__ nrm2, float* __restrict__ amaxpos, const NormsExtra ex)
 {
     if ((int)blockIdx.x >= ex.tiles) {                 // weight preparation CTAs
-        const int o = ((int)blockIdx.x - ex.tiles) * 4 + (int)(threadIdx.x >> 5);
+        const int o = ((int)blockIdx.x - ex.tiles) * NORMS_WARPS + (int)(threadIdx.x >> 5);
         if (o < ex.Cout) weight_prep_row(ex.Wt, o, C, ex.kpad, ex.bits, ex.Wq, ex.scale_w);
         return;
     }
     using TT = HaarTile<L>;
-    using Ring = PatchRing<T>;
-    constexpr int LU = Ring::LU, RC = 4 * LU;          // channels per warp and per round
+    using Ring = PatchRing<T, (sizeof(T) == 2) ? 2 : 1>;
+    constexpr int LU = Ring::LU, RC = NORMS_WARPS * LU;   // channels per warp and per round
     constexpr int RING = 4;                            // stages per warp
     __shared__ float2 buf[RC][4][32];                  // [channel of the round][slot pair][lane]
-    __shared__ __align__(16) uint8_t ring_mem[VEC ? 4 * RING * Ring::STAGE_BYTES : 16];
+    __shared__ __align__(16) uint8_t ring_mem[VEC ? NORMS_WARPS * RING * Ring::STAGE_BYTES : 16];
     const int tiles_x = (W + TT::TW - 1) / TT::TW, tiles_y = H / TT::TH;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int n, ty, tx;
@@ -499,17 +501,21 @@ haar_norms_kernel(const T* __restrict__ x, int N, int C, int H, int W,
             if (ex.coef && c < C) store_slots<L, VEC>(ex.coef + ((size_t)n * C + c) * P, lp, o);
         }
         __syncthreads();
-        // channels beyond C contribute fma(0, 0, acc) = acc and max(acc, 0) = acc: no special case needed
+        // the chain: warps 0..3 own slot pair `warp` of every lane.  Channels beyond C contribute fma(0, 0, acc) = acc
+        // and max(acc, 0) = acc: no special case needed
+        if (warp < 4) {
 #pragma unroll
-        for (int c = 0; c < RC; ++c) {
-            const float2 v = buf[c][warp][lane];
-            nn = __ffma2_rn(v, v, nn);
-            a0 = fmaxf(a0, fabsf(v.x));
-            a1 = fmaxf(a1, fabsf(v.y));
+            for (int c = 0; c < RC; ++c) {
+                const float2 v = buf[c][warp][lane];
+                nn = __ffma2_rn(v, v, nn);
+                a0 = fmaxf(a0, fabsf(v.x));
+                a1 = fmaxf(a1, fabsf(v.y));
+            }
         }
         __syncthreads();
     }
     if (VEC) Ring::template wait<0>();
+    if (warp >= 4) return;
     const float n0 = nn.x, n1 = nn.y;
     int p0 = 0, p1 = 0;
     bool ok0 = false, ok1 = false;
@@ -634,7 +640,7 @@ static wcc_status haar_fwd_dispatch(const void* x, int N, int C, int H, int W, f
     if (!coef && nrm2) {          // norms only: four warps per tile
         NormsExtra ex = {};
         ex.tiles = (int)warps;
-        haar_norms_kernel<T, L, VEC><<<(unsigned)warps, 128, 0, st>>>(static_cast<const T*>(x), N, C, H, W, nrm2, amaxpos, ex);
+        haar_norms_kernel<T, L, VEC><<<(unsigned)warps, NORMS_WARPS * 32, 0, st>>>(static_cast<const T*>(x), N, C, H, W, nrm2, amaxpos, ex);
         WCC_LAUNCH_CHECK();
         return WCC_OK;
     }
@@ -664,8 +670,8 @@ static wcc_status haar_norms_dispatch(const void* x, int N, int C, int H, int W,
     using TT = HaarTile<L>;
     const long long tiles = (long long)N * ceil_div(W, TT::TW) * (H / TT::TH);
     ex.tiles = (int)tiles;
-    const long long grid = tiles + (ex.Wt ? ceil_div(ex.Cout, 4) : 0);
-    haar_norms_kernel<T, L, VEC><<<(unsigned)grid, 128, 0, st>>>(static_cast<const T*>(x), N, C, H, W, nrm2, amaxpos, ex);
+    const long long grid = tiles + (ex.Wt ? ceil_div(ex.Cout, NORMS_WARPS) : 0);
+    haar_norms_kernel<T, L, VEC><<<(unsigned)grid, NORMS_WARPS * 32, 0, st>>>(static_cast<const T*>(x), N, C, H, W, nrm2, amaxpos, ex);
     WCC_LAUNCH_CHECK();
     return WCC_OK;
 }

@@ -605,8 +605,8 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
     const uint32_t k1 = (uint32_t)k - above;
     // round 2: next 11 bits of the keys that match
 #pragma unroll
-    for (int i = 0; i < CL_MAXKPT; ++i)
-        if (i < kpt) hist_add(sm.hist, (key[i] >> 10) & 0x7FFu, valid(i) && (key[i] >> 21) == b1);
+    for (int i = 0; i < CL_MAXKPT; ++i)     // plain atomics: these digits are mantissa bits, spread over the bins
+        if (valid(i) && (key[i] >> 21) == b1) atomicAdd(&sm.hist[(key[i] >> 10) & 0x7FFu], 1u);
     uint32_t b2;
     cluster_find_bin(cluster, sm, cs, crank, SEL_BINS, k1, b2, above);
     const uint32_t k2 = k1 - above;
@@ -616,7 +616,7 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
     __syncthreads();
 #pragma unroll
     for (int i = 0; i < CL_MAXKPT; ++i)
-        if (i < kpt) hist_add(sm.hist, key[i] & 0x3FFu, valid(i) && (key[i] >> 10) == prefix);
+        if (valid(i) && (key[i] >> 10) == prefix) atomicAdd(&sm.hist[key[i] & 0x3FFu], 1u);
     uint32_t b3;
     cluster_find_bin(cluster, sm, cs, crank, 1024, k2, b3, above);
     const uint32_t tkey = (prefix << 10) | b3, need_eq = k2 - above;
