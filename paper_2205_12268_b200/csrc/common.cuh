@@ -91,7 +91,8 @@ wcc_status launch_scatter_inv(const int32_t* acc, int ldc, bool acc_is_float, co
 size_t select_ws_bytes(int N, int P);
 wcc_status launch_select(const float* nrm2, int N, int P, int k, int32_t* idx, float* tau,
                          int32_t* rank, const float* amaxpos, bool want_amax,
-                         void* ws, size_t ws_bytes, cudaStream_t st, bool hist1_ready = false);
+                         void* ws, size_t ws_bytes, cudaStream_t st, bool hist1_ready = false,
+                         const uint32_t* fine = nullptr, uint32_t* thr = nullptr, bool want_rank = true);
 
 // Weight quantization (bits >= 2: int8 codes + per-row scale; bits == 0: bf16 copy), rows padded to kpad.
 wcc_status launch_weight_prep(const float* Wt, int Cout, int Cin, int kpad, int bits,

@@ -54,7 +54,7 @@ struct Ctl {
 template <typename T, int L, bool VEC, bool I8>
 __global__ void __launch_bounds__(128, 4)
 fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, const int32_t* __restrict__ rank,
-                   const float* __restrict__ amax_kept, float qmax, const float* __restrict__ scale_w,
+                   const float* __restrict__ nrm2, const uint32_t* __restrict__ thr, const float* __restrict__ amax_kept, float qmax, const float* __restrict__ scale_w,
                    int N, int Cin, int Cout, int H, int W, int k, int kpad, int npad, int nchunk, int tmem_cols, int a_ksteps,
                    T* __restrict__ y, uint8_t* __restrict__ xq_tap, int32_t* __restrict__ acc_tap, int* __restrict__ status)
 {
@@ -92,10 +92,17 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
                      ::"r"(tc::smem_u32(&ctl->tmem_base)), "r"((uint32_t)tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    // kept or dropped: from the rank map when the select wrote one (thr[n][2] != 0: partial ties, or a test wants
+    // the ranks), else by comparing the position's norm with the threshold key
+    const uint32_t tkey = thr[n * 4], use_rank = thr[n * 4 + 2];
     int rk[8];
 #pragma unroll
     for (int s = 0; s < 8; ++s) {
-        rk[s] = slot_ok<L>(lp, s) ? rank[(size_t)n * P + lp.pos[s]] : -1;
+        rk[s] = -1;
+        if (slot_ok<L>(lp, s)) {
+            if (use_rank) rk[s] = rank[(size_t)n * P + lp.pos[s]];
+            else rk[s] = (float_key(nrm2[(size_t)n * P + lp.pos[s]]) >= tkey) ? 0 : -1;
+        }
         if (warp == 0) srank[s * 32 + lane] = rk[s];
     }
     for (int i = threadIdx.x; i < npad * kchunks; i += 128) {
@@ -310,7 +317,8 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
 static inline size_t vmax(size_t a, size_t b) { return a > b ? a : b; }
 
 template <typename T, int L, bool VEC>
-static wcc_status fused_pass2_dispatch(const void* x, const void* Wq, const int32_t* rank, const float* amax_kept, int bits,
+static wcc_status fused_pass2_dispatch(const void* x, const void* Wq, const int32_t* rank, const float* nrm2,
+                                       const uint32_t* thr, const float* amax_kept, int bits,
                                        const float* scale_w, int N, int Cin, int Cout, int H, int W, int k, int kpad,
                                        void* y, void* xq_tap, int32_t* acc_tap, cudaStream_t st)
 {
@@ -336,7 +344,7 @@ static wcc_status fused_pass2_dispatch(const void* x, const void* Wq, const int3
     if (ctas > 0x7FFFFFFFLL) return WCC_ERR_SHAPE;
     auto launch = [&](auto kern) -> wcc_status {
         WCC_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-        kern<<<(unsigned)ctas, 128, smem, st>>>(static_cast<const T*>(x), static_cast<const uint8_t*>(Wq), rank, amax_kept, qmax,
+        kern<<<(unsigned)ctas, 128, smem, st>>>(static_cast<const T*>(x), static_cast<const uint8_t*>(Wq), rank, nrm2, thr, amax_kept, qmax,
                                                 scale_w, N, Cin, Cout, H, W, k, kpad, npad, nchunk, tmem_cols, a_ksteps,
                                                 static_cast<T*>(y), static_cast<uint8_t*>(xq_tap), acc_tap, status);
         WCC_LAUNCH_CHECK();
@@ -347,12 +355,13 @@ static wcc_status fused_pass2_dispatch(const void* x, const void* Wq, const int3
 }
 
 // Fused second pass.  xq_tap ([N*k][kpad] of int8 or bf16) and acc_tap (int32 [N*k][Cout]) may be NULL.
-wcc_status launch_fused_pass2(const void* x, const void* Wq, const int32_t* rank, const float* amax_kept, int bits,
+wcc_status launch_fused_pass2(const void* x, const void* Wq, const int32_t* rank, const float* nrm2, const uint32_t* thr,
+                              const float* amax_kept, int bits,
                               const float* scale_w, int N, int Cin, int Cout, int H, int W, int L, int k, int kpad,
                               wcc_dtype dt, void* y, void* xq_tap, int32_t* acc_tap, cudaStream_t st)
 {
     const bool vec = (W % 4) == 0;
-    WCC_DISPATCH_TLV(fused_pass2_dispatch, dt, L, vec, x, Wq, rank, amax_kept, bits, scale_w, N, Cin, Cout, H, W, k, kpad,
+    WCC_DISPATCH_TLV(fused_pass2_dispatch, dt, L, vec, x, Wq, rank, nrm2, thr, amax_kept, bits, scale_w, N, Cin, Cout, H, W, k, kpad,
                      y, xq_tap, acc_tap, st);
 }
 

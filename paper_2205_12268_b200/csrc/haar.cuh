@@ -435,6 +435,7 @@ struct PatchRing {
 struct NormsExtra {
     float* coef;          // fp32 [N][C][P] or NULL
     uint32_t* hist1;      // [N][3][2048] (round 1 first), zeroed by the caller, or NULL
+    uint32_t* fine;       // [N][65536]: histogram of the top 16 key bits, zeroed by the caller, or NULL
     const float* Wt;      // weights to prepare in the extra CTAs, or NULL
     void* Wq;
     float* scale_w;
@@ -547,6 +548,11 @@ haar_norms_kernel(const T* __restrict__ x, int N, int C, int H, int W,
         uint32_t* h = ex.hist1 + (size_t)n * 3 * 2048;
         hist_add(h, float_key(n0) >> 21, ok0);
         hist_add(h, float_key(n1) >> 21, ok1);
+    }
+    if (ex.fine) {                                     // 16-bit digits are spread out: plain atomics
+        uint32_t* f = ex.fine + (size_t)n * 65536;
+        if (ok0) atomicAdd(&f[float_key(n0) >> 16], 1u);
+        if (ok1) atomicAdd(&f[float_key(n1) >> 16], 1u);
     }
 }
 

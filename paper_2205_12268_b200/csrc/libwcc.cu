@@ -165,6 +165,7 @@ static wcc_status staged_impl(const void* x, const float* Wt, int N, int Cin, in
 // ---- fused path ----------------------------------------------------------------------------------
 struct FusedWs {
     float* nrm2; float* amaxpos; int32_t* rank; int32_t* idx; void* sel; size_t sel_bytes;
+    uint32_t* fine; uint32_t* thr; size_t fine_bytes;
     float* amax_kept; void* Wq; float* scale_w;
     int kpad, es;
     size_t total;
@@ -183,6 +184,10 @@ static FusedWs carve_fused_ws(void* ws, int N, int Cin, int Cout, int H, int W, 
     f.amaxpos = reinterpret_cast<float*>(take((size_t)N * P * 4));
     f.rank = reinterpret_cast<int32_t*>(take((size_t)N * P * 4));
     f.idx = reinterpret_cast<int32_t*>(take(M * 4));
+    f.thr = reinterpret_cast<uint32_t*>(take((size_t)N * 16));
+    // the 16-bit histogram sits right before the select scratch, whose zeroed part comes first: one memset clears both
+    f.fine_bytes = align_up((size_t)N * FINE_BINS * 4, 256);
+    f.fine = reinterpret_cast<uint32_t*>(take(f.fine_bytes));
     f.sel_bytes = select_ws_bytes(N, (int)P);
     f.sel = take(f.sel_bytes);
     f.amax_kept = b ? carve_select_ws(f.sel, N, (int)P).amax : nullptr;
@@ -211,22 +216,24 @@ static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, i
     // coefficient map is written only when a test asks for it).  The same launch fills round 1 of the select's
     // histogram and quantizes the weights in a few extra CTAs.
     const SelectWs sw = carve_select_ws(f.sel, N, P);
-    WCC_CUDA_TRY(cudaMemsetAsync(sw.hist, 0, sw.zero_bytes, st));          // histograms, max |kept|, barrier counters
+    WCC_CUDA_TRY(cudaMemsetAsync(f.fine, 0, f.fine_bytes + sw.zero_bytes, st));   // histograms, max |kept|, barrier counters
     NormsExtra ex = {};
     ex.coef = taps ? taps->coef : nullptr;
     ex.hist1 = sw.hist;
+    ex.fine = f.fine;
     ex.Wt = Wt; ex.Wq = f.Wq; ex.scale_w = f.scale_w; ex.Cout = Cout; ex.kpad = f.kpad; ex.bits = bits;
     s = launch_haar_norms(x, N, Cin, H, W, L, dt, f.nrm2, f.amaxpos, ex, st);
     if (s != WCC_OK) return s;
     if ((s = profile_mark(1, st)) != WCC_OK) return s;
     // joint shrinkage: index list, rank map, max |kept|
-    s = launch_select(f.nrm2, N, P, k, f.idx, nullptr, f.rank, f.amaxpos, true, f.sel, f.sel_bytes, st, true);
+    s = launch_select(f.nrm2, N, P, k, f.idx, nullptr, f.rank, f.amaxpos, true, f.sel, f.sel_bytes, st, true,
+                      f.fine, f.thr, taps != nullptr);
     if (s != WCC_OK) return s;
     if ((s = profile_mark(2, st)) != WCC_OK) return s;
     if ((s = profile_mark(3, st)) != WCC_OK) return s;
     // second pass over x: transform, mask + quantize, tensor-core contraction, dequantize, inverse, store
     void* xq_tap = taps ? (bits >= 2 ? static_cast<void*>(taps->Xq) : taps->Xb) : nullptr;
-    s = launch_fused_pass2(x, f.Wq, f.rank, f.amax_kept, bits, f.scale_w, N, Cin, Cout, H, W, L, k, f.kpad, dt, y,
+    s = launch_fused_pass2(x, f.Wq, f.rank, f.nrm2, f.thr, f.amax_kept, bits, f.scale_w, N, Cin, Cout, H, W, L, k, f.kpad, dt, y,
                            xq_tap, taps ? taps->acc : nullptr, st);
     if (s != WCC_OK) return s;
     for (int i = 4; i <= WCC_NUM_STAGES; ++i)

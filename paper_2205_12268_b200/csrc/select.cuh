@@ -443,6 +443,9 @@ select_coop_kernel(const float* __restrict__ nrm2, int P, int k, uint32_t* __res
 constexpr int CL_THREADS = 1024;
 constexpr int CL_MAXKPT = 16;
 constexpr int CL_MAXCS = 8;
+constexpr int CL_CAND_CTA = 512;     // candidate slots per CTA
+constexpr int CL_CAND_MAX = 1024;    // most candidates ranked by brute force; beyond that: histogram rounds
+constexpr int FINE_BINS = 65536;     // histogram of the top 16 key bits, filled by the producer of the norms
 
 struct ClusterSmem {
     uint32_t hist[SEL_BINS];
@@ -450,9 +453,13 @@ struct ClusterSmem {
     uint32_t warp_sums[CL_THREADS / 32 + 1];
     uint32_t slice_total;
     uint32_t cnt[2];                // keys above / equal to the threshold in this CTA
-    uint32_t res[2];
+    uint32_t res[3];                // found bin, keys above it, keys in it
     uint32_t tot[CL_MAXCS];
     uint32_t amax;
+    uint32_t ncand;                 // candidates of this CTA (keys whose top 16 bits hold the threshold)
+    uint32_t cand[CL_CAND_CTA];
+    uint32_t all[CL_CAND_MAX];      // candidates of the whole cluster
+    uint32_t thr[3];                // threshold key, ties to keep, ties in total
 };
 
 // exclusive scan over the threads of the block (256, 512 or 1024); every thread also gets the total
@@ -529,7 +536,7 @@ __device__ __forceinline__ void cluster_find_bin(cg::cluster_group& cluster, Clu
         uint32_t a = before;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            if (a < kin && kin <= a + c[i]) { sm.res[0] = (uint32_t)(target * B + top - i); sm.res[1] = above_slices + a; }
+            if (a < kin && kin <= a + c[i]) { sm.res[0] = (uint32_t)(target * B + top - i); sm.res[1] = above_slices + a; sm.res[2] = c[i]; }
             a += c[i];
         }
     }
@@ -559,7 +566,7 @@ __device__ __forceinline__ void block_find_bin_2048(const uint32_t* __restrict__
         uint32_t a = before;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            if (a < krem && krem <= a + c[i]) { sm.res[0] = (uint32_t)(top - i); sm.res[1] = a; }
+            if (a < krem && krem <= a + c[i]) { sm.res[0] = (uint32_t)(top - i); sm.res[1] = a; sm.res[2] = c[i]; }
             a += c[i];
         }
     }
@@ -569,10 +576,17 @@ __device__ __forceinline__ void block_find_bin_2048(const uint32_t* __restrict__
     __syncthreads();
 }
 
+// hist1 ([N][3][2048], round 1 first) and fine ([N][65536]) are optional histograms of the top 11 and top 16 key bits
+// that the producer of the norms filled; with both, the threshold is usually found without any histogram round:
+// the 16-bit bin that holds the k-th key contains few keys, which the cluster gathers and ranks directly.
+// idx and rank are written only when asked for (want_rank) or when the threshold's ties are kept only in part
+// (then the order of positions matters); otherwise consumers compare keys with thr[n] = {threshold key, ties
+// kept, use_rank flag}.
 __global__ void __launch_bounds__(CL_THREADS, 1)
 select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int32_t* __restrict__ idx, float* __restrict__ tau,
                       int32_t* __restrict__ rank, const float* __restrict__ amaxpos, float* __restrict__ amax_kept,
-                      const uint32_t* __restrict__ hist1)
+                      const uint32_t* __restrict__ hist1, const uint32_t* __restrict__ fine, uint32_t* __restrict__ thr,
+                      int want_rank)
 {
     __shared__ ClusterSmem sm;
     cg::cluster_group cluster = cg::this_cluster();
@@ -580,6 +594,7 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
     const int n = blockIdx.y;
     const float* v = nrm2 + (size_t)n * P;
     const int base = (crank * (int)blockDim.x + (int)threadIdx.x) * kpt;  // kpt consecutive keys per thread
+    const int lane = threadIdx.x & 31;
 
     uint32_t key[CL_MAXKPT];
 #pragma unroll
@@ -587,89 +602,179 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
     auto valid = [&](int i) { return i < kpt && base + i < P; };
 
     for (int i = threadIdx.x; i < SEL_BINS; i += blockDim.x) sm.hist[i] = 0u;
-    if (threadIdx.x == 0) sm.amax = 0u;
+    if (threadIdx.x == 0) { sm.amax = 0u; sm.ncand = 0u; }
     __syncthreads();
-    // round 1: top 11 bits.  When the producer of the norms already histogrammed them (hist1: [N][3][2048], round 1
-    // first), only the bin search is left.
-    uint32_t b1, above;
-    if (hist1) {
+
+    uint32_t tkey = 0, need_eq = 0, total_eq = 0;
+    bool found = false;
+    if (hist1 && fine) {
+        // the 11-bit bin, then the 16-bit bin inside it (32 fine bins, one per lane of warp 0, top bin in lane 0)
+        uint32_t b1, above;
         block_find_bin_2048(hist1 + (size_t)n * 3 * SEL_BINS, (uint32_t)k, sm, b1, above);
-    } else {
+        const uint32_t k1 = (uint32_t)k - above;
+        if (threadIdx.x < 32) {
+            const uint32_t f = __ldcg(&fine[(size_t)n * FINE_BINS + (b1 << 5) + 31u - (uint32_t)lane]);
+            uint32_t inc = f;
 #pragma unroll
-        for (int i = 0; i < CL_MAXKPT; ++i)
-            if (i < kpt) hist_add(sm.hist, key[i] >> 21, valid(i));
-        cluster_find_bin(cluster, sm, cs, crank, SEL_BINS, (uint32_t)k, b1, above);
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+                if (lane >= d) inc += t;
+            }
+            const uint32_t before = inc - f;
+            if (before < k1 && k1 <= inc) { sm.res[0] = (b1 << 5) + 31u - (uint32_t)lane; sm.res[1] = before; sm.res[2] = f; }
+        }
+        __syncthreads();
+        const uint32_t prefix16 = sm.res[0], k16 = k1 - sm.res[1];
+        __syncthreads();
+        // collect this CTA's candidates
+#pragma unroll
+        for (int i = 0; i < CL_MAXKPT; ++i) {
+            if (i >= kpt) break;
+            const bool c = valid(i) && (key[i] >> 16) == prefix16;
+            const unsigned m = __ballot_sync(0xFFFFFFFFu, c);
+            if (m) {
+                uint32_t off = 0;
+                if (lane == 0) off = atomicAdd(&sm.ncand, (uint32_t)__popc(m));
+                off = __shfl_sync(0xFFFFFFFFu, off, 0);
+                const uint32_t slot = off + (uint32_t)__popc(m & ((1u << lane) - 1u));
+                if (c && slot < CL_CAND_CTA) sm.cand[slot] = key[i];
+            }
+        }
+        cluster.sync();
+        if (threadIdx.x < cs) sm.tot[threadIdx.x] = *cluster.map_shared_rank(&sm.ncand, threadIdx.x);
+        __syncthreads();
+        uint32_t M = 0;
+        bool overflow = false;
+        for (int r = 0; r < cs; ++r) { overflow = overflow || sm.tot[r] > CL_CAND_CTA; M += sm.tot[r]; }
+        overflow = overflow || M > CL_CAND_MAX;
+        if (!overflow) {
+            uint32_t off = 0;
+            for (int r = 0; r < cs; ++r) {
+                const uint32_t* rc = cluster.map_shared_rank(sm.cand, r);
+                for (uint32_t i = threadIdx.x; i < sm.tot[r]; i += blockDim.x) sm.all[off + i] = rc[i];
+                off += sm.tot[r];
+            }
+            __syncthreads();
+            // the k16-th largest candidate, by counting (M is small)
+            for (uint32_t i = threadIdx.x; i < M; i += blockDim.x) {
+                const uint32_t ci = sm.all[i];
+                uint32_t g = 0, e = 0;
+                for (uint32_t j = 0; j < M; ++j) { const uint32_t cj = sm.all[j]; g += cj > ci; e += cj == ci; }
+                if (g < k16 && k16 <= g + e) { sm.thr[0] = ci; sm.thr[1] = k16 - g; sm.thr[2] = e; }   // equal keys write equal values
+            }
+            __syncthreads();
+            tkey = sm.thr[0]; need_eq = sm.thr[1]; total_eq = sm.thr[2];
+            found = true;
+        }
+    }
+    if (!found) {
+        // round 1: top 11 bits (only the bin search when the producer of the norms histogrammed them)
+        uint32_t b1, above;
+        if (hist1) {
+            block_find_bin_2048(hist1 + (size_t)n * 3 * SEL_BINS, (uint32_t)k, sm, b1, above);
+        } else {
+#pragma unroll
+            for (int i = 0; i < CL_MAXKPT; ++i)
+                if (i < kpt) hist_add(sm.hist, key[i] >> 21, valid(i));
+            cluster_find_bin(cluster, sm, cs, crank, SEL_BINS, (uint32_t)k, b1, above);
+            for (int i = threadIdx.x; i < SEL_BINS; i += blockDim.x) sm.hist[i] = 0u;
+            __syncthreads();
+        }
+        const uint32_t k1 = (uint32_t)k - above;
+        // round 2: next 11 bits of the keys that match
+#pragma unroll
+        for (int i = 0; i < CL_MAXKPT; ++i)     // plain atomics: these digits are mantissa bits, spread over the bins
+            if (valid(i) && (key[i] >> 21) == b1) atomicAdd(&sm.hist[(key[i] >> 10) & 0x7FFu], 1u);
+        uint32_t b2;
+        cluster_find_bin(cluster, sm, cs, crank, SEL_BINS, k1, b2, above);
+        const uint32_t k2 = k1 - above;
+        const uint32_t prefix = (b1 << 11) | b2;
+        // round 3: last 10 bits
         for (int i = threadIdx.x; i < SEL_BINS; i += blockDim.x) sm.hist[i] = 0u;
         __syncthreads();
+#pragma unroll
+        for (int i = 0; i < CL_MAXKPT; ++i)
+            if (valid(i) && (key[i] >> 10) == prefix) atomicAdd(&sm.hist[key[i] & 0x3FFu], 1u);
+        uint32_t b3;
+        cluster_find_bin(cluster, sm, cs, crank, 1024, k2, b3, above);
+        tkey = (prefix << 10) | b3;
+        need_eq = k2 - above;
+        total_eq = sm.res[2];
     }
-    const uint32_t k1 = (uint32_t)k - above;
-    // round 2: next 11 bits of the keys that match
-#pragma unroll
-    for (int i = 0; i < CL_MAXKPT; ++i)     // plain atomics: these digits are mantissa bits, spread over the bins
-        if (valid(i) && (key[i] >> 21) == b1) atomicAdd(&sm.hist[(key[i] >> 10) & 0x7FFu], 1u);
-    uint32_t b2;
-    cluster_find_bin(cluster, sm, cs, crank, SEL_BINS, k1, b2, above);
-    const uint32_t k2 = k1 - above;
-    const uint32_t prefix = (b1 << 11) | b2;
-    // round 3: last 10 bits
-    for (int i = threadIdx.x; i < SEL_BINS; i += blockDim.x) sm.hist[i] = 0u;
-    __syncthreads();
-#pragma unroll
-    for (int i = 0; i < CL_MAXKPT; ++i)
-        if (valid(i) && (key[i] >> 10) == prefix) atomicAdd(&sm.hist[key[i] & 0x3FFu], 1u);
-    uint32_t b3;
-    cluster_find_bin(cluster, sm, cs, crank, 1024, k2, b3, above);
-    const uint32_t tkey = (prefix << 10) | b3, need_eq = k2 - above;
     if (tau && crank == 0 && threadIdx.x == 0) tau[n] = key_float(tkey);
 
-    // ordered compaction
-    uint32_t gt = 0, eq = 0;
-#pragma unroll
-    for (int i = 0; i < CL_MAXKPT; ++i) {
-        if (!valid(i)) continue;
-        gt += key[i] > tkey;
-        eq += key[i] == tkey;
-    }
-    uint32_t tot_gt, tot_eq;
-    uint32_t gt_before = block_scan_1024(gt, sm.warp_sums, &tot_gt);
-    uint32_t eq_before = block_scan_1024(eq, sm.warp_sums, &tot_eq);
-    if (threadIdx.x == 0) { sm.cnt[0] = tot_gt; sm.cnt[1] = tot_eq; }
-    cluster.sync();
-    for (int r = 0; r < crank; ++r) {
-        const uint32_t* c = cluster.map_shared_rank(sm.cnt, r);
-        gt_before += c[0];
-        eq_before += c[1];
-    }
+    const bool ordered = want_rank || need_eq < total_eq;       // uniform over the cluster
     float amax = 0.0f;
+    if (!ordered) {
+        // every key >= threshold is kept; nobody needs the order
+        if (amaxpos) {
 #pragma unroll
-    for (int i = 0; i < CL_MAXKPT; ++i) {
-        if (!valid(i)) continue;
-        const bool is_gt = key[i] > tkey, is_eq = key[i] == tkey;
-        const bool keep = is_gt || (is_eq && eq_before < need_eq);
-        const uint32_t pos = gt_before + min(eq_before, need_eq);
-        if (keep) {
-            idx[(size_t)n * k + pos] = base + i;
-            if (amaxpos) amax = fmaxf(amax, amaxpos[(size_t)n * P + base + i]);
+            for (int i = 0; i < CL_MAXKPT; ++i)
+                if (valid(i) && key[i] >= tkey) amax = fmaxf(amax, amaxpos[(size_t)n * P + base + i]);
         }
-        if (rank) rank[(size_t)n * P + base + i] = keep ? (int32_t)pos : -1;
-        gt_before += is_gt;
-        eq_before += is_eq;
+    } else {
+        // ordered compaction: ascending idx, rank map, ties to the lowest positions
+        uint32_t gt = 0, eq = 0;
+#pragma unroll
+        for (int i = 0; i < CL_MAXKPT; ++i) {
+            if (!valid(i)) continue;
+            gt += key[i] > tkey;
+            eq += key[i] == tkey;
+        }
+        uint32_t tot_gt, tot_eq;
+        uint32_t gt_before = block_scan_1024(gt, sm.warp_sums, &tot_gt);
+        uint32_t eq_before = block_scan_1024(eq, sm.warp_sums, &tot_eq);
+        if (threadIdx.x == 0) { sm.cnt[0] = tot_gt; sm.cnt[1] = tot_eq; }
+        cluster.sync();
+        for (int r = 0; r < crank; ++r) {
+            const uint32_t* c = cluster.map_shared_rank(sm.cnt, r);
+            gt_before += c[0];
+            eq_before += c[1];
+        }
+#pragma unroll
+        for (int i = 0; i < CL_MAXKPT; ++i) {
+            if (!valid(i)) continue;
+            const bool is_gt = key[i] > tkey, is_eq = key[i] == tkey;
+            const bool keep = is_gt || (is_eq && eq_before < need_eq);
+            const uint32_t pos = gt_before + min(eq_before, need_eq);
+            if (keep) {
+                if (idx) idx[(size_t)n * k + pos] = base + i;
+                if (amaxpos) amax = fmaxf(amax, amaxpos[(size_t)n * P + base + i]);
+            }
+            if (rank) rank[(size_t)n * P + base + i] = keep ? (int32_t)pos : -1;
+            gt_before += is_gt;
+            eq_before += is_eq;
+        }
+    }
+    if (thr && crank == 0 && threadIdx.x == 0) {
+        thr[n * 4 + 0] = tkey;
+        thr[n * 4 + 1] = need_eq;
+        thr[n * 4 + 2] = ordered ? 1u : 0u;
     }
     if (amax_kept) {
 #pragma unroll
         for (int d = 16; d > 0; d >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, d));
-        if ((threadIdx.x & 31) == 0) atomicMax(&sm.amax, __float_as_uint(amax));
+        if (lane == 0) atomicMax(&sm.amax, __float_as_uint(amax));
         __syncthreads();
         if (threadIdx.x == 0 && sm.amax) atomicMax(reinterpret_cast<uint32_t*>(amax_kept), sm.amax);
     }
     cluster.sync();                                  // nobody leaves while a neighbour may still read its shared memory
 }
 
+__global__ void thr_use_rank_kernel(uint32_t* thr, int N)
+{
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    if (n < N) { thr[n * 4 + 0] = 0u; thr[n * 4 + 1] = 0u; thr[n * 4 + 2] = 1u; }
+}
+
 // hist1_ready: the caller has already cleared the zero region of the workspace (carve_select_ws(...).hist,
 // zero_bytes) and filled round 1 of the histogram (top 11 key bits of every norm) before this call.
+// fine / thr: see select_cluster_kernel; want_rank: idx (if non-NULL) and rank must be written even when the
+// threshold alone would do.  Without thr the rank map and idx are always written.
 wcc_status launch_select(const float* nrm2, int N, int P, int k, int32_t* idx, float* tau,
                          int32_t* rank, const float* amaxpos, bool want_amax,
-                         void* ws, size_t ws_bytes, cudaStream_t st, bool hist1_ready)
+                         void* ws, size_t ws_bytes, cudaStream_t st, bool hist1_ready,
+                         const uint32_t* fine, uint32_t* thr, bool want_rank)
 {
     if (ws_bytes < select_ws_bytes(N, P)) return WCC_ERR_WORKSPACE;
     const SelectWs s = carve_select_ws(ws, N, P);
@@ -697,11 +802,16 @@ wcc_status launch_select(const float* nrm2, int N, int P, int k, int32_t* idx, f
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        WCC_CUDA_TRY(cudaLaunchKernelEx(&cfg, select_cluster_kernel, nrm2, P, k, kpt, idx, tau, rank, amaxpos, amax_kept, hist1));
+        WCC_CUDA_TRY(cudaLaunchKernelEx(&cfg, select_cluster_kernel, nrm2, P, k, kpt, idx, tau, rank, amaxpos, amax_kept, hist1,
+                                        hist1_ready ? fine : (const uint32_t*)nullptr, thr, (want_rank || !thr) ? 1 : 0));
         WCC_LAUNCH_CHECK();
         return WCC_OK;
     }
-    // (a round-1 histogram supplied by the caller is not used by these paths: they start from a clean slate)
+    if (thr) {                                        // these paths always write idx and the rank map
+        thr_use_rank_kernel<<<ceil_div(N, 128), 128, 0, st>>>(thr, N);
+        ++g_launches;
+    }
+    // (histograms supplied by the caller are not used by these paths: they start from a clean slate)
     WCC_CUDA_TRY(cudaMemsetAsync(s.hist, 0, s.zero_bytes, st));
     const dim3 grid(s.chunks, N);
 
