@@ -57,8 +57,8 @@ def stage_bytes(w, stage: str) -> float:
     NP, Nk = w.N * w.P, w.N * w.k
     es = 2 if w.bits == 0 else 1
     return {
-        "haar_norms": NP * w.Cin * s + 8 * NP,                                  # x once; norms and per-position max out
-        "fused_pass2": NP * w.Cin * s + 4 * NP + s * NP * w.Cout,               # x again, rank map, y once
+        "haar_norms": NP * w.Cin * s + 8 * NP + 5 * w.Cout * w.Cin,             # x once; norms and per-position max out; weights
+        "fused_pass2": NP * w.Cin * s + 4 * NP + s * NP * w.Cout,               # x again, norms (or rank map), y once
         "haar_fwd_norms": NP * w.Cin * (s + 4) + 4 * NP,
         "select_topk": 4 * NP + 4 * Nk,
         "weight_quant": w.Cout * w.Cin * (4 + es),

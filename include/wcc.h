@@ -122,11 +122,12 @@ wcc_status wcc_select_topk_static(const float* nrm2, int N, int P, int k, int32_
  *            0: no quantization; columns and weights rounded to bf16, fp32 accumulation.
  *   y   out: [N][Cout][H][Wd] of dt; must not overlap x
  *   ws     : scratch of at least wcc_workspace_bytes(...) bytes, 256-byte aligned; contents undefined afterwards
- * Execution: two passes over x around the selection.  Pass 1 transforms x in registers and keeps only the channel
- * norms and the per-position max |coefficient|; the selection yields the index list, the rank of every position in
- * it and max|kept|; pass 2 transforms x again, zeroes the dropped positions, quantizes into shared memory, runs the
- * contraction on tensor cores, dequantizes, applies the inverse transform and stores y.  The results are those of
- * the step-by-step definition above (same integers, same fp32 operation order).
+ * Execution: three launches, two passes over x around the selection.  Pass 1 transforms x in registers and keeps
+ * only the channel norms, the per-position max |coefficient| and two histograms of the norms' leading key bits (it
+ * also quantizes the weights); the selection finds the threshold norm, max|kept| and, only if ties at the threshold
+ * are kept in part, the rank of every position; pass 2 transforms x again, zeroes the dropped positions, quantizes
+ * into shared memory, runs the contraction on tensor cores, dequantizes, applies the inverse transform and stores y.
+ * The results are those of the step-by-step definition above (same integers, same fp32 operation order).
  */
 wcc_status wcc_forward(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int Wd,
                        int levels, int k, int bits, void* y, wcc_dtype dt,
@@ -184,8 +185,8 @@ const char* wcc_status_str(wcc_status s);
  * stream around each stage; wcc_profile_read waits for the last recorded call and writes, to the HOST array ms, the
  * milliseconds of, for wcc_forward_staged: 0 Haar transform + norms, 1 top-k select + compaction, 2 weight
  * quantization, 3 gather + quantize, 4 tensor-core contraction, 5 dequantize + scatter + inverse Haar; for wcc_forward:
- * 0 transform + norms (pass 1), 1 select, 2 weight quantization, 3 fused pass 2, 4 and 5 zero.  Off by default; not
- * thread-safe.
+ * 0 pass 1 (transform + norms, select histograms, weight quantization), 1 select, 2 fused pass 2, 3 to 5 zero.
+ * Off by default; not thread-safe.
  */
 #define WCC_NUM_STAGES 6
 wcc_status wcc_profile_enable(int on);

@@ -786,7 +786,8 @@ wcc_status launch_select(const float* nrm2, int N, int P, int k, int32_t* idx, f
         int cs = 1;
         while (cs < CL_MAXCS && cs * 512 < P) cs <<= 1;
         int threads = 256;
-        while (threads < CL_THREADS && (long long)cs * threads * CL_MAXKPT < P) threads <<= 1;
+        const int kpt_goal = hist1_ready ? 4 : CL_MAXKPT;               // few keys per thread when no scans are needed
+        while (threads < CL_THREADS && (long long)cs * threads * kpt_goal < P) threads <<= 1;
         const int kpt = ceil_div(P, cs * threads);
         if (amax_kept && !hist1_ready) WCC_CUDA_TRY(cudaMemsetAsync(amax_kept, 0, sizeof(float), st));
         const uint32_t* hist1 = hist1_ready ? s.hist : nullptr;
