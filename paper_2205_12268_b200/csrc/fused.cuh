@@ -92,6 +92,7 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
                      ::"r"(tc::smem_u32(&ctl->tmem_base)), "r"((uint32_t)tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    grid_dependency_wait();                            // the select (and with it the first pass) is complete from here on
     // kept or dropped: from the rank map when the select wrote one (thr[n][2] != 0: partial ties, or a test wants
     // the ranks), else by comparing the position's norm with the threshold key
     const uint32_t tkey = thr[n * 4], use_rank = thr[n * 4 + 2];
@@ -162,7 +163,8 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
             if (!ok) break;
             tc::fence_after();
         }
-        const int my_units = (u1 - u0 - warp + 3) / 4;
+        const int ur = min(u1, max(u0, (Cin + 7) / 8));         // units from ur on hold only zero padding
+        const int my_units = max(0, (ur - u0 - warp + 3) / 4);
         const int nq = my_units * SUBS;                // ring stages this warp will consume in this half
         auto chan0 = [&](int q) { return (u0 + warp + 4 * (q / SUBS)) * 8 + (q % SUBS) * LU; };
         if (VEC) {
@@ -231,6 +233,21 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
                     uint8_t* g = xq_tap + ((size_t)n * k + rk[s]) * krow + (size_t)u * UNIT_BYTES;
                     if (I8) *reinterpret_cast<uint2*>(g) = make_uint2(packed[s][0], packed[s][1]);
                     else *reinterpret_cast<uint4*>(g) = make_uint4(packed[s][0], packed[s][1], packed[s][2], packed[s][3]);
+                }
+            }
+        }
+        for (int u = ur + warp; u < u1; u += 4) {          // padding of K up to a multiple of 32 bytes: zeros
+            const int j = ((u - u0) * UNIT_BYTES) >> 4;
+            const int off = (u * UNIT_BYTES) & 15;
+#pragma unroll
+            for (int s = 0; s < 8; ++s) {
+                uint8_t* dst = sA + ((size_t)j * ROWS + s * 32 + lane) * 16 + off;
+                if (I8) *reinterpret_cast<uint2*>(dst) = make_uint2(0u, 0u);
+                else *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
+                if (xq_tap && rk[s] >= 0) {
+                    uint8_t* g = xq_tap + ((size_t)n * k + rk[s]) * krow + (size_t)u * UNIT_BYTES;
+                    if (I8) *reinterpret_cast<uint2*>(g) = make_uint2(0u, 0u);
+                    else *reinterpret_cast<uint4*>(g) = make_uint4(0u, 0u, 0u, 0u);
                 }
             }
         }
@@ -344,9 +361,19 @@ static wcc_status fused_pass2_dispatch(const void* x, const void* Wq, const int3
     if (ctas > 0x7FFFFFFFLL) return WCC_ERR_SHAPE;
     auto launch = [&](auto kern) -> wcc_status {
         WCC_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-        kern<<<(unsigned)ctas, 128, smem, st>>>(static_cast<const T*>(x), static_cast<const uint8_t*>(Wq), rank, nrm2, thr, amax_kept, qmax,
-                                                scale_w, N, Cin, Cout, H, W, k, kpad, npad, nchunk, tmem_cols, a_ksteps,
-                                                static_cast<T*>(y), static_cast<uint8_t*>(xq_tap), acc_tap, status);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)ctas);
+        cfg.blockDim = dim3(128);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];                       // may be scheduled while the select still runs
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = use_pdl() ? 1 : 0;
+        WCC_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, static_cast<const T*>(x), static_cast<const uint8_t*>(Wq), rank, nrm2, thr,
+                                        amax_kept, qmax, scale_w, N, Cin, Cout, H, W, k, kpad, npad, nchunk, tmem_cols, a_ksteps,
+                                        static_cast<T*>(y), static_cast<uint8_t*>(xq_tap), acc_tap, status));
         WCC_LAUNCH_CHECK();
         return WCC_OK;
     };
