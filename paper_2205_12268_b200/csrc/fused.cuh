@@ -27,7 +27,7 @@ namespace wcc {
 namespace fz {
 
 constexpr int ROWS = 256;            // positions per CTA
-constexpr int SUB = 8;               // output channels per transpose round
+constexpr int SUB = 16;              // output channels per transpose round
 constexpr int RING2 = 3;             // cp.async stages per warp in phase 1
 constexpr float MAGIC = 12582912.0f; // 1.5 * 2^23: adding it rounds to the nearest integer, ties to even
 
@@ -275,10 +275,13 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
         tc::fence_after();
 
         for (int s0 = 0; s0 < cur; s0 += SUB) {
-            uint32_t r0[8], r1[8];
+            uint32_t r0[SUB], r1[SUB];
             const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)s0;
-            tmem_ld8_nowait(taddr, r0);                              // slot `warp`
-            tmem_ld8_nowait(taddr + (uint32_t)nchunk, r1);           // slot `warp + 4`
+#pragma unroll
+            for (int q8 = 0; q8 < SUB / 8; ++q8) {
+                tmem_ld8_nowait(taddr + 8 * q8, *reinterpret_cast<uint32_t(*)[8]>(&r0[8 * q8]));                      // slot `warp`
+                tmem_ld8_nowait(taddr + (uint32_t)nchunk + 8 * q8, *reinterpret_cast<uint32_t(*)[8]>(&r1[8 * q8]));   // slot `warp + 4`
+            }
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
             const int rka = srank[warp * 32 + lane], rkb = srank[(warp + 4) * 32 + lane];
 #pragma unroll
