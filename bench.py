@@ -27,11 +27,15 @@ if ROOT not in sys.path:
 METRIC = "WCC layer output Gpix/s"
 UNIT = "Gpix/s"
 FLUSH_BYTES = 256 << 20          # > 126 MB of L2
-STAGE_FILES = ("haar.cuh", "select.cuh", "gather.cuh", "contract.cuh", "libwcc.cu", "common.cuh")
+STAGE_FILES = ("haar.cuh", "select.cuh", "gather.cuh", "contract.cuh", "fused.cuh", "libwcc.cu", "common.cuh")
 
 # DRAM bytes per launch of the dominant kernel from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum),
 # keyed by (workload, stage); valid only while the kernel sources still hash to `src`.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    # captured with N=16 images of C2 (x = 151 MB > L2) and divided by 4: every stage is per image
+    ("C2", "fused_pass2"): {"bytes": (153169920 + 15681280) / 4, "src": "ca85d59a7c0d"},
+    ("C2", "haar_norms"): {"bytes": (151243776 + 6776576) / 4, "src": "ca85d59a7c0d"},
+}
 
 
 def _source_hash() -> str:
