@@ -102,6 +102,25 @@ def test_layer_small(wcc, cfg, staged):
     _run_and_compare(wcc, w, staged=staged)
 
 
+@pytest.mark.parametrize("staged", [False, True], ids=["fused", "staged"])
+def test_layer_image_larger_than_one_cluster(wcc, staged):
+    """More positions per image (512 x 512) than the cluster select holds in registers: the cooperative select runs and
+    the fused second pass takes its keep / drop decisions from the rank map."""
+    w = inputs.custom("large", 9, 1, 4, 6, 512, 512, "f32", 3, 0.1, 8, n_sin=6, fmax=6.0)
+    _run_and_compare(wcc, w, staged=staged)
+
+
+def test_layer_partial_ties_at_the_threshold(wcc):
+    """Many positions share the k-th norm exactly and only some of them are kept (lowest positions first): the select
+    must fall back to the ordered compaction and the second pass to the rank map."""
+    w = inputs.custom("ties", 2, 2, 3, 5, 32, 64, "f32", 2, 0.5, 8, n_sin=3, fmax=2.0)
+    blk = w.x[:, :, :4, :4].copy()                           # one 4x4 block (a whole level-2 unit) tiled over the map
+    w.x[:] = np.tile(blk, (1, 1, 8, 16))
+    for k in (1, 100, 777, 1024, 2047):
+        w.k = k
+        _run_and_compare(wcc, w)
+
+
 def test_layer_k_equals_one_and_all(wcc):
     for k in (1, 16 * 16):
         w = inputs.custom("edge", 5, 2, 5, 7, 16, 16, "f32", 2, 0.5, 8, k=k)
