@@ -442,7 +442,7 @@ select_coop_kernel(const float* __restrict__ nrm2, int P, int k, uint32_t* __res
 // round trips, no spinning, no scratch memory.
 constexpr int CL_THREADS = 1024;
 constexpr int CL_MAXKPT = 16;
-constexpr int CL_MAXCS = 8;
+constexpr int CL_MAXCS = 16;          // 8 is the portable cluster size; 16 needs the non-portable opt-in
 constexpr int CL_CAND_CTA = 512;     // candidate slots per CTA
 constexpr int CL_CAND_MAX = 1024;    // most candidates ranked by brute force; beyond that: histogram rounds
 constexpr int FINE_BINS = 65536;     // histogram of the top 16 key bits, filled by the producer of the norms
@@ -581,7 +581,7 @@ __device__ __forceinline__ void block_find_bin_2048(const uint32_t* __restrict__
 // the 16-bit bin that holds the k-th key contains few keys, which the cluster gathers and ranks directly.
 // idx and rank are written only when asked for (want_rank) or when the threshold's ties are kept only in part
 // (then the order of positions matters); otherwise consumers compare keys with thr[n] = {threshold key, ties
-// kept, use_rank flag}.
+// kept, use_rank flag, number of candidate keys that were ranked (diagnostic)}.
 __global__ void __launch_bounds__(CL_THREADS, 1)
 select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int32_t* __restrict__ idx, float* __restrict__ tau,
                       int32_t* __restrict__ rank, const float* __restrict__ amaxpos, float* __restrict__ amax_kept,
@@ -607,7 +607,7 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
     if (threadIdx.x == 0) { sm.amax = 0u; sm.ncand = 0u; }
     __syncthreads();
 
-    uint32_t tkey = 0, need_eq = 0, total_eq = 0;
+    uint32_t tkey = 0, need_eq = 0, total_eq = 0, ranked = 0;    // ranked: candidates counted through (diagnostic)
     bool found = false;
     if (hist1 && fine) {
         // the 11-bit bin, then the 16-bit bin inside it (32 fine bins, one per lane of warp 0, top bin in lane 0)
@@ -666,6 +666,7 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
             }
             __syncthreads();
             tkey = sm.thr[0]; need_eq = sm.thr[1]; total_eq = sm.thr[2];
+            ranked = M;
             found = true;
         }
     }
@@ -752,6 +753,7 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
         thr[n * 4 + 0] = tkey;
         thr[n * 4 + 1] = need_eq;
         thr[n * 4 + 2] = ordered ? 1u : 0u;
+        thr[n * 4 + 3] = ranked;
     }
     if (amax_kept) {
 #pragma unroll
@@ -782,11 +784,32 @@ wcc_status launch_select(const float* nrm2, int N, int P, int k, int32_t* idx, f
     const SelectWs s = carve_select_ws(ws, N, P);
     float* amax_kept = want_amax ? s.amax : nullptr;
     // one cluster per image while its keys fit in the registers of 8 x 1024 threads
-    if (P <= CL_MAXCS * CL_THREADS * CL_MAXKPT) {
+    // clusters of 16 CTAs (opt-in) for images beyond 64 K positions, when the device schedules them
+    static int max_cs[64] = {0};
+    int devc = 0;
+    WCC_CUDA_TRY(cudaGetDevice(&devc));
+    if (devc >= 0 && devc < 64 && max_cs[devc] == 0) {
+        max_cs[devc] = 8;
+        if (cudaFuncSetAttribute(select_cluster_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+            cudaLaunchConfig_t q = {};
+            q.gridDim = dim3(16, 1);
+            q.blockDim = dim3(CL_THREADS);
+            cudaLaunchAttribute qa[1];
+            qa[0].id = cudaLaunchAttributeClusterDimension;
+            qa[0].val.clusterDim.x = 16; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
+            q.attrs = qa; q.numAttrs = 1;
+            int nclusters = 0;
+            if (cudaOccupancyMaxActiveClusters(&nclusters, select_cluster_kernel, &q) == cudaSuccess && nclusters > 0) max_cs[devc] = 16;
+        }
+        (void)cudaGetLastError();
+    }
+    const int cs_cap = (devc >= 0 && devc < 64) ? max_cs[devc] : 8;
+    if (P <= 8 * CL_THREADS * CL_MAXKPT) {
         // as many CTAs per image as useful, then as few threads as hold the keys (<= 16 each): the per-thread cost of
         // the scans and barriers is fixed, so fewer, busier threads finish sooner
         int cs = 1;
-        while (cs < CL_MAXCS && cs * 512 < P) cs <<= 1;
+        while (cs < 8 && cs * 512 < P) cs <<= 1;
+        if (cs == 8 && cs_cap == 16 && P > 65536) cs = 16;
         int threads = 256;
         const int kpt_goal = hist1_ready ? 4 : CL_MAXKPT;               // few keys per thread when no scans are needed
         while (threads < CL_THREADS && (long long)cs * threads * kpt_goal < P) threads <<= 1;
