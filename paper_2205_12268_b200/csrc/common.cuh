@@ -69,21 +69,6 @@ __device__ __forceinline__ void hist_add(uint32_t* h, uint32_t bin, bool pred)
     }
 }
 
-// ---- programmatic dependent launch -----------------------------------------------------------------
-// A kernel launched with the programmatic-serialization attribute may become resident while its predecessor in the
-// stream still runs; it must call grid_dependency_wait() before touching anything the predecessor writes (the wait
-// returns once the predecessor has completed and its writes are visible; it is a no-op for an ordinary launch).
-// allow_dependents() lets the successor be scheduled early.
-__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void allow_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-
-inline bool use_pdl()
-{
-    static int v = -1;
-    if (v < 0) v = getenv("WCC_NO_PDL") ? 0 : 1;
-    return v == 1;
-}
-
 // ---- geometry of one call -------------------------------------------------------------------
 struct Geom {
     int N, C, H, W, L;

@@ -92,7 +92,31 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
                      ::"r"(tc::smem_u32(&ctl->tmem_base)), "r"((uint32_t)tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    grid_dependency_wait();                            // the select (and with it the first pass) is complete from here on
+    // start the first ring stages before the (slower) scattered loads of the keep / drop decisions
+    const T* xin = x + (size_t)n * Cin * P;
+    constexpr int LU = Ring::LU, SUBS = 8 / LU;
+    constexpr int UPK = 32 / UNIT_BYTES;               // units per K step
+    const int ksteps = krow / 32;
+    const int halves = (a_ksteps < ksteps) ? 2 : 1;
+    uint8_t* my_ring = shared_region + (VEC ? warp * RING2 * Ring::STAGE_BYTES : 0);
+    const uint32_t my_ring_s = tc::smem_u32(my_ring);
+    // units of half h taken by this warp: u0 + warp, u0 + warp + 4, ... below ur (units from ur on are zero padding)
+    auto half_units = [&](int h, int& u0, int& u1, int& ur, int& my_units) {
+        const int ks0 = h * a_ksteps, ks1 = min(ksteps, ks0 + a_ksteps);
+        u0 = ks0 * UPK; u1 = ks1 * UPK;
+        ur = min(u1, max(u0, (Cin + 7) / 8));
+        my_units = max(0, (ur - u0 - warp + 3) / 4);
+    };
+    auto ring_prologue = [&](int h) {
+        if (!VEC) return;
+        int u0, u1, ur, my_units;
+        half_units(h, u0, u1, ur, my_units);
+        const int nq = my_units * SUBS;
+#pragma unroll
+        for (int q = 0; q < RING2 - 1; ++q)
+            Ring::issue(my_ring_s, q, xin, P, W, q < nq ? Cin : 0, (u0 + warp + 4 * (q / SUBS)) * 8 + (q % SUBS) * LU, lp, lane);
+    };
+    ring_prologue(0);
     // kept or dropped: from the rank map when the select wrote one (thr[n][2] != 0: partial ties, or a test wants
     // the ranks), else by comparing the position's norm with the threshold key
     const uint32_t tkey = thr[n * 4], use_rank = thr[n * 4 + 2];
@@ -129,13 +153,6 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
     // single chunk of output channels) the K range is done in two halves that accumulate into the same TMEM tile, so
     // that A stays small enough for four CTAs per SM.
     // Warp w takes the 8-channel units w, w+4, ... of a half; inputs arrive LU channels at a time through its ring.
-    const T* xin = x + (size_t)n * Cin * P;
-    constexpr int LU = Ring::LU, SUBS = 8 / LU;
-    constexpr int UPK = 32 / UNIT_BYTES;               // units per K step
-    const int ksteps = krow / 32;
-    const int halves = (a_ksteps < ksteps) ? 2 : 1;
-    uint8_t* my_ring = shared_region + (VEC ? warp * RING2 * Ring::STAGE_BYTES : 0);
-    const uint32_t my_ring_s = tc::smem_u32(my_ring);
     const uint32_t a_addr = tc::smem_u32(sA), b_addr = tc::smem_u32(sB);
     volatile int no_abort = 0;
     uint32_t commits = 0;                              // MMA batches committed so far (same value in every thread)
@@ -156,21 +173,16 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
 
     for (int h = 0; h < halves; ++h) {
         const int ks0 = h * a_ksteps, ks1 = min(ksteps, ks0 + a_ksteps);
-        const int u0 = ks0 * UPK, u1 = ks1 * UPK;
+        int u0, u1, ur, my_units;
+        half_units(h, u0, u1, ur, my_units);
         if (h > 0) {                                   // the tensor core still reads A: wait for the first half
             ok = tc::mbar_wait(tc::smem_u32(&ctl->mma_done), (commits - 1u) & 1u, &no_abort);
             ok = __syncthreads_and(ok ? 1 : 0) != 0;
             if (!ok) break;
             tc::fence_after();
         }
-        const int ur = min(u1, max(u0, (Cin + 7) / 8));         // units from ur on hold only zero padding
-        const int my_units = max(0, (ur - u0 - warp + 3) / 4);
-        const int nq = my_units * SUBS;                // ring stages this warp will consume in this half
+        const int nq = my_units * SUBS;                // ring stages this warp consumes in this half (first ones in flight)
         auto chan0 = [&](int q) { return (u0 + warp + 4 * (q / SUBS)) * 8 + (q % SUBS) * LU; };
-        if (VEC) {
-#pragma unroll
-            for (int q = 0; q < RING2 - 1; ++q) Ring::issue(my_ring_s, q, xin, P, W, q < nq ? Cin : 0, chan0(q), lp, lane);
-        }
         for (int ui = 0; ui < my_units; ++ui) {
             const int u = u0 + warp + 4 * ui;
             uint32_t packed[8][4];     // per slot: 8 int8 codes (2 words) or 8 bf16 values (4 words)
@@ -260,6 +272,7 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
         if (h + 1 < halves) {                          // first half of K: start accumulating now (single chunk of N)
             if (threadIdx.x == 0) issue_mmas(ks0, ks1, ks0, 0, npad);
             ++commits;
+            ring_prologue(h + 1);                      // the second half's inputs fly while the tensor core works
         }
     }
 
@@ -364,19 +377,9 @@ static wcc_status fused_pass2_dispatch(const void* x, const void* Wq, const int3
     if (ctas > 0x7FFFFFFFLL) return WCC_ERR_SHAPE;
     auto launch = [&](auto kern) -> wcc_status {
         WCC_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)ctas);
-        cfg.blockDim = dim3(128);
-        cfg.dynamicSmemBytes = smem;
-        cfg.stream = st;
-        cudaLaunchAttribute attr[1];                       // may be scheduled while the select still runs
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = use_pdl() ? 1 : 0;
-        WCC_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, static_cast<const T*>(x), static_cast<const uint8_t*>(Wq), rank, nrm2, thr,
-                                        amax_kept, qmax, scale_w, N, Cin, Cout, H, W, k, kpad, npad, nchunk, tmem_cols, a_ksteps,
-                                        static_cast<T*>(y), static_cast<uint8_t*>(xq_tap), acc_tap, status));
+        kern<<<(unsigned)ctas, 128, smem, st>>>(static_cast<const T*>(x), static_cast<const uint8_t*>(Wq), rank, nrm2, thr, amax_kept,
+                                                qmax, scale_w, N, Cin, Cout, H, W, k, kpad, npad, nchunk, tmem_cols, a_ksteps,
+                                                static_cast<T*>(y), static_cast<uint8_t*>(xq_tap), acc_tap, status);
         WCC_LAUNCH_CHECK();
         return WCC_OK;
     };

@@ -450,7 +450,6 @@ __global__ void __launch_bounds__(NORMS_WARPS * 32)
 haar_norms_kernel(const T* __restrict__ x, int N, int C, int H, int W,
                   float* __restrict__ nrm2, float* __restrict__ amaxpos, const NormsExtra ex)
 {
-    allow_dependents();                                // the select may be scheduled behind this grid right away
     if ((int)blockIdx.x >= ex.tiles) {                 // weight preparation CTAs
         const int o = ((int)blockIdx.x - ex.tiles) * NORMS_WARPS + (int)(threadIdx.x >> 5);
         if (o < ex.Cout) weight_prep_row(ex.Wt, o, C, ex.kpad, ex.bits, ex.Wq, ex.scale_w);

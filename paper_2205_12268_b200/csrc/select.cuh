@@ -595,8 +595,6 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
     const float* v = nrm2 + (size_t)n * P;
     const int base = (crank * (int)blockDim.x + (int)threadIdx.x) * kpt;  // kpt consecutive keys per thread
     const int lane = threadIdx.x & 31;
-    grid_dependency_wait();                          // the norms and histograms of the preceding launch are complete
-    allow_dependents();                              // whoever follows may set itself up now (it waits for this grid)
 
     uint32_t key[CL_MAXKPT];
 #pragma unroll
@@ -821,15 +819,13 @@ wcc_status launch_select(const float* nrm2, int N, int P, int k, int32_t* idx, f
         cfg.blockDim = dim3(threads);
         cfg.dynamicSmemBytes = 0;
         cfg.stream = st;
-        cudaLaunchAttribute attr[2];
+        cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = cs;
         attr[0].val.clusterDim.y = 1;
         attr[0].val.clusterDim.z = 1;
-        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[1].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
-        cfg.numAttrs = (hist1_ready && use_pdl()) ? 2 : 1;    // behind the first pass of the fused layer: overlap the launch
+        cfg.numAttrs = 1;
         WCC_CUDA_TRY(cudaLaunchKernelEx(&cfg, select_cluster_kernel, nrm2, P, k, kpt, idx, tau, rank, amaxpos, amax_kept, hist1,
                                         hist1_ready ? fine : (const uint32_t*)nullptr, thr, (want_rank || !thr) ? 1 : 0));
         WCC_LAUNCH_CHECK();
