@@ -189,6 +189,7 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
 #pragma unroll
             for (int g = 0; g < 2; ++g) {                  // two groups of 4 channels
                 uint32_t code[4][8];                       // int8: float bits whose low byte is the code; bf16: value bits
+                float p[4][2][4], o[4][8];
 #pragma unroll
                 for (int dd4 = 0; dd4 < 4; ++dd4) {
                     const int d = g * 4 + dd4;             // channel within the unit
@@ -208,12 +209,14 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
                         for (int i = 0; i < 8; ++i) rawp.w[i] = 0u;
                         if (c < Cin) load_patch<T, VEC>(xin + (size_t)c * P, W, lp, rawp);
                     }
-                    float p[2][4], o[8];
-                    unpack_patch<T>(rawp, p);
-                    haar_fwd_lane<L>(p, o, lane);
+                    unpack_patch<T>(rawp, p[dd4]);
+                }
+                haar_fwd_lanes<L, 4>(p, o, lane);
+#pragma unroll
+                for (int dd4 = 0; dd4 < 4; ++dd4) {
 #pragma unroll
                     for (int s = 0; s < 8; s += 2) {
-                        float2 t = mul2(make_float2(o[s], o[s + 1]), make_float2(mul[s], mul[s + 1]));
+                        float2 t = mul2(make_float2(o[dd4][s], o[dd4][s + 1]), make_float2(mul[s], mul[s + 1]));
                         // int8: the low byte of (t + 1.5*2^23) is the two's complement code of rint(t); |t| <= qmax by
                         // construction.  Scalar adds on purpose: a packed add right after the packed product gets
                         // contracted into one fused operation, which rounds once and changes half-way codes.
@@ -318,16 +321,18 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
                 }
             }
             __syncthreads();
+            {
+                float sl[SUB / 4][8], p[SUB / 4][2][4];
 #pragma unroll
-            for (int jj = 0; jj < SUB / 4; ++jj) {
-                const int j = warp + 4 * jj;
-                const int o = n0 + s0 + j;
-                if (o < Cout) {                                      // warp-uniform
-                    float sl[8], p[2][4];
+                for (int jj = 0; jj < SUB / 4; ++jj) {
 #pragma unroll
-                    for (int s = 0; s < 8; ++s) sl[s] = stage[(j * 8 + s) * 32 + lane];
-                    haar_inv_lane<L>(sl, p, lane);
-                    store_patch<T, VEC>(y + ((size_t)n * Cout + o) * P, W, lp, p);
+                    for (int s = 0; s < 8; ++s) sl[jj][s] = stage[((warp + 4 * jj) * 8 + s) * 32 + lane];
+                }
+                haar_inv_lanes<L, SUB / 4>(sl, p, lane);
+#pragma unroll
+                for (int jj = 0; jj < SUB / 4; ++jj) {
+                    const int o = n0 + s0 + warp + 4 * jj;
+                    if (o < Cout) store_patch<T, VEC>(y + ((size_t)n * Cout + o) * P, W, lp, p[jj]);
                 }
             }
             __syncthreads();

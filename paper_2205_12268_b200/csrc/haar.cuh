@@ -18,6 +18,7 @@
 #pragma once
 
 #include "common.cuh"
+#include "tma.cuh"
 
 namespace wcc {
 
@@ -186,6 +187,115 @@ __device__ __forceinline__ void haar_inv_lane(const float (&o)[8], float (&p)[2]
     const float2 c = half2x(add2(t1, u1)), d = half2x(sub2(t1, u1));
     p[0][0] = a.x; p[0][1] = b.x; p[0][2] = a.y; p[0][3] = b.y;
     p[1][0] = c.x; p[1][1] = d.x; p[1][2] = c.y; p[1][3] = d.y;
+}
+
+// The same transforms on U independent channels at once, stage by stage: the shuffles of one stage are issued back to
+// back for all U channels, so their latencies overlap (shuffles keep their program order; channel after channel they
+// would form one long dependent chain).  Arithmetic per channel is exactly that of haar_fwd_lane / haar_inv_lane.
+template <int L, int U>
+__device__ __forceinline__ void haar_fwd_lanes(const float (&p)[U][2][4], float (&o)[U][8], int lane)
+{
+    using T = HaarTile<L>;
+    float2 ll[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const float2 a = make_float2(p[u][0][0], p[u][0][2]), b = make_float2(p[u][0][1], p[u][0][3]);
+        const float2 c = make_float2(p[u][1][0], p[u][1][2]), d = make_float2(p[u][1][1], p[u][1][3]);
+        const float2 s0 = add2(a, b), d0 = sub2(a, b), s1 = add2(c, d), d1 = sub2(c, d);
+        ll[u] = half2x(add2(s0, s1));
+        const float2 y2 = half2x(add2(d0, d1));
+        const float2 y3 = half2x(sub2(s0, s1));
+        const float2 y4 = half2x(sub2(d0, d1));
+        o[u][0] = y2.x; o[u][1] = y2.y; o[u][2] = y3.x; o[u][3] = y3.y; o[u][4] = y4.x; o[u][5] = y4.y;
+        if (L == 1) { o[u][6] = ll[u].x; o[u][7] = ll[u].y; }
+    }
+    if (L == 1) return;
+    const int rp = lane / T::CG, cg = lane % T::CG;
+    const bool even = (rp & 1) == 0;
+    const float sg = even ? 1.0f : -1.0f;
+    float s[U], dd[U], ps[U], pd[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) { s[u] = __fadd_rn(ll[u].x, ll[u].y); dd[u] = __fsub_rn(ll[u].x, ll[u].y); }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        ps[u] = __shfl_xor_sync(0xFFFFFFFFu, s[u], T::CG);
+        pd[u] = __shfl_xor_sync(0xFFFFFFFFu, dd[u], T::CG);
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const float2 l2 = half2x(__ffma2_rn(make_float2(s[u], dd[u]), make_float2(sg, sg), make_float2(ps[u], pd[u])));
+        o[u][6] = l2.x;
+        o[u][7] = l2.y;
+    }
+    if (L == 3) {
+        const float sgh = (cg & 1) == 0 ? 1.0f : -1.0f;
+        const float sgv = (rp & 2) == 0 ? 1.0f : -1.0f;
+        float h[U], t[U], q[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) h[u] = __shfl_xor_sync(0xFFFFFFFFu, o[u][6], 1);
+#pragma unroll
+        for (int u = 0; u < U; ++u) t[u] = __fmaf_rn(o[u][6], sgh, h[u]);
+#pragma unroll
+        for (int u = 0; u < U; ++u) q[u] = __shfl_xor_sync(0xFFFFFFFFu, t[u], 2 * T::CG);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const float r = __fmul_rn(__fmaf_rn(t[u], sgv, q[u]), 0.5f);
+            if (even) o[u][6] = r;
+        }
+    }
+}
+
+template <int L, int U>
+__device__ __forceinline__ void haar_inv_lanes(const float (&o)[U][8], float (&p)[U][2][4], int lane)
+{
+    using T = HaarTile<L>;
+    float2 ll[U];
+    if (L == 1) {
+#pragma unroll
+        for (int u = 0; u < U; ++u) ll[u] = make_float2(o[u][6], o[u][7]);
+    } else {
+        const int rp = lane / T::CG, cg = lane % T::CG;
+        const float sg = (rp & 1) == 0 ? 1.0f : -1.0f;
+        float m0[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) m0[u] = o[u][6];
+        if (L == 3) {
+            const float sgh = (cg & 1) == 0 ? 1.0f : -1.0f;
+            const float sgv = (rp & 2) == 0 ? 1.0f : -1.0f;
+            float pv[U], w[U], q[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) pv[u] = __shfl_xor_sync(0xFFFFFFFFu, m0[u], 2 * T::CG);
+#pragma unroll
+            for (int u = 0; u < U; ++u) w[u] = __fmaf_rn(m0[u], sgv, pv[u]);
+#pragma unroll
+            for (int u = 0; u < U; ++u) q[u] = __shfl_xor_sync(0xFFFFFFFFu, w[u], 1);
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const float r = __fmul_rn(__fmaf_rn(w[u], sgh, q[u]), 0.5f);
+                if ((rp & 1) == 0) m0[u] = r;
+            }
+        }
+        float p0[U], p1[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            p0[u] = __shfl_xor_sync(0xFFFFFFFFu, m0[u], T::CG);
+            p1[u] = __shfl_xor_sync(0xFFFFFFFFu, o[u][7], T::CG);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const float2 tu = __ffma2_rn(make_float2(m0[u], o[u][7]), make_float2(sg, sg), make_float2(p0[u], p1[u]));
+            ll[u] = make_float2(__fmul_rn(__fadd_rn(tu.x, tu.y), 0.5f), __fmul_rn(__fsub_rn(tu.x, tu.y), 0.5f));
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const float2 y2 = make_float2(o[u][0], o[u][1]), y3 = make_float2(o[u][2], o[u][3]), y4 = make_float2(o[u][4], o[u][5]);
+        const float2 t0 = add2(ll[u], y3), t1 = sub2(ll[u], y3), u0 = add2(y2, y4), u1 = sub2(y2, y4);
+        const float2 a = half2x(add2(t0, u0)), b = half2x(sub2(t0, u0));
+        const float2 c = half2x(add2(t1, u1)), d = half2x(sub2(t1, u1));
+        p[u][0][0] = a.x; p[u][0][1] = b.x; p[u][0][2] = a.y; p[u][0][3] = b.y;
+        p[u][1][0] = c.x; p[u][1][1] = d.x; p[u][1][2] = c.y; p[u][1][3] = d.y;
+    }
 }
 
 // ---- patch load / store ------------------------------------------------------------------------
@@ -423,7 +533,7 @@ struct PatchRing {
     }
 };
 
-// ---- first pass of the fused layer: norms only -------------------------------------------------
+// ---- first pass of the fused layer: norms only (inputs through per-warp cp.async rings) -----------
 // One CTA of 4 warps per (image, tile).  The warps split the channels: in every round of 4 * LU channels warp w
 // transforms channels [w * LU, (w + 1) * LU) of the round in registers and hands the slot values over through shared
 // memory; then the 128 threads run the fused multiply-add chain of two positions each (warp w: slots 2w and 2w+1
@@ -442,6 +552,50 @@ struct NormsExtra {
     int Cout, kpad, bits;
     int tiles;            // CTAs that transform; CTAs beyond prepare weights
 };
+
+// Last step of the first pass for warps 0..3: thread (warp, lane) owns slot pair `warp` of its lane; write the norms and
+// the max |coef|, and count the norms in the select's histograms.
+template <int L, bool VEC>
+__device__ __forceinline__ void norms_finish(const LanePos& lp, int warp, int n, size_t P, float n0, float n1, float a0, float a1,
+                                             float* __restrict__ nrm2, float* __restrict__ amaxpos, const NormsExtra& ex)
+{
+    int p0 = 0, p1 = 0;
+    bool ok0 = false, ok1 = false;
+#pragma unroll
+    for (int s = 0; s < 8; s += 2) {
+        if (s == 2 * warp) {
+            p0 = lp.pos[s]; p1 = lp.pos[s + 1];
+            ok0 = slot_ok<L>(lp, s); ok1 = slot_ok<L>(lp, s + 1);
+        }
+    }
+    const bool pair = VEC && (L == 1 || warp < 3);     // adjacent, 8-byte aligned positions
+    float* nr = nrm2 + (size_t)n * P;
+    if (pair) {
+        if (ok0) *reinterpret_cast<float2*>(nr + p0) = make_float2(n0, n1);
+    } else {
+        if (ok0) nr[p0] = n0;
+        if (ok1) nr[p1] = n1;
+    }
+    if (amaxpos) {
+        float* am = amaxpos + (size_t)n * P;
+        if (pair) {
+            if (ok0) *reinterpret_cast<float2*>(am + p0) = make_float2(a0, a1);
+        } else {
+            if (ok0) am[p0] = a0;
+            if (ok1) am[p1] = a1;
+        }
+    }
+    if (ex.hist1) {                                    // norms are >= +0: key = bits | sign bit, digit = top 11 bits
+        uint32_t* h = ex.hist1 + (size_t)n * 3 * 2048;
+        hist_add(h, float_key(n0) >> 21, ok0);
+        hist_add(h, float_key(n1) >> 21, ok1);
+    }
+    if (ex.fine) {                                     // 16-bit digits are spread out: plain atomics
+        uint32_t* f = ex.fine + (size_t)n * 65536;
+        if (ok0) atomicAdd(&f[float_key(n0) >> 16], 1u);
+        if (ok1) atomicAdd(&f[float_key(n1) >> 16], 1u);
+    }
+}
 
 constexpr int NORMS_WARPS = 8;     // warps per CTA: the transform is issue-latency bound, more warps hide it
 
@@ -483,6 +637,7 @@ haar_norms_kernel(const T* __restrict__ x, int N, int C, int H, int W,
             Ring::issue(my_ring_s, (r + RING - 1) % RING, xin, P, W, C, (r + RING - 1) * RC + warp * LU, lp, lane);
             Ring::template wait<RING - 1>();
         }
+        float p[LU][2][4], o[LU][8];
 #pragma unroll
         for (int d = 0; d < LU; ++d) {
             const int c = r * RC + warp * LU + d;
@@ -494,12 +649,15 @@ haar_norms_kernel(const T* __restrict__ x, int N, int C, int H, int W,
                 for (int i = 0; i < 8; ++i) raw.w[i] = 0u;
                 if (c < C) load_patch<T, VEC>(xin + (size_t)c * P, W, lp, raw);
             }
-            float p[2][4], o[8];
-            unpack_patch<T>(raw, p);
-            haar_fwd_lane<L>(p, o, lane);
+            unpack_patch<T>(raw, p[d]);
+        }
+        haar_fwd_lanes<L, LU>(p, o, lane);
 #pragma unroll
-            for (int s = 0; s < 8; s += 2) buf[warp * LU + d][s >> 1][lane] = make_float2(o[s], o[s + 1]);
-            if (ex.coef && c < C) store_slots<L, VEC>(ex.coef + ((size_t)n * C + c) * P, lp, o);
+        for (int d = 0; d < LU; ++d) {
+            const int c = r * RC + warp * LU + d;
+#pragma unroll
+            for (int s = 0; s < 8; s += 2) buf[warp * LU + d][s >> 1][lane] = make_float2(o[d][s], o[d][s + 1]);
+            if (ex.coef && c < C) store_slots<L, VEC>(ex.coef + ((size_t)n * C + c) * P, lp, o[d]);
         }
         __syncthreads();
         // the chain: warps 0..3 own slot pair `warp` of every lane.  Channels beyond C contribute fma(0, 0, acc) = acc
@@ -517,43 +675,173 @@ haar_norms_kernel(const T* __restrict__ x, int N, int C, int H, int W,
     }
     if (VEC) Ring::template wait<0>();
     if (warp >= 4) return;
-    const float n0 = nn.x, n1 = nn.y;
-    int p0 = 0, p1 = 0;
-    bool ok0 = false, ok1 = false;
+    norms_finish<L, VEC>(lp, warp, n, P, nn.x, nn.y, a0, a1, nrm2, amaxpos, ex);
+}
+
+// ---- per-warp ring of TMA boxes --------------------------------------------------------------------
+// One lane of a warp asks the TMA unit for boxes of CB channels x (tile rows) x (tile columns) of one image
+// (cp.async.bulk.tensor, completion counted on an mbarrier per stage); no thread spends instructions or registers on
+// addresses, and the copies bypass the load/store pipe.  A stage is laid out [channel][row][column], dense.  Only the
+// owning warp reads a stage and only its lane 0 refills it (after __syncwarp), so no "empty" barrier is needed.
+template <typename T, int L, int CB_, int S_>
+struct TileRing {
+    using TT = HaarTile<L>;
+    static constexpr int CB = CB_, S = S_;
+    static constexpr int ROW_BYTES = TT::TW * (int)sizeof(T);
+    static constexpr int CH_BYTES = TT::TH * ROW_BYTES;          // 256 positions: 512 (bf16) or 1024 (fp32) bytes
+    static constexpr int STAGE_BYTES = CB * CH_BYTES;
+    static constexpr int BYTES = S * STAGE_BYTES;
+    // bf16, L = 3: rows are 64 bytes, so the rows 2rp of the four lane rows would all start in the same banks; lanes
+    // with odd rp read their second row first, which spreads one load over all 32 banks
+    static constexpr bool ALT = (sizeof(T) == 2 && L == 3);
+
+    uint32_t ring_s, bar_s;      // shared-space addresses of the stages and of the S mbarriers
+    const uint8_t* ring;
+    int off_a, off_b;            // byte offsets (inside a channel) of the row this lane reads first / second
+    bool swap;                   // the first row read is the patch's second row
+
+    __device__ __forceinline__ void init(uint8_t* stages, uint64_t* bars, int lane)
+    {
+        ring = stages;
+        ring_s = tc::smem_u32(stages);
+        bar_s = tc::smem_u32(bars);
+        set_lane(lane);
+        if (lane == 0) {
 #pragma unroll
-    for (int s = 0; s < 8; s += 2) {
-        if (s == 2 * warp) {
-            p0 = lp.pos[s]; p1 = lp.pos[s + 1];
-            ok0 = slot_ok<L>(lp, s); ok1 = slot_ok<L>(lp, s + 1);
+            for (int i = 0; i < S; ++i) tc::mbar_init(bar_s + 8 * i, 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
+        __syncwarp();
     }
-    const bool pair = VEC && (L == 1 || warp < 3);     // adjacent, 8-byte aligned positions
-    float* nr = nrm2 + (size_t)n * P;
-    if (pair) {
-        if (ok0) *reinterpret_cast<float2*>(nr + p0) = make_float2(n0, n1);
-    } else {
-        if (ok0) nr[p0] = n0;
-        if (ok1) nr[p1] = n1;
+    __device__ __forceinline__ void set_lane(int lane)
+    {
+        const int rp = lane / TT::CG, cg = lane % TT::CG;
+        swap = ALT && (rp & 1);
+        const int base = 2 * rp * ROW_BYTES + 4 * cg * (int)sizeof(T);
+        off_a = base + (swap ? ROW_BYTES : 0);
+        off_b = base + (swap ? 0 : ROW_BYTES);
     }
-    if (amaxpos) {
-        float* am = amaxpos + (size_t)n * P;
-        if (pair) {
-            if (ok0) *reinterpret_cast<float2*>(am + p0) = make_float2(a0, a1);
+    // lane 0 only: request channels [c0, c0 + CB) of image n at tile origin (x0, y0) into `stage`
+    __device__ __forceinline__ void issue(const CUtensorMap* tm, int stage, int x0, int y0, int c0, int n) const
+    {
+        tc::mbar_expect_tx(bar_s + 8 * stage, STAGE_BYTES);
+        tc::tma_load_4d(ring_s + stage * STAGE_BYTES, tm, x0, y0, c0, n, bar_s + 8 * stage);
+    }
+    __device__ __forceinline__ bool wait(int stage, uint32_t parity) const { return tc::mbar_wait(bar_s + 8 * stage, parity); }
+
+    __device__ __forceinline__ void read(int stage, int d, RawPatch& raw) const
+    {
+        const uint8_t* ch = ring + stage * STAGE_BYTES + d * CH_BYTES;
+        if (sizeof(T) == 4) {
+            const uint4 a = *reinterpret_cast<const uint4*>(ch + off_a);
+            const uint4 b = *reinterpret_cast<const uint4*>(ch + off_b);
+            raw.w[0] = a.x; raw.w[1] = a.y; raw.w[2] = a.z; raw.w[3] = a.w;
+            raw.w[4] = b.x; raw.w[5] = b.y; raw.w[6] = b.z; raw.w[7] = b.w;
         } else {
-            if (ok0) am[p0] = a0;
-            if (ok1) am[p1] = a1;
+            const uint2 a = *reinterpret_cast<const uint2*>(ch + off_a);
+            const uint2 b = *reinterpret_cast<const uint2*>(ch + off_b);
+            raw.w[0] = (ALT && swap) ? b.x : a.x; raw.w[1] = (ALT && swap) ? b.y : a.y;
+            raw.w[4] = (ALT && swap) ? a.x : b.x; raw.w[5] = (ALT && swap) ? a.y : b.y;
         }
     }
-    if (ex.hist1) {                                    // norms are >= +0: key = bits | sign bit, digit = top 11 bits
-        uint32_t* h = ex.hist1 + (size_t)n * 3 * 2048;
-        hist_add(h, float_key(n0) >> 21, ok0);
-        hist_add(h, float_key(n1) >> 21, ok1);
+};
+
+// After a wait ran out: report it and give copies that may still be in flight time to land before the CTA's shared
+// memory is handed to another CTA.
+__device__ __noinline__ void tma_timeout(int* status)
+{
+    if ((threadIdx.x & 31) == 0) atomicExch(status, (int)WCC_ERR_TIMEOUT);
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+}
+
+// ---- first pass, eight warps per tile, TMA-fed -----------------------------------------------------
+// The work split of haar_norms_kernel (warps transform different channels of a round, hand the values over through
+// shared memory, four warps run the chains) with the inputs of a whole round arriving as one TMA box.
+template <typename T, int L>
+struct NormsTmaCfg {
+    static constexpr int LU = (sizeof(T) == 2) ? 2 : 1;
+    static constexpr int RC = NORMS_WARPS * LU;                   // channels per round = per box
+    using Ring = TileRing<T, L, RC, 4>;                           // 4 x 8 KB
+    static constexpr size_t SMEM = 128 + Ring::BYTES + Ring::S * 8 + (size_t)RC * 4 * 32 * sizeof(float2);
+};
+
+template <typename T, int L>
+__global__ void __launch_bounds__(NORMS_WARPS * 32)
+haar_norms_tma_kernel(const __grid_constant__ CUtensorMap tmx, int N, int C, int H, int W,
+                       float* __restrict__ nrm2, float* __restrict__ amaxpos, const NormsExtra ex, int* __restrict__ status)
+{
+    if ((int)blockIdx.x >= ex.tiles) {                 // weight preparation CTAs
+        const int o = ((int)blockIdx.x - ex.tiles) * NORMS_WARPS + (int)(threadIdx.x >> 5);
+        if (o < ex.Cout) weight_prep_row(ex.Wt, o, C, ex.kpad, ex.bits, ex.Wq, ex.scale_w);
+        return;
     }
-    if (ex.fine) {                                     // 16-bit digits are spread out: plain atomics
-        uint32_t* f = ex.fine + (size_t)n * 65536;
-        if (ok0) atomicAdd(&f[float_key(n0) >> 16], 1u);
-        if (ok1) atomicAdd(&f[float_key(n1) >> 16], 1u);
+    using TT = HaarTile<L>;
+    using Cfg = NormsTmaCfg<T, L>;
+    using Ring = typename Cfg::Ring;
+    constexpr int LU = Cfg::LU, RC = Cfg::RC, S = Ring::S;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_s = tc::smem_u32(smem_raw);
+    uint8_t* sm = smem_raw + (((raw_s + 127u) & ~127u) - raw_s);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sm + Ring::BYTES);
+    float2 (*buf)[4][32] = reinterpret_cast<float2 (*)[4][32]>(sm + Ring::BYTES + S * 8);   // [channel of the round][slot pair][lane]
+
+    const int tiles_x = (W + TT::TW - 1) / TT::TW, tiles_y = H / TT::TH;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int n, ty, tx;
+    tile_coords(blockIdx.x, tiles_x, tiles_y, n, ty, tx);
+    const LanePos lp = lane_positions<L>(H, W, ty, tx, lane);
+    const size_t P = (size_t)H * W;
+    const int x0 = tx * TT::TW, y0 = ty * TT::TH;
+
+    Ring ring;
+    ring.init(sm, bars, threadIdx.x == 0 ? 0 : 1);     // thread 0 initializes the barriers
+    __syncthreads();
+    const int rounds = (C + RC - 1) / RC;
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int i = 0; i < S; ++i)
+            if (i < rounds) ring.issue(&tmx, i, x0, y0, i * RC, n);
     }
+    // lane geometry of the ring reads (init() computed them for lane 0 / 1 only)
+    ring.set_lane(lane);
+
+    float2 nn = make_float2(0.0f, 0.0f);
+    float a0 = 0.0f, a1 = 0.0f;
+    bool ok = true;
+    for (int r = 0; r < rounds; ++r) {
+        const int stage = r % S;
+        if (ok) ok = ring.wait(stage, (uint32_t)(r / S) & 1u);   // after a timeout: no more waits, same barrier count
+        float p[LU][2][4], o[LU][8];
+#pragma unroll
+        for (int d = 0; d < LU; ++d) {
+            RawPatch raw;
+            ring.read(stage, warp * LU + d, raw);      // channels beyond C arrive as zeros
+            unpack_patch<T>(raw, p[d]);
+        }
+        haar_fwd_lanes<L, LU>(p, o, lane);
+#pragma unroll
+        for (int d = 0; d < LU; ++d) {
+            const int c = r * RC + warp * LU + d;
+#pragma unroll
+            for (int s = 0; s < 8; s += 2) buf[warp * LU + d][s >> 1][lane] = make_float2(o[d][s], o[d][s + 1]);
+            if (ex.coef && c < C) store_slots<L, true>(ex.coef + ((size_t)n * C + c) * P, lp, o[d]);
+        }
+        __syncthreads();                               // values handed over; every warp is done reading the stage
+        if (threadIdx.x == 0 && r + S < rounds) ring.issue(&tmx, stage, x0, y0, (r + S) * RC, n);
+        if (warp < 4) {
+#pragma unroll
+            for (int c = 0; c < RC; ++c) {
+                const float2 v = buf[c][warp][lane];
+                nn = __ffma2_rn(v, v, nn);
+                a0 = fmaxf(a0, fabsf(v.x));
+                a1 = fmaxf(a1, fabsf(v.y));
+            }
+        }
+        __syncthreads();
+    }
+    if (!__syncthreads_and(ok ? 1 : 0)) { tma_timeout(status); return; }
+    if (warp >= 4) return;
+    norms_finish<L, true>(lp, warp, n, P, nn.x, nn.y, a0, a1, nrm2, amaxpos, ex);
 }
 
 // ---- plain inverse -------------------------------------------------------------------------------
@@ -637,19 +925,17 @@ scatter_inv_kernel(const int32_t* __restrict__ acc, int ldc, const int32_t* __re
 
 // ---- launchers -------------------------------------------------------------------------------
 template <typename T, int L, bool VEC>
+static wcc_status haar_norms_dispatch(const void* x, int N, int C, int H, int W, float* nrm2, float* amaxpos,
+                                      NormsExtra ex, cudaStream_t st);
+
+template <typename T, int L, bool VEC>
 static wcc_status haar_fwd_dispatch(const void* x, int N, int C, int H, int W, float* coef, float* nrm2,
                                     float* amaxpos, cudaStream_t st)
 {
     using TT = HaarTile<L>;
     constexpr int D = (sizeof(T) == 4) ? 4 : 8;
     const long long warps = (long long)N * ceil_div(W, TT::TW) * (H / TT::TH);
-    if (!coef && nrm2) {          // norms only: four warps per tile
-        NormsExtra ex = {};
-        ex.tiles = (int)warps;
-        haar_norms_kernel<T, L, VEC><<<(unsigned)warps, NORMS_WARPS * 32, 0, st>>>(static_cast<const T*>(x), N, C, H, W, nrm2, amaxpos, ex);
-        WCC_LAUNCH_CHECK();
-        return WCC_OK;
-    }
+    if (!coef && nrm2) return haar_norms_dispatch<T, L, VEC>(x, N, C, H, W, nrm2, amaxpos, NormsExtra{}, st);   // norms only
     const int blocks = (int)((warps + 3) / 4);
     haar_fwd_kernel<T, L, VEC, D><<<blocks, 128, 0, st>>>(static_cast<const T*>(x), N, C, H, W, coef, nrm2, amaxpos);
     WCC_LAUNCH_CHECK();
@@ -675,6 +961,19 @@ static wcc_status haar_norms_dispatch(const void* x, int N, int C, int H, int W,
 {
     using TT = HaarTile<L>;
     const long long tiles = (long long)N * ceil_div(W, TT::TW) * (H / TT::TH);
+    if (VEC && tc::tma_ok_x(x, (int)sizeof(T), W)) {
+        using Cfg = NormsTmaCfg<T, L>;
+        CUtensorMap tmx;
+        if (!tc::make_map_x(&tmx, x, (int)sizeof(T), N, C, H, W, TT::TW, TT::TH, Cfg::RC)) return WCC_ERR_CUDA;
+        int* status = nullptr;
+        WCC_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_status));
+        WCC_CUDA_TRY(cudaFuncSetAttribute(haar_norms_tma_kernel<T, L>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM));
+        ex.tiles = (int)tiles;
+        const long long grid = tiles + (ex.Wt ? ceil_div(ex.Cout, NORMS_WARPS) : 0);
+        haar_norms_tma_kernel<T, L><<<(unsigned)grid, NORMS_WARPS * 32, Cfg::SMEM, st>>>(tmx, N, C, H, W, nrm2, amaxpos, ex, status);
+        WCC_LAUNCH_CHECK();
+        return WCC_OK;
+    }
     ex.tiles = (int)tiles;
     const long long grid = tiles + (ex.Wt ? ceil_div(ex.Cout, NORMS_WARPS) : 0);
     haar_norms_kernel<T, L, VEC><<<(unsigned)grid, NORMS_WARPS * 32, 0, st>>>(static_cast<const T*>(x), N, C, H, W, nrm2, amaxpos, ex);
