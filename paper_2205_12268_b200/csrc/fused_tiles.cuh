@@ -1,0 +1,412 @@
+// Second pass of the fused layer, four tiles per CTA (steps A, C, D, E of the WCC workflow, Eq. 9 / Alg. 1, with the
+// index set and the activation scale of step B already known): transform from x, keep / drop, quantize, pointwise
+// convolution on tensor cores, dequantize, inverse transform, store y.
+//
+// A CTA owns four warp tiles (4 x 256 = 1024 wavelet-domain positions, see haar.cuh) and runs 4 * WPT compute warps
+// plus one warp that issues the tensor-core instructions.  Compute warp w works for tile t = w % 4; the WPT warps of a
+// tile split the input channels (in 16-byte chunks of an operand row) on the way in and the output channels (in groups
+// of eight) on the way out.  Rows of the A operand are ordered  slot * 128 + t * 32 + lane,  so MMA block b (128 rows)
+// holds slot b of all four tiles and the accumulators of tile t's lanes sit in TMEM lanes 32t .. 32t+31: exactly the
+// lane quarter that warp w = t (mod 4) may read.  Every thread therefore reads back its own eight slots of an output
+// channel with tcgen05.ld and runs the inverse transform in registers; nothing is transposed through shared memory.
+//
+// Inputs arrive through a per-warp ring of TMA boxes (CB channels of the warp's tile each); the A operand is handed to
+// the tensor core one K step (32 bytes of K per row, 32 KB) at a time through mbarriers:
+//   full_a[buf]  8 arrivals (4 tiles x 2 chunks)  -> the issuing warp runs 8 MMAs (one per block) on that K step
+//   empty_a[buf] tcgen05.commit                   -> the buffer may be overwritten
+//   ready[tb]    tcgen05.commit                   -> accumulator buffer tb holds a finished chunk of output channels
+//   tfree[tb]    one arrival per compute warp     -> accumulator buffer tb has been read back
+// With one chunk of output channels (<= 64) K steps stream through two A buffers; with several chunks (32 channels each,
+// two accumulator buffers) every K step stays resident.  No block-wide barrier between set-up and tear-down.
+// Every mbarrier wait is bounded and reports WCC_ERR_TIMEOUT.
+#pragma once
+
+#include "common.cuh"
+#include "contract.cuh"
+#include "fused.cuh"
+#include "haar.cuh"
+
+namespace wcc {
+namespace ft {
+
+constexpr int TILES = 4;                    // warp tiles per CTA
+constexpr int ROWS = TILES * 256;           // operand rows per CTA
+constexpr int KSTEP_BYTES = ROWS * 32;      // one K step of A
+constexpr int MAX_NA = 4;
+
+struct Ctl {
+    uint64_t full_a[MAX_NA];
+    uint64_t empty_a[MAX_NA];
+    uint64_t ready[2];
+    uint64_t tfree[2];
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+template <typename T, bool I8, int WPT>
+struct Cfg {
+    static constexpr int CWARPS = TILES * WPT;
+    static constexpr int THREADS = (CWARPS + 1) * 32;
+    static constexpr int CB = (sizeof(T) == 2) ? 8 : 4;          // channels per TMA box: 4 KB
+    static constexpr int S = (WPT >= 4) ? 2 : 4;                  // boxes in flight per warp
+    static constexpr int CCH = I8 ? 16 : 8;                       // channels per 16-byte operand chunk
+    static constexpr int BPC = CCH / CB;                          // boxes per chunk
+    static constexpr int GROUPS = CCH / 4;                        // groups of four channels per chunk
+};
+
+struct Params {
+    const uint8_t* Wq; const int32_t* rank; const float* nrm2; const uint32_t* thr; const float* amax_kept;
+    const float* scale_w; float qmax;
+    int N, Cin, Cout, H, W, k, kpad, npad, nchunk, nn, nbuf, tmem_cols, na, tiles_total;
+    void* y; uint8_t* xq_tap; int32_t* acc_tap; int* status;
+};
+
+template <typename T, int L, bool I8, int WPT>
+__global__ void __launch_bounds__(Cfg<T, I8, WPT>::THREADS, 1)
+fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
+{
+    using TT = HaarTile<L>;
+    using C = Cfg<T, I8, WPT>;
+    using Ring = TileRing<T, L, C::CB, C::S>;
+    constexpr int ES = I8 ? 1 : 2;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = tc::smem_u32(smem_raw);
+    uint8_t* sm = smem_raw + (((raw + 127u) & ~127u) - raw);
+    const int krow = pr.kpad * ES, kchunks = krow / 16, ksteps = krow / 32;
+    uint8_t* sA = sm;                                                         // [na][2][ROWS][16]
+    uint8_t* sRing = sA + (size_t)pr.na * KSTEP_BYTES;                        // [CWARPS][S][4 KB]
+    uint8_t* sB = sRing + (size_t)C::CWARPS * Ring::BYTES;                    // [kchunks][npad][16]
+    uint64_t* ring_bars = reinterpret_cast<uint64_t*>(sB + (size_t)kchunks * pr.npad * 16);   // [CWARPS][S]
+    Ctl* ctl = reinterpret_cast<Ctl*>(ring_bars + C::CWARPS * C::S);
+    volatile int* abort_flag = &ctl->abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool is_mma = warp == C::CWARPS;
+    const int t = warp & 3, q = warp >> 2;
+
+    // ---- set-up -------------------------------------------------------------------------------------
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < MAX_NA; ++i) { tc::mbar_init(tc::smem_u32(&ctl->full_a[i]), 2 * TILES); tc::mbar_init(tc::smem_u32(&ctl->empty_a[i]), 1); }
+        for (int i = 0; i < 2; ++i) { tc::mbar_init(tc::smem_u32(&ctl->ready[i]), 1); tc::mbar_init(tc::smem_u32(&ctl->tfree[i]), C::CWARPS); }
+        ctl->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (is_mma) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(tc::smem_u32(&ctl->tmem_base)), "r"((uint32_t)pr.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    const int tile = (int)blockIdx.x * TILES + t;
+    const bool live = !is_mma && tile < pr.tiles_total;
+    const int tiles_x = (pr.W + TT::TW - 1) / TT::TW, tiles_y = pr.H / TT::TH;
+    int n = 0, ty = 0, tx = 0;
+    if (live) tile_coords(tile, tiles_x, tiles_y, n, ty, tx);
+    const LanePos lp = lane_positions<L>(pr.H, pr.W, ty, tx, lane);
+    const size_t P = (size_t)pr.H * pr.W;
+    const int x0 = tx * TT::TW, y0 = ty * TT::TH;
+
+    // this warp's operand chunks: j = q, q + WPT, ... < kchunks; boxes in consumption order: m -> chunk m / BPC
+    const int my_chunks = is_mma ? 0 : (kchunks - q + WPT - 1) / WPT;
+    const int my_boxes = live ? my_chunks * C::BPC : 0;
+    auto box_c0 = [&](int m) { return (q + (m / C::BPC) * WPT) * C::CCH + (m % C::BPC) * C::CB; };
+    Ring ring;
+    if (!is_mma) {
+        ring.init(sRing + (size_t)warp * Ring::BYTES, ring_bars + warp * C::S, lane);
+        if (lane == 0) {
+#pragma unroll
+            for (int m = 0; m < C::S; ++m)
+                if (m < my_boxes) ring.issue(&tmx, m, x0, y0, box_c0(m), n);
+        }
+    }
+    // weights -> B operand (core-matrix layout), all threads
+    for (int i = threadIdx.x; i < pr.npad * kchunks; i += C::THREADS) {
+        const int row = i / kchunks, j = i - row * kchunks;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (row < pr.Cout) v = *reinterpret_cast<const uint4*>(pr.Wq + (size_t)row * krow + j * 16);
+        *reinterpret_cast<uint4*>(sB + ((size_t)j * pr.npad + row) * 16) = v;
+    }
+    // kept or dropped: from the rank map when the select wrote one (thr[n][2] != 0), else by the threshold key
+    float mul[8];
+    int rk[8];
+#pragma unroll
+    for (int s = 0; s < 8; ++s) { mul[s] = 0.0f; rk[s] = -1; }
+    float scale_a = 1.0f;
+    if (live) {
+        float inv = 1.0f;
+        if (I8) {
+            const float amax = *pr.amax_kept;
+            inv = (amax > 0.0f) ? __fdiv_rn(pr.qmax, amax) : 0.0f;
+            scale_a = __fdiv_rn(amax, pr.qmax);
+        }
+        const uint32_t tkey = pr.thr[n * 4], use_rank = pr.thr[n * 4 + 2];
+#pragma unroll
+        for (int s = 0; s < 8; ++s) {
+            if (slot_ok<L>(lp, s)) {
+                if (use_rank) rk[s] = pr.rank[(size_t)n * P + lp.pos[s]];
+                else rk[s] = (float_key(pr.nrm2[(size_t)n * P + lp.pos[s]]) >= tkey) ? 0 : -1;
+            }
+            mul[s] = (rk[s] >= 0) ? inv : 0.0f;
+        }
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");       // B operand -> visible to the tensor core
+    tc::fence_before();
+    __syncthreads();
+    tc::fence_after();
+    const uint32_t tmem = ctl->tmem_base;
+    const uint32_t a_addr = tc::smem_u32(sA), b_addr = tc::smem_u32(sB);
+    bool ok = true;
+
+    if (is_mma) {
+        // ---- tensor-core issue ------------------------------------------------------------------------
+        if (lane == 0) {
+            auto idesc_of = [&](int cur) {
+                return (I8 ? (2u << 4) : (1u << 4)) | (1u << 7) | (1u << 10) | ((uint32_t)(cur >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+            };
+            auto mma_kstep = [&](int ks, int buf, int n0, int cur, uint32_t d0, bool first) {
+#pragma unroll 1
+                for (int b = 0; b < 8; ++b) {
+                    const uint64_t ad = fz::smem_desc_plain(a_addr + (uint32_t)(buf * KSTEP_BYTES + b * 128 * 16), ROWS * 16, 128);
+                    const uint64_t bd = fz::smem_desc_plain(b_addr + (uint32_t)((ks * 2 * pr.npad + n0) * 16), (uint32_t)pr.npad * 16, 128);
+                    tc::mma_ss<I8>(d0 + (uint32_t)(b * pr.nchunk), ad, bd, idesc_of(cur), first ? 0u : 1u);
+                }
+            };
+            if (pr.nn == 1) {
+                for (int ks = 0; ks < ksteps && ok; ++ks) {
+                    const int buf = ks % pr.na;
+                    ok = tc::mbar_wait(tc::smem_u32(&ctl->full_a[buf]), (uint32_t)(ks / pr.na) & 1u, abort_flag);
+                    if (!ok) break;
+                    tc::fence_after();
+                    mma_kstep(ks, buf, 0, pr.npad, tmem, ks == 0);
+                    tc::mma_commit(tc::smem_u32(&ctl->empty_a[buf]));
+                }
+                if (ok) tc::mma_commit(tc::smem_u32(&ctl->ready[0]));
+            } else {
+                for (int ks = 0; ks < ksteps && ok; ++ks) ok = tc::mbar_wait(tc::smem_u32(&ctl->full_a[ks]), 0u, abort_flag);
+                tc::fence_after();
+                for (int c = 0; c < pr.nn && ok; ++c) {
+                    const int tb = c % pr.nbuf;
+                    if (c >= pr.nbuf) {
+                        ok = tc::mbar_wait(tc::smem_u32(&ctl->tfree[tb]), (uint32_t)(c / pr.nbuf - 1) & 1u, abort_flag);
+                        if (!ok) break;
+                        tc::fence_after();
+                    }
+                    const int n0 = c * pr.nchunk, cur = min(pr.nchunk, pr.npad - n0);
+                    for (int ks = 0; ks < ksteps; ++ks) mma_kstep(ks, ks, n0, cur, tmem + (uint32_t)(tb * 8 * pr.nchunk), ks == 0);
+                    tc::mma_commit(tc::smem_u32(&ctl->ready[tb]));
+                }
+            }
+        }
+        __syncwarp();
+    } else {
+        // ---- phase 1: transform + quantize into the A operand ---------------------------------------------
+        int m = 0;                                     // boxes consumed so far
+        for (int ci = 0; ci < my_chunks && ok; ++ci) {
+            const int j = q + ci * WPT, ks = j >> 1, jj = j & 1, buf = ks % pr.na;
+            uint32_t packed[8][4];                     // per slot: 16 int8 codes or 8 bf16 values
+            if (live) {
+#pragma unroll
+                for (int g = 0; g < C::GROUPS; ++g) {
+                    const int bx = (g * 4) / C::CB, cin_box = (g * 4) % C::CB;
+                    const int stage = (m + bx) % C::S;
+                    if (cin_box == 0) {
+                        ok = ok && ring.wait(stage, (uint32_t)((m + bx) / C::S) & 1u);
+                    }
+                    float p[4][2][4], o[4][8];
+#pragma unroll
+                    for (int d = 0; d < 4; ++d) {
+                        RawPatch rawp;
+                        ring.read(stage, cin_box + d, rawp);           // channels beyond Cin arrive as zeros
+                        unpack_patch<T>(rawp, p[d]);
+                    }
+                    if (cin_box + 4 == C::CB) {                        // last read of this box: refill its stage
+                        __syncwarp();
+                        if (lane == 0 && m + bx + C::S < my_boxes) ring.issue(&tmx, stage, x0, y0, box_c0(m + bx + C::S), n);
+                    }
+                    haar_fwd_lanes<L, 4>(p, o, lane);
+                    uint32_t code[4][8];
+#pragma unroll
+                    for (int d = 0; d < 4; ++d) {
+#pragma unroll
+                        for (int s = 0; s < 8; s += 2) {
+                            float2 v = mul2(make_float2(o[d][s], o[d][s + 1]), make_float2(mul[s], mul[s + 1]));
+                            // int8: the low byte of (v + 1.5*2^23) is the two's complement code of rint(v).  Scalar adds on
+                            // purpose: a packed add right after the packed product would be contracted into one fused
+                            // operation, which rounds once and changes half-way codes.
+                            if (I8) v = make_float2(__fadd_rn(v.x, fz::MAGIC), __fadd_rn(v.y, fz::MAGIC));
+                            code[d][s] = __float_as_uint(v.x);
+                            code[d][s + 1] = __float_as_uint(v.y);
+                        }
+                    }
+#pragma unroll
+                    for (int s = 0; s < 8; ++s) {
+                        if (I8) {
+                            const uint32_t lo = __byte_perm(code[0][s], code[1][s], 0x0040);
+                            const uint32_t hi = __byte_perm(code[2][s], code[3][s], 0x0040);
+                            packed[s][g] = __byte_perm(lo, hi, 0x5410);
+                        } else {
+                            packed[s][2 * g] = pack_bf16x2(__uint_as_float(code[0][s]), __uint_as_float(code[1][s]));
+                            packed[s][2 * g + 1] = pack_bf16x2(__uint_as_float(code[2][s]), __uint_as_float(code[3][s]));
+                        }
+                    }
+                }
+                m += C::BPC;
+            }
+            if (ks >= pr.na) {                         // the tensor core must be done with the buffer's previous K step
+                ok = ok && tc::mbar_wait(tc::smem_u32(&ctl->empty_a[buf]), (uint32_t)(ks / pr.na - 1) & 1u, abort_flag);
+                tc::fence_after();
+            }
+            if (live) {
+#pragma unroll
+                for (int s = 0; s < 8; ++s) {
+                    uint8_t* dst = sA + (size_t)buf * KSTEP_BYTES + ((size_t)jj * ROWS + s * 128 + t * 32 + lane) * 16;
+                    *reinterpret_cast<uint4*>(dst) = make_uint4(packed[s][0], packed[s][1], packed[s][2], packed[s][3]);
+                    if (pr.xq_tap && rk[s] >= 0)
+                        *reinterpret_cast<uint4*>(pr.xq_tap + ((size_t)n * pr.k + rk[s]) * krow + (size_t)j * 16) =
+                            make_uint4(packed[s][0], packed[s][1], packed[s][2], packed[s][3]);
+                }
+            } else {
+#pragma unroll
+                for (int s = 0; s < 8; ++s)
+                    *reinterpret_cast<uint4*>(sA + (size_t)buf * KSTEP_BYTES + ((size_t)jj * ROWS + s * 128 + t * 32 + lane) * 16) =
+                        make_uint4(0u, 0u, 0u, 0u);
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(tc::smem_u32(&ctl->full_a[buf]));
+        }
+
+        // ---- phase 3: accumulators -> dequantize -> inverse transform -> y ---------------------------------
+        T* yout = static_cast<T*>(pr.y);
+        for (int c = 0; c < pr.nn && ok; ++c) {
+            const int tb = c % pr.nbuf;
+            ok = tc::mbar_wait(tc::smem_u32(&ctl->ready[tb]), (uint32_t)(c / pr.nbuf) & 1u, abort_flag);
+            ok = __all_sync(0xFFFFFFFFu, ok ? 1 : 0) != 0;
+            if (!ok) break;
+            tc::fence_after();
+            const int n0 = c * pr.nchunk, cur = min(pr.nchunk, pr.npad - n0);
+            for (int g = q; g * 8 < cur; g += WPT) {
+                const int o0 = n0 + g * 8;
+                if (!live || o0 >= pr.Cout) continue;
+                uint32_t r[8][8];                      // [slot][channel]
+                const uint32_t taddr = tmem + ((uint32_t)(t * 32) << 16) + (uint32_t)(tb * 8 * pr.nchunk + g * 8);
+#pragma unroll
+                for (int s = 0; s < 8; ++s) fz::tmem_ld8_nowait(taddr + (uint32_t)(s * pr.nchunk), r[s]);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (pr.acc_tap) {
+#pragma unroll
+                    for (int s = 0; s < 8; ++s) {
+                        if (rk[s] >= 0) {
+#pragma unroll
+                            for (int jn = 0; jn < 8; ++jn)
+                                if (o0 + jn < pr.Cout) pr.acc_tap[((size_t)n * pr.k + rk[s]) * pr.Cout + o0 + jn] = (int32_t)r[s][jn];
+                        }
+                    }
+                }
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    float sl[4][8], p[4][2][4];
+#pragma unroll
+                    for (int d = 0; d < 4; ++d) {
+                        const int o = o0 + hh * 4 + d;
+                        if (I8) {
+                            const float sc = (o < pr.Cout) ? __fmul_rn(scale_a, pr.scale_w[o]) : 0.0f;
+#pragma unroll
+                            for (int s = 0; s < 8; ++s)   // exact int -> float for |acc| < 2^22: bits(1.5*2^23) + acc, minus 1.5*2^23
+                                sl[d][s] = __fmul_rn(__fsub_rn(__uint_as_float(0x4B400000u + r[s][hh * 4 + d]), fz::MAGIC), sc);
+                        } else {
+#pragma unroll
+                            for (int s = 0; s < 8; ++s) sl[d][s] = __uint_as_float(r[s][hh * 4 + d]);
+                        }
+                    }
+                    haar_inv_lanes<L, 4>(sl, p, lane);
+#pragma unroll
+                    for (int d = 0; d < 4; ++d) {
+                        const int o = o0 + hh * 4 + d;
+                        if (o < pr.Cout) store_patch<T, true>(yout + ((size_t)n * pr.Cout + o) * P, pr.W, lp, p[d]);
+                    }
+                }
+            }
+            tc::fence_before();
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(tc::smem_u32(&ctl->tfree[tb]));
+        }
+    }
+
+    // ---- tear-down ------------------------------------------------------------------------------------
+    ok = __all_sync(0xFFFFFFFFu, ok ? 1 : 0) != 0;
+    if (!ok) {
+        *abort_flag = 1;
+        if (lane == 0) atomicExch(pr.status, (int)WCC_ERR_TIMEOUT);
+    }
+    tc::fence_before();
+    __syncthreads();
+    if (*abort_flag) {                                 // give copies that were already issued time to land
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (is_mma) {
+        tc::fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)pr.tmem_cols) : "memory");
+    }
+}
+
+}  // namespace ft
+
+// Returns WCC_ERR_SHAPE when this kernel does not cover the problem (the caller then uses fused_pass2_kernel).
+template <typename T, int L>
+static wcc_status fused_tiles_dispatch(const void* x, const void* Wq, const int32_t* rank, const float* nrm2, const uint32_t* thr,
+                                       const float* amax_kept, int bits, const float* scale_w, int N, int Cin, int Cout, int H,
+                                       int W, int k, int kpad, void* y, void* xq_tap, int32_t* acc_tap, cudaStream_t st)
+{
+    using TT = HaarTile<L>;
+    constexpr int WPT = 2;
+    const bool i8 = bits >= 2;
+    const int es = i8 ? 1 : 2;
+    if (!tc::tma_ok_x(x, (int)sizeof(T), W) || (kpad * es) % 32 != 0) return WCC_ERR_SHAPE;
+    ft::Params pr = {};
+    pr.npad = ceil_div(Cout, 16) * 16;
+    const int kchunks = kpad * es / 16, ksteps = kpad * es / 32;
+    if (pr.npad <= 64) { pr.nchunk = pr.npad; pr.nn = 1; pr.nbuf = 1; pr.na = ksteps < 2 ? ksteps : 2; }
+    else { pr.nchunk = 32; pr.nn = ceil_div(pr.npad, 32); pr.nbuf = 2; pr.na = ksteps; }
+    if (pr.na > ft::MAX_NA) return WCC_ERR_SHAPE;
+    pr.tmem_cols = 32;
+    while (pr.tmem_cols < 8 * pr.nchunk * pr.nbuf) pr.tmem_cols <<= 1;
+    if (pr.tmem_cols > 512) return WCC_ERR_SHAPE;
+    const size_t ring_bytes = (size_t)ft::TILES * WPT * (i8 ? ft::Cfg<T, true, WPT>::S : ft::Cfg<T, false, WPT>::S) * 4096;
+    const size_t smem = 128 + (size_t)pr.na * ft::KSTEP_BYTES + ring_bytes + (size_t)kchunks * pr.npad * 16 +
+                        (size_t)ft::TILES * WPT * 8 * 8 + sizeof(ft::Ctl) + 64;
+    if (smem > 227 * 1024) return WCC_ERR_SHAPE;
+    const long long tiles = (long long)N * ceil_div(W, TT::TW) * (H / TT::TH);
+    if (tiles > 0x7FFFFFFFLL) return WCC_ERR_SHAPE;
+    CUtensorMap tmx;
+    if (!tc::make_map_x(&tmx, x, (int)sizeof(T), N, Cin, H, W, TT::TW, TT::TH, (sizeof(T) == 2) ? 8 : 4)) return WCC_ERR_CUDA;
+    pr.Wq = static_cast<const uint8_t*>(Wq); pr.rank = rank; pr.nrm2 = nrm2; pr.thr = thr; pr.amax_kept = amax_kept;
+    pr.scale_w = scale_w; pr.qmax = i8 ? (float)((1 << (bits - 1)) - 1) : 1.0f;
+    pr.N = N; pr.Cin = Cin; pr.Cout = Cout; pr.H = H; pr.W = W; pr.k = k; pr.kpad = kpad; pr.tiles_total = (int)tiles;
+    pr.y = y; pr.xq_tap = static_cast<uint8_t*>(xq_tap); pr.acc_tap = acc_tap;
+    WCC_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&pr.status), g_status));
+    const unsigned ctas = (unsigned)((tiles + ft::TILES - 1) / ft::TILES);
+    auto launch = [&](auto kern, int threads) -> wcc_status {
+        WCC_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        kern<<<ctas, threads, smem, st>>>(tmx, pr);
+        WCC_LAUNCH_CHECK();
+        return WCC_OK;
+    };
+    if (i8) return launch(ft::fused_tiles_kernel<T, L, true, WPT>, ft::Cfg<T, true, WPT>::THREADS);
+    return launch(ft::fused_tiles_kernel<T, L, false, WPT>, ft::Cfg<T, false, WPT>::THREADS);
+}
+
+wcc_status launch_fused_tiles(const void* x, const void* Wq, const int32_t* rank, const float* nrm2, const uint32_t* thr,
+                              const float* amax_kept, int bits, const float* scale_w, int N, int Cin, int Cout, int H, int W,
+                              int L, int k, int kpad, wcc_dtype dt, void* y, void* xq_tap, int32_t* acc_tap, cudaStream_t st)
+{
+    if ((W % 4) != 0) return WCC_ERR_SHAPE;
+#define WCC_FT(TY, LL) return fused_tiles_dispatch<TY, LL>(x, Wq, rank, nrm2, thr, amax_kept, bits, scale_w, N, Cin, Cout, H, W, k, kpad, y, xq_tap, acc_tap, st)
+    if (dt == WCC_F32) { if (L == 1) WCC_FT(float, 1); if (L == 2) WCC_FT(float, 2); WCC_FT(float, 3); }
+    if (L == 1) WCC_FT(__nv_bfloat16, 1);
+    if (L == 2) WCC_FT(__nv_bfloat16, 2);
+    WCC_FT(__nv_bfloat16, 3);
+#undef WCC_FT
+}
+
+}  // namespace wcc

@@ -754,94 +754,106 @@ __device__ __noinline__ void tma_timeout(int* status)
     for (int i = 0; i < 2000; ++i) __nanosleep(1000);
 }
 
-// ---- first pass, eight warps per tile, TMA-fed -----------------------------------------------------
-// The work split of haar_norms_kernel (warps transform different channels of a round, hand the values over through
-// shared memory, four warps run the chains) with the inputs of a whole round arriving as one TMA box.
+// ---- first pass, one warp per tile, TMA-fed ----------------------------------------------------------
+// Every warp owns one tile and walks all channels itself, so the per-position chains of fused multiply-adds stay in
+// its registers (ascending channel order, no hand-off between warps, no block-wide barrier).  Memory parallelism
+// comes from the warp's own ring of TMA boxes (S stages of CB channels in flight), not from the number of warps.
 template <typename T, int L>
-struct NormsTmaCfg {
-    static constexpr int LU = (sizeof(T) == 2) ? 2 : 1;
-    static constexpr int RC = NORMS_WARPS * LU;                   // channels per round = per box
-    using Ring = TileRing<T, L, RC, 4>;                           // 4 x 8 KB
-    static constexpr size_t SMEM = 128 + Ring::BYTES + Ring::S * 8 + (size_t)RC * 4 * 32 * sizeof(float2);
+struct NormsWarpCfg {
+    static constexpr int WARPS = 2;                               // independent warps per CTA
+    static constexpr int CB = (sizeof(T) == 2) ? 8 : 4;           // channels per box: 4 KB
+    static constexpr int S = 6;                                   // boxes in flight per warp: 24 KB
+    using Ring = TileRing<T, L, CB, S>;
+    static constexpr size_t SMEM = 128 + (size_t)WARPS * (Ring::BYTES + S * 8);
 };
 
 template <typename T, int L>
-__global__ void __launch_bounds__(NORMS_WARPS * 32)
-haar_norms_tma_kernel(const __grid_constant__ CUtensorMap tmx, int N, int C, int H, int W,
+__global__ void __launch_bounds__(NormsWarpCfg<T, L>::WARPS * 32)
+haar_norms_warp_kernel(const __grid_constant__ CUtensorMap tmx, int N, int C, int H, int W, int tiles_total, int tile_ctas,
                        float* __restrict__ nrm2, float* __restrict__ amaxpos, const NormsExtra ex, int* __restrict__ status)
 {
-    if ((int)blockIdx.x >= ex.tiles) {                 // weight preparation CTAs
-        const int o = ((int)blockIdx.x - ex.tiles) * NORMS_WARPS + (int)(threadIdx.x >> 5);
+    using TT = HaarTile<L>;
+    using Cfg = NormsWarpCfg<T, L>;
+    using Ring = typename Cfg::Ring;
+    constexpr int CB = Cfg::CB, S = Cfg::S, U = 4;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if ((int)blockIdx.x >= tile_ctas) {                // weight preparation CTAs
+        const int o = ((int)blockIdx.x - tile_ctas) * Cfg::WARPS + warp;
         if (o < ex.Cout) weight_prep_row(ex.Wt, o, C, ex.kpad, ex.bits, ex.Wq, ex.scale_w);
         return;
     }
-    using TT = HaarTile<L>;
-    using Cfg = NormsTmaCfg<T, L>;
-    using Ring = typename Cfg::Ring;
-    constexpr int LU = Cfg::LU, RC = Cfg::RC, S = Ring::S;
+    const int tile = (int)blockIdx.x * Cfg::WARPS + warp;
+    if (tile >= tiles_total) return;                   // warps never meet at a block-wide barrier
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_s = tc::smem_u32(smem_raw);
     uint8_t* sm = smem_raw + (((raw_s + 127u) & ~127u) - raw_s);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sm + Ring::BYTES);
-    float2 (*buf)[4][32] = reinterpret_cast<float2 (*)[4][32]>(sm + Ring::BYTES + S * 8);   // [channel of the round][slot pair][lane]
+    uint8_t* stages = sm + (size_t)warp * Ring::BYTES;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sm + (size_t)Cfg::WARPS * Ring::BYTES) + warp * S;
 
     const int tiles_x = (W + TT::TW - 1) / TT::TW, tiles_y = H / TT::TH;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int n, ty, tx;
-    tile_coords(blockIdx.x, tiles_x, tiles_y, n, ty, tx);
+    tile_coords(tile, tiles_x, tiles_y, n, ty, tx);
     const LanePos lp = lane_positions<L>(H, W, ty, tx, lane);
     const size_t P = (size_t)H * W;
     const int x0 = tx * TT::TW, y0 = ty * TT::TH;
 
     Ring ring;
-    ring.init(sm, bars, threadIdx.x == 0 ? 0 : 1);     // thread 0 initializes the barriers
-    __syncthreads();
-    const int rounds = (C + RC - 1) / RC;
-    if (threadIdx.x == 0) {
+    ring.init(stages, bars, lane);
+    const int rounds = (C + CB - 1) / CB;
+    if (lane == 0) {
 #pragma unroll
         for (int i = 0; i < S; ++i)
-            if (i < rounds) ring.issue(&tmx, i, x0, y0, i * RC, n);
+            if (i < rounds) ring.issue(&tmx, i, x0, y0, i * CB, n);
     }
-    // lane geometry of the ring reads (init() computed them for lane 0 / 1 only)
-    ring.set_lane(lane);
-
-    float2 nn = make_float2(0.0f, 0.0f);
-    float a0 = 0.0f, a1 = 0.0f;
+    float nacc[8], amax[8];
+#pragma unroll
+    for (int s = 0; s < 8; ++s) { nacc[s] = 0.0f; amax[s] = 0.0f; }
     bool ok = true;
     for (int r = 0; r < rounds; ++r) {
         const int stage = r % S;
-        if (ok) ok = ring.wait(stage, (uint32_t)(r / S) & 1u);   // after a timeout: no more waits, same barrier count
-        float p[LU][2][4], o[LU][8];
+        if (ok) ok = ring.wait(stage, (uint32_t)(r / S) & 1u);
 #pragma unroll
-        for (int d = 0; d < LU; ++d) {
-            RawPatch raw;
-            ring.read(stage, warp * LU + d, raw);      // channels beyond C arrive as zeros
-            unpack_patch<T>(raw, p[d]);
-        }
-        haar_fwd_lanes<L, LU>(p, o, lane);
+        for (int g = 0; g < CB / U; ++g) {
+            float p[U][2][4], o[U][8];
 #pragma unroll
-        for (int d = 0; d < LU; ++d) {
-            const int c = r * RC + warp * LU + d;
+            for (int d = 0; d < U; ++d) {
+                RawPatch raw;
+                ring.read(stage, g * U + d, raw);      // channels beyond C arrive as zeros: fma(0, 0, acc) = acc
+                unpack_patch<T>(raw, p[d]);
+            }
+            haar_fwd_lanes<L, U>(p, o, lane);
 #pragma unroll
-            for (int s = 0; s < 8; s += 2) buf[warp * LU + d][s >> 1][lane] = make_float2(o[d][s], o[d][s + 1]);
-            if (ex.coef && c < C) store_slots<L, true>(ex.coef + ((size_t)n * C + c) * P, lp, o[d]);
-        }
-        __syncthreads();                               // values handed over; every warp is done reading the stage
-        if (threadIdx.x == 0 && r + S < rounds) ring.issue(&tmx, stage, x0, y0, (r + S) * RC, n);
-        if (warp < 4) {
+            for (int d = 0; d < U; ++d) {
+                const int c = r * CB + g * U + d;
+                if (ex.coef && c < C) store_slots<L, true>(ex.coef + ((size_t)n * C + c) * P, lp, o[d]);
 #pragma unroll
-            for (int c = 0; c < RC; ++c) {
-                const float2 v = buf[c][warp][lane];
-                nn = __ffma2_rn(v, v, nn);
-                a0 = fmaxf(a0, fabsf(v.x));
-                a1 = fmaxf(a1, fabsf(v.y));
+                for (int s = 0; s < 8; s += 2) {
+                    const float2 v = make_float2(o[d][s], o[d][s + 1]);
+                    const float2 a = __ffma2_rn(v, v, make_float2(nacc[s], nacc[s + 1]));
+                    nacc[s] = a.x; nacc[s + 1] = a.y;
+                    amax[s] = fmaxf(amax[s], fabsf(v.x));
+                    amax[s + 1] = fmaxf(amax[s + 1], fabsf(v.y));
+                }
             }
         }
-        __syncthreads();
+        __syncwarp();                                  // every lane is done reading the stage
+        if (lane == 0 && r + S < rounds) ring.issue(&tmx, stage, x0, y0, (r + S) * CB, n);
     }
-    if (!__syncthreads_and(ok ? 1 : 0)) { tma_timeout(status); return; }
-    if (warp >= 4) return;
-    norms_finish<L, true>(lp, warp, n, P, nn.x, nn.y, a0, a1, nrm2, amaxpos, ex);
+    if (!__all_sync(0xFFFFFFFFu, ok ? 1 : 0)) { tma_timeout(status); return; }
+    store_slots<L, true>(nrm2 + (size_t)n * P, lp, nacc);
+    if (amaxpos) store_slots<L, true>(amaxpos + (size_t)n * P, lp, amax);
+    if (ex.hist1) {                                    // norms are >= +0: key = bits | sign bit, digit = top 11 bits
+        uint32_t* h = ex.hist1 + (size_t)n * 3 * 2048;
+#pragma unroll
+        for (int s = 0; s < 8; ++s) hist_add(h, float_key(nacc[s]) >> 21, lp.ok0);
+    }
+    if (ex.fine) {                                     // 16-bit digits are spread out: plain atomics
+        uint32_t* f = ex.fine + (size_t)n * 65536;
+        if (lp.ok0) {
+#pragma unroll
+            for (int s = 0; s < 8; ++s) atomicAdd(&f[float_key(nacc[s]) >> 16], 1u);
+        }
+    }
 }
 
 // ---- plain inverse -------------------------------------------------------------------------------
@@ -962,15 +974,18 @@ static wcc_status haar_norms_dispatch(const void* x, int N, int C, int H, int W,
     using TT = HaarTile<L>;
     const long long tiles = (long long)N * ceil_div(W, TT::TW) * (H / TT::TH);
     if (VEC && tc::tma_ok_x(x, (int)sizeof(T), W)) {
-        using Cfg = NormsTmaCfg<T, L>;
+        using Cfg = NormsWarpCfg<T, L>;
         CUtensorMap tmx;
-        if (!tc::make_map_x(&tmx, x, (int)sizeof(T), N, C, H, W, TT::TW, TT::TH, Cfg::RC)) return WCC_ERR_CUDA;
+        if (!tc::make_map_x(&tmx, x, (int)sizeof(T), N, C, H, W, TT::TW, TT::TH, Cfg::CB)) return WCC_ERR_CUDA;
         int* status = nullptr;
         WCC_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_status));
-        WCC_CUDA_TRY(cudaFuncSetAttribute(haar_norms_tma_kernel<T, L>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM));
+        WCC_CUDA_TRY(cudaFuncSetAttribute(haar_norms_warp_kernel<T, L>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM));
+        const long long tile_ctas = (tiles + Cfg::WARPS - 1) / Cfg::WARPS;
+        const long long grid = tile_ctas + (ex.Wt ? ceil_div(ex.Cout, Cfg::WARPS) : 0);
+        if (grid > 0x7FFFFFFFLL) return WCC_ERR_SHAPE;
         ex.tiles = (int)tiles;
-        const long long grid = tiles + (ex.Wt ? ceil_div(ex.Cout, NORMS_WARPS) : 0);
-        haar_norms_tma_kernel<T, L><<<(unsigned)grid, NORMS_WARPS * 32, Cfg::SMEM, st>>>(tmx, N, C, H, W, nrm2, amaxpos, ex, status);
+        haar_norms_warp_kernel<T, L><<<(unsigned)grid, Cfg::WARPS * 32, Cfg::SMEM, st>>>(tmx, N, C, H, W, (int)tiles, (int)tile_ctas,
+                                                                                        nrm2, amaxpos, ex, status);
         WCC_LAUNCH_CHECK();
         return WCC_OK;
     }

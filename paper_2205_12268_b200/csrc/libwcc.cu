@@ -5,6 +5,7 @@
 #include "select.cuh"
 #include "contract.cuh"
 #include "fused.cuh"
+#include "fused_tiles.cuh"
 
 namespace wcc {
 
@@ -232,8 +233,11 @@ static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, i
     if ((s = profile_mark(2, st)) != WCC_OK) return s;
     // second pass over x: transform, mask + quantize, tensor-core contraction, dequantize, inverse, store
     void* xq_tap = taps ? (bits >= 2 ? static_cast<void*>(taps->Xq) : taps->Xb) : nullptr;
-    s = launch_fused_pass2(x, f.Wq, f.rank, f.nrm2, f.thr, f.amax_kept, bits, f.scale_w, N, Cin, Cout, H, W, L, k, f.kpad, dt, y,
+    s = launch_fused_tiles(x, f.Wq, f.rank, f.nrm2, f.thr, f.amax_kept, bits, f.scale_w, N, Cin, Cout, H, W, L, k, f.kpad, dt, y,
                            xq_tap, taps ? taps->acc : nullptr, st);
+    if (s == WCC_ERR_SHAPE)                            // shapes the four-tile kernel does not cover (nothing was launched)
+        s = launch_fused_pass2(x, f.Wq, f.rank, f.nrm2, f.thr, f.amax_kept, bits, f.scale_w, N, Cin, Cout, H, W, L, k, f.kpad, dt, y,
+                               xq_tap, taps ? taps->acc : nullptr, st);
     if (s != WCC_OK) return s;
     for (int i = 3; i <= WCC_NUM_STAGES; ++i)
         if ((s = profile_mark(i, st)) != WCC_OK) return s;
