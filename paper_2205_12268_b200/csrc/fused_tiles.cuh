@@ -78,6 +78,7 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
     uint8_t* sB = sRing + (size_t)C::CWARPS * Ring::BYTES;                    // [kchunks][npad][16]
     uint64_t* ring_bars = reinterpret_cast<uint64_t*>(sB + (size_t)kchunks * pr.npad * 16);   // [CWARPS][S]
     Ctl* ctl = reinterpret_cast<Ctl*>(ring_bars + C::CWARPS * C::S);
+    float* sscale = reinterpret_cast<float*>(ctl + 1);                        // [npad]
     volatile int* abort_flag = &ctl->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -130,23 +131,34 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
     int rk[8];
 #pragma unroll
     for (int s = 0; s < 8; ++s) { mul[s] = 0.0f; rk[s] = -1; }
-    float scale_a = 1.0f;
+    // all independent loads first (threshold, norms, max |kept|), so that their latencies overlap
+    float amax = 0.0f;
+    if (I8) amax = *pr.amax_kept;
     if (live) {
+        const uint4 th = *reinterpret_cast<const uint4*>(pr.thr + n * 4);      // {threshold key, ties kept, use-rank flag, -}
+        float nv[8];
+#pragma unroll
+        for (int s = 0; s < 8; ++s) nv[s] = slot_ok<L>(lp, s) ? pr.nrm2[(size_t)n * P + lp.pos[s]] : 0.0f;
         float inv = 1.0f;
-        if (I8) {
-            const float amax = *pr.amax_kept;
-            inv = (amax > 0.0f) ? __fdiv_rn(pr.qmax, amax) : 0.0f;
-            scale_a = __fdiv_rn(amax, pr.qmax);
-        }
-        const uint32_t tkey = pr.thr[n * 4], use_rank = pr.thr[n * 4 + 2];
+        if (I8) inv = (amax > 0.0f) ? __fdiv_rn(pr.qmax, amax) : 0.0f;
+        const uint32_t tkey = th.x, use_rank = th.z;
 #pragma unroll
         for (int s = 0; s < 8; ++s) {
             if (slot_ok<L>(lp, s)) {
                 if (use_rank) rk[s] = pr.rank[(size_t)n * P + lp.pos[s]];
-                else rk[s] = (float_key(pr.nrm2[(size_t)n * P + lp.pos[s]]) >= tkey) ? 0 : -1;
+                else rk[s] = (float_key(nv[s]) >= tkey) ? 0 : -1;
             }
             mul[s] = (rk[s] >= 0) ? inv : 0.0f;
         }
+        // the transform runs without its halvings: they go into the per-slot factor (exact, a power of two)
+        float sc[8];
+        slot_scales<L>(lane, ring.swap, sc);
+#pragma unroll
+        for (int s = 0; s < 8; ++s) mul[s] = __fmul_rn(mul[s], sc[s]);
+    }
+    if (I8) {                                          // dequantization factor of every output channel
+        const float scale_a = __fdiv_rn(amax, pr.qmax);
+        for (int o = threadIdx.x; o < pr.npad; o += C::THREADS) sscale[o] = (o < pr.Cout) ? __fmul_rn(scale_a, pr.scale_w[o]) : 0.0f;
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");       // B operand -> visible to the tensor core
     tc::fence_before();
@@ -215,24 +227,24 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
 #pragma unroll
                     for (int d = 0; d < 4; ++d) {
                         RawPatch rawp;
-                        ring.read(stage, cin_box + d, rawp);           // channels beyond Cin arrive as zeros
+                        ring.read_raw(stage, cin_box + d, rawp);       // channels beyond Cin arrive as zeros
                         unpack_patch<T>(rawp, p[d]);
                     }
                     if (cin_box + 4 == C::CB) {                        // last read of this box: refill its stage
                         __syncwarp();
                         if (lane == 0 && m + bx + C::S < my_boxes) ring.issue(&tmx, stage, x0, y0, box_c0(m + bx + C::S), n);
                     }
-                    haar_fwd_lanes<L, 4>(p, o, lane);
+                    haar_fwd_lanes_raw<L, 4>(p, o, lane);
                     uint32_t code[4][8];
 #pragma unroll
                     for (int d = 0; d < 4; ++d) {
 #pragma unroll
                         for (int s = 0; s < 8; s += 2) {
                             float2 v = mul2(make_float2(o[d][s], o[d][s + 1]), make_float2(mul[s], mul[s + 1]));
-                            // int8: the low byte of (v + 1.5*2^23) is the two's complement code of rint(v).  Scalar adds on
-                            // purpose: a packed add right after the packed product would be contracted into one fused
-                            // operation, which rounds once and changes half-way codes.
-                            if (I8) v = make_float2(__fadd_rn(v.x, fz::MAGIC), __fadd_rn(v.y, fz::MAGIC));
+                            // int8: the low byte of (v + 1.5*2^23) is the two's complement code of rint(v).  The sum is
+                            // written as fma(v, 1, 1.5*2^23): the product above keeps its own rounding (a packed add right
+                            // after the packed product gets contracted into one fused operation, which changes half-way codes).
+                            if (I8) v = __ffma2_rn(v, make_float2(1.0f, 1.0f), make_float2(fz::MAGIC, fz::MAGIC));
                             code[d][s] = __float_as_uint(v.x);
                             code[d][s + 1] = __float_as_uint(v.y);
                         }
@@ -277,6 +289,7 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
 
         // ---- phase 3: accumulators -> dequantize -> inverse transform -> y ---------------------------------
         T* yout = static_cast<T*>(pr.y);
+        const bool coarse6 = L == 3 && ((lane / TT::CG) & 1) == 0;     // slot 6 holds a level-3 coefficient
         for (int c = 0; c < pr.nn && ok; ++c) {
             const int tb = c % pr.nbuf;
             ok = tc::mbar_wait(tc::smem_u32(&ctl->ready[tb]), (uint32_t)(c / pr.nbuf) & 1u, abort_flag);
@@ -308,17 +321,18 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
 #pragma unroll
                     for (int d = 0; d < 4; ++d) {
                         const int o = o0 + hh * 4 + d;
-                        if (I8) {
-                            const float sc = (o < pr.Cout) ? __fmul_rn(scale_a, pr.scale_w[o]) : 0.0f;
+                        // dequantize straight into the pre-scaled slots of haar_inv_lanes_raw: acc * (scale * 2^-level)
+                        float sc = 1.0f;
+                        if (I8) sc = sscale[o];
+                        const float s1 = __fmul_rn(sc, 0.5f), s2 = __fmul_rn(sc, 0.25f);
+                        const float s6 = (L == 1) ? s1 : (coarse6 ? __fmul_rn(sc, 0.125f) : s2), s7 = (L == 1) ? s1 : s2;
 #pragma unroll
-                            for (int s = 0; s < 8; ++s)   // exact int -> float for |acc| < 2^22: bits(1.5*2^23) + acc, minus 1.5*2^23
-                                sl[d][s] = __fmul_rn(__fsub_rn(__uint_as_float(0x4B400000u + r[s][hh * 4 + d]), fz::MAGIC), sc);
-                        } else {
-#pragma unroll
-                            for (int s = 0; s < 8; ++s) sl[d][s] = __uint_as_float(r[s][hh * 4 + d]);
+                        for (int s = 0; s < 8; ++s) {
+                            const float f = I8 ? __int2float_rn((int)r[s][hh * 4 + d]) : __uint_as_float(r[s][hh * 4 + d]);
+                            sl[d][s] = __fmul_rn(f, s < 6 ? s1 : (s == 6 ? s6 : s7));
                         }
                     }
-                    haar_inv_lanes<L, 4>(sl, p, lane);
+                    haar_inv_lanes_raw<L, 4>(sl, p, lane);
 #pragma unroll
                     for (int d = 0; d < 4; ++d) {
                         const int o = o0 + hh * 4 + d;
@@ -374,7 +388,7 @@ static wcc_status fused_tiles_dispatch(const void* x, const void* Wq, const int3
     if (pr.tmem_cols > 512) return WCC_ERR_SHAPE;
     const size_t ring_bytes = (size_t)ft::TILES * WPT * (i8 ? ft::Cfg<T, true, WPT>::S : ft::Cfg<T, false, WPT>::S) * 4096;
     const size_t smem = 128 + (size_t)pr.na * ft::KSTEP_BYTES + ring_bytes + (size_t)kchunks * pr.npad * 16 +
-                        (size_t)ft::TILES * WPT * 8 * 8 + sizeof(ft::Ctl) + 64;
+                        (size_t)ft::TILES * WPT * 8 * 8 + sizeof(ft::Ctl) + (size_t)pr.npad * 4 + 64;
     if (smem > 227 * 1024) return WCC_ERR_SHAPE;
     const long long tiles = (long long)N * ceil_div(W, TT::TW) * (H / TT::TH);
     if (tiles > 0x7FFFFFFFLL) return WCC_ERR_SHAPE;

@@ -298,6 +298,133 @@ __device__ __forceinline__ void haar_inv_lanes(const float (&o)[U][8], float (&p
     }
 }
 
+// ---- transforms with the halvings taken out ------------------------------------------------------------
+// Multiplying by a power of two commutes with every rounding (barring overflow and subnormal results), so the forward
+// transform can run on sums and differences alone and leave one exact multiplication per slot to the consumer:
+// true coefficient of slot s = raw value * slot_scale[s], where |slot_scale| = 2^-level.  The same holds for squares
+// (norm = raw norm * scale^2) and maxima.  Results are bit-identical to haar_fwd_lanes for inputs whose partial sums stay
+// below 2^125 and above the subnormal range.
+// `swapped`: the lane passes its two patch rows in exchanged order (a shared-memory bank trick of the TMA rings); the sums
+// over rows are unchanged and the differences over rows (y3, y4 of level 1) change sign, which goes into the scale.
+template <int L>
+__device__ __forceinline__ void slot_scales(int lane, bool swapped, float (&sc)[8])
+{
+    using T = HaarTile<L>;
+    const int rp = lane / T::CG;
+    const float h = 0.5f, hs = swapped ? -0.5f : 0.5f;
+    sc[0] = h; sc[1] = h; sc[2] = hs; sc[3] = hs; sc[4] = hs; sc[5] = hs;
+    if (L == 1) { sc[6] = h; sc[7] = h; }
+    else {
+        sc[7] = 0.25f;
+        sc[6] = (L == 3 && (rp & 1) == 0) ? 0.125f : 0.25f;
+    }
+}
+
+template <int L, int U>
+__device__ __forceinline__ void haar_fwd_lanes_raw(const float (&p)[U][2][4], float (&o)[U][8], int lane)
+{
+    using T = HaarTile<L>;
+    float2 ll[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const float2 a = make_float2(p[u][0][0], p[u][0][2]), b = make_float2(p[u][0][1], p[u][0][3]);
+        const float2 c = make_float2(p[u][1][0], p[u][1][2]), d = make_float2(p[u][1][1], p[u][1][3]);
+        const float2 s0 = add2(a, b), d0 = sub2(a, b), s1 = add2(c, d), d1 = sub2(c, d);
+        ll[u] = add2(s0, s1);
+        const float2 y2 = add2(d0, d1), y3 = sub2(s0, s1), y4 = sub2(d0, d1);
+        o[u][0] = y2.x; o[u][1] = y2.y; o[u][2] = y3.x; o[u][3] = y3.y; o[u][4] = y4.x; o[u][5] = y4.y;
+        if (L == 1) { o[u][6] = ll[u].x; o[u][7] = ll[u].y; }
+    }
+    if (L == 1) return;
+    const int rp = lane / T::CG, cg = lane % T::CG;
+    const bool even = (rp & 1) == 0;
+    const float sg = even ? 1.0f : -1.0f;
+    float s[U], dd[U], ps[U], pd[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) { s[u] = __fadd_rn(ll[u].x, ll[u].y); dd[u] = __fsub_rn(ll[u].x, ll[u].y); }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        ps[u] = __shfl_xor_sync(0xFFFFFFFFu, s[u], T::CG);
+        pd[u] = __shfl_xor_sync(0xFFFFFFFFu, dd[u], T::CG);
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const float2 l2 = __ffma2_rn(make_float2(s[u], dd[u]), make_float2(sg, sg), make_float2(ps[u], pd[u]));
+        o[u][6] = l2.x;
+        o[u][7] = l2.y;
+    }
+    if (L == 3) {
+        const float sgh = (cg & 1) == 0 ? 1.0f : -1.0f;
+        const float sgv = (rp & 2) == 0 ? 1.0f : -1.0f;
+        float h[U], t[U], q[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) h[u] = __shfl_xor_sync(0xFFFFFFFFu, o[u][6], 1);
+#pragma unroll
+        for (int u = 0; u < U; ++u) t[u] = __fmaf_rn(o[u][6], sgh, h[u]);
+#pragma unroll
+        for (int u = 0; u < U; ++u) q[u] = __shfl_xor_sync(0xFFFFFFFFu, t[u], 2 * T::CG);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const float r = __fmaf_rn(t[u], sgv, q[u]);
+            if (even) o[u][6] = r;
+        }
+    }
+}
+
+// Inverse on slots that the caller has already multiplied by slot_scales (not swapped): sums and differences only.
+template <int L, int U>
+__device__ __forceinline__ void haar_inv_lanes_raw(const float (&o)[U][8], float (&p)[U][2][4], int lane)
+{
+    using T = HaarTile<L>;
+    float2 ll[U];
+    if (L == 1) {
+#pragma unroll
+        for (int u = 0; u < U; ++u) ll[u] = make_float2(o[u][6], o[u][7]);
+    } else {
+        const int rp = lane / T::CG, cg = lane % T::CG;
+        const float sg = (rp & 1) == 0 ? 1.0f : -1.0f;
+        float m0[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) m0[u] = o[u][6];
+        if (L == 3) {
+            const float sgh = (cg & 1) == 0 ? 1.0f : -1.0f;
+            const float sgv = (rp & 2) == 0 ? 1.0f : -1.0f;
+            float pv[U], w[U], q[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) pv[u] = __shfl_xor_sync(0xFFFFFFFFu, m0[u], 2 * T::CG);
+#pragma unroll
+            for (int u = 0; u < U; ++u) w[u] = __fmaf_rn(m0[u], sgv, pv[u]);
+#pragma unroll
+            for (int u = 0; u < U; ++u) q[u] = __shfl_xor_sync(0xFFFFFFFFu, w[u], 1);
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const float r = __fmaf_rn(w[u], sgh, q[u]);
+                if ((rp & 1) == 0) m0[u] = r;
+            }
+        }
+        float p0[U], p1[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            p0[u] = __shfl_xor_sync(0xFFFFFFFFu, m0[u], T::CG);
+            p1[u] = __shfl_xor_sync(0xFFFFFFFFu, o[u][7], T::CG);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const float2 tu = __ffma2_rn(make_float2(m0[u], o[u][7]), make_float2(sg, sg), make_float2(p0[u], p1[u]));
+            ll[u] = make_float2(__fadd_rn(tu.x, tu.y), __fsub_rn(tu.x, tu.y));
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const float2 y2 = make_float2(o[u][0], o[u][1]), y3 = make_float2(o[u][2], o[u][3]), y4 = make_float2(o[u][4], o[u][5]);
+        const float2 t0 = add2(ll[u], y3), t1 = sub2(ll[u], y3), u0 = add2(y2, y4), u1 = sub2(y2, y4);
+        const float2 a = add2(t0, u0), b = sub2(t0, u0);
+        const float2 c = add2(t1, u1), d = sub2(t1, u1);
+        p[u][0][0] = a.x; p[u][0][1] = b.x; p[u][0][2] = a.y; p[u][0][3] = b.y;
+        p[u][1][0] = c.x; p[u][1][1] = d.x; p[u][1][2] = c.y; p[u][1][3] = d.y;
+    }
+}
+
 // ---- patch load / store ------------------------------------------------------------------------
 struct RawPatch { uint32_t w[8]; };   // fp32: 2 rows x 4 words; bf16: 2 rows x 2 words (w[0..1], w[4..5])
 
@@ -729,6 +856,21 @@ struct TileRing {
     }
     __device__ __forceinline__ bool wait(int stage, uint32_t parity) const { return tc::mbar_wait(bar_s + 8 * stage, parity); }
 
+    // rows in the order they were read: for lanes with `swap` set the patch's second row comes first
+    __device__ __forceinline__ void read_raw(int stage, int d, RawPatch& raw) const
+    {
+        const uint8_t* ch = ring + stage * STAGE_BYTES + d * CH_BYTES;
+        if (sizeof(T) == 4) {
+            const uint4 a = *reinterpret_cast<const uint4*>(ch + off_a);
+            const uint4 b = *reinterpret_cast<const uint4*>(ch + off_b);
+            raw.w[0] = a.x; raw.w[1] = a.y; raw.w[2] = a.z; raw.w[3] = a.w;
+            raw.w[4] = b.x; raw.w[5] = b.y; raw.w[6] = b.z; raw.w[7] = b.w;
+        } else {
+            const uint2 a = *reinterpret_cast<const uint2*>(ch + off_a);
+            const uint2 b = *reinterpret_cast<const uint2*>(ch + off_b);
+            raw.w[0] = a.x; raw.w[1] = a.y; raw.w[4] = b.x; raw.w[5] = b.y;
+        }
+    }
     __device__ __forceinline__ void read(int stage, int d, RawPatch& raw) const
     {
         const uint8_t* ch = ring + stage * STAGE_BYTES + d * CH_BYTES;
@@ -805,6 +947,9 @@ haar_norms_warp_kernel(const __grid_constant__ CUtensorMap tmx, int N, int C, in
         for (int i = 0; i < S; ++i)
             if (i < rounds) ring.issue(&tmx, i, x0, y0, i * CB, n);
     }
+    // the transform runs without its halvings (haar_fwd_lanes_raw); one exact multiplication per slot at the end
+    float sc[8];
+    slot_scales<L>(lane, ring.swap, sc);
     float nacc[8], amax[8];
 #pragma unroll
     for (int s = 0; s < 8; ++s) { nacc[s] = 0.0f; amax[s] = 0.0f; }
@@ -818,14 +963,21 @@ haar_norms_warp_kernel(const __grid_constant__ CUtensorMap tmx, int N, int C, in
 #pragma unroll
             for (int d = 0; d < U; ++d) {
                 RawPatch raw;
-                ring.read(stage, g * U + d, raw);      // channels beyond C arrive as zeros: fma(0, 0, acc) = acc
+                ring.read_raw(stage, g * U + d, raw);  // channels beyond C arrive as zeros: fma(0, 0, acc) = acc
                 unpack_patch<T>(raw, p[d]);
             }
-            haar_fwd_lanes<L, U>(p, o, lane);
+            haar_fwd_lanes_raw<L, U>(p, o, lane);
 #pragma unroll
             for (int d = 0; d < U; ++d) {
                 const int c = r * CB + g * U + d;
-                if (ex.coef && c < C) store_slots<L, true>(ex.coef + ((size_t)n * C + c) * P, lp, o[d]);
+                if (ex.coef && c < C) {                // test tap: the plain transform (also gets the signs of zeros right)
+                    RawPatch raw;
+                    float pp[2][4], oc[8];
+                    ring.read(stage, g * U + d, raw);
+                    unpack_patch<T>(raw, pp);
+                    haar_fwd_lane<L>(pp, oc, lane);
+                    store_slots<L, true>(ex.coef + ((size_t)n * C + c) * P, lp, oc);
+                }
 #pragma unroll
                 for (int s = 0; s < 8; s += 2) {
                     const float2 v = make_float2(o[d][s], o[d][s + 1]);
@@ -840,6 +992,11 @@ haar_norms_warp_kernel(const __grid_constant__ CUtensorMap tmx, int N, int C, in
         if (lane == 0 && r + S < rounds) ring.issue(&tmx, stage, x0, y0, (r + S) * CB, n);
     }
     if (!__all_sync(0xFFFFFFFFu, ok ? 1 : 0)) { tma_timeout(status); return; }
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+        nacc[s] = __fmul_rn(nacc[s], __fmul_rn(sc[s], sc[s]));
+        amax[s] = __fmul_rn(amax[s], fabsf(sc[s]));
+    }
     store_slots<L, true>(nrm2 + (size_t)n * P, lp, nacc);
     if (amaxpos) store_slots<L, true>(amaxpos + (size_t)n * P, lp, amax);
     if (ex.hist1) {                                    // norms are >= +0: key = bits | sign bit, digit = top 11 bits
