@@ -216,48 +216,56 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
             const int j = q + ci * WPT, ks = j >> 1, jj = j & 1, buf = ks % pr.na;
             uint32_t packed[8][4];                     // per slot: 16 int8 codes or 8 bf16 values
             if (live) {
+                // all of the chunk's input words first (one wait per box), refill the stages right away, then compute:
+                // the groups of four channels below carry no barrier between them and overlap freely
+                constexpr int HB = (sizeof(T) == 2) ? C::CCH : ((C::CCH < 8) ? C::CCH : 8);   // channels loaded ahead (<= 64 registers)
 #pragma unroll
-                for (int g = 0; g < C::GROUPS; ++g) {
-                    const int bx = (g * 4) / C::CB, cin_box = (g * 4) % C::CB;
-                    const int stage = (m + bx) % C::S;
-                    if (cin_box == 0) {
+                for (int hb = 0; hb < C::CCH / HB; ++hb) {
+                    RawPatch rawp[HB];
+#pragma unroll
+                    for (int bx = hb * (HB / C::CB); bx < (hb + 1) * (HB / C::CB); ++bx) {
+                        const int stage = (m + bx) % C::S;
                         ok = ok && ring.wait(stage, (uint32_t)((m + bx) / C::S) & 1u);
-                    }
-                    float p[4][2][4], o[4][8];
 #pragma unroll
-                    for (int d = 0; d < 4; ++d) {
-                        RawPatch rawp;
-                        ring.read_raw(stage, cin_box + d, rawp);       // channels beyond Cin arrive as zeros
-                        unpack_patch<T>(rawp, p[d]);
+                        for (int d = 0; d < C::CB; ++d) ring.read_raw(stage, d, rawp[bx * C::CB + d - hb * HB]);   // channels beyond Cin arrive as zeros
                     }
-                    if (cin_box + 4 == C::CB) {                        // last read of this box: refill its stage
-                        __syncwarp();
-                        if (lane == 0 && m + bx + C::S < my_boxes) ring.issue(&tmx, stage, x0, y0, box_c0(m + bx + C::S), n);
+                    __syncwarp();
+                    if (lane == 0) {
+#pragma unroll
+                        for (int bx = hb * (HB / C::CB); bx < (hb + 1) * (HB / C::CB); ++bx)
+                            if (m + bx + C::S < my_boxes) ring.issue(&tmx, (m + bx) % C::S, x0, y0, box_c0(m + bx + C::S), n);
                     }
-                    haar_fwd_lanes_raw<L, 4>(p, o, lane);
-                    uint32_t code[4][8];
 #pragma unroll
-                    for (int d = 0; d < 4; ++d) {
+                    for (int gg = 0; gg < HB / 4; ++gg) {
+                        const int g = hb * (HB / 4) + gg;
+                        float p[4][2][4], o[4][8];
 #pragma unroll
-                        for (int s = 0; s < 8; s += 2) {
-                            float2 v = mul2(make_float2(o[d][s], o[d][s + 1]), make_float2(mul[s], mul[s + 1]));
-                            // int8: the low byte of (v + 1.5*2^23) is the two's complement code of rint(v).  The sum is
-                            // written as fma(v, 1, 1.5*2^23): the product above keeps its own rounding (a packed add right
-                            // after the packed product gets contracted into one fused operation, which changes half-way codes).
-                            if (I8) v = __ffma2_rn(v, make_float2(1.0f, 1.0f), make_float2(fz::MAGIC, fz::MAGIC));
-                            code[d][s] = __float_as_uint(v.x);
-                            code[d][s + 1] = __float_as_uint(v.y);
+                        for (int d = 0; d < 4; ++d) unpack_patch<T>(rawp[gg * 4 + d], p[d]);
+                        haar_fwd_lanes_raw<L, 4>(p, o, lane);
+                        uint32_t code[4][8];
+#pragma unroll
+                        for (int d = 0; d < 4; ++d) {
+#pragma unroll
+                            for (int s = 0; s < 8; s += 2) {
+                                float2 v = mul2(make_float2(o[d][s], o[d][s + 1]), make_float2(mul[s], mul[s + 1]));
+                                // int8: the low byte of (v + 1.5*2^23) is the two's complement code of rint(v).  The sum is
+                                // written as fma(v, 1, 1.5*2^23): the product above keeps its own rounding (a packed add right
+                                // after the packed product gets contracted into one fused operation, which changes half-way codes).
+                                if (I8) v = __ffma2_rn(v, make_float2(1.0f, 1.0f), make_float2(fz::MAGIC, fz::MAGIC));
+                                code[d][s] = __float_as_uint(v.x);
+                                code[d][s + 1] = __float_as_uint(v.y);
+                            }
                         }
-                    }
 #pragma unroll
-                    for (int s = 0; s < 8; ++s) {
-                        if (I8) {
-                            const uint32_t lo = __byte_perm(code[0][s], code[1][s], 0x0040);
-                            const uint32_t hi = __byte_perm(code[2][s], code[3][s], 0x0040);
-                            packed[s][g] = __byte_perm(lo, hi, 0x5410);
-                        } else {
-                            packed[s][2 * g] = pack_bf16x2(__uint_as_float(code[0][s]), __uint_as_float(code[1][s]));
-                            packed[s][2 * g + 1] = pack_bf16x2(__uint_as_float(code[2][s]), __uint_as_float(code[3][s]));
+                        for (int s = 0; s < 8; ++s) {
+                            if (I8) {
+                                const uint32_t lo = __byte_perm(code[0][s], code[1][s], 0x0040);
+                                const uint32_t hi = __byte_perm(code[2][s], code[3][s], 0x0040);
+                                packed[s][g] = __byte_perm(lo, hi, 0x5410);
+                            } else {
+                                packed[s][2 * g] = pack_bf16x2(__uint_as_float(code[0][s]), __uint_as_float(code[1][s]));
+                                packed[s][2 * g + 1] = pack_bf16x2(__uint_as_float(code[2][s]), __uint_as_float(code[3][s]));
+                            }
                         }
                     }
                 }

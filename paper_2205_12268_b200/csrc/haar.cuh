@@ -896,120 +896,167 @@ __device__ __noinline__ void tma_timeout(int* status)
     for (int i = 0; i < 2000; ++i) __nanosleep(1000);
 }
 
-// ---- first pass, one warp per tile, TMA-fed ----------------------------------------------------------
-// Every warp owns one tile and walks all channels itself, so the per-position chains of fused multiply-adds stay in
-// its registers (ascending channel order, no hand-off between warps, no block-wide barrier).  Memory parallelism
-// comes from the warp's own ring of TMA boxes (S stages of CB channels in flight), not from the number of warps.
+// ---- first pass, TMA-fed, the norm chain handed from warp to warp ------------------------------------------
+// One CTA of W warps per tile.  The warps take the boxes of CB channels in turn (box r goes to warp r % W): each transforms
+// its box on its own, fed by its own ring of TMA boxes, and only the chain of fused multiply-adds that builds the norms
+// (one per position, ascending channel order) runs in sequence: the eight partial sums of every lane travel from the warp
+// of box r to the warp of box r + 1 through shared memory (a "token", signalled on an mbarrier).  So the sums are the
+// same sequential chains a single thread would build, while loads, unpacking, transforms and maxima of different boxes
+// overlap.  The transform runs without its halvings (haar_fwd_lanes_raw); one exact multiplication per slot at the end.
 template <typename T, int L>
-struct NormsWarpCfg {
-    static constexpr int WARPS = 2;                               // independent warps per CTA
+struct NormsTokCfg {
+    static constexpr int W = 4;                                   // warps per tile
     static constexpr int CB = (sizeof(T) == 2) ? 8 : 4;           // channels per box: 4 KB
-    static constexpr int S = 6;                                   // boxes in flight per warp: 24 KB
+    static constexpr int S = 3;                                   // boxes in flight per warp
     using Ring = TileRing<T, L, CB, S>;
-    static constexpr size_t SMEM = 128 + (size_t)WARPS * (Ring::BYTES + S * 8);
+    static constexpr size_t SMEM = 128 + (size_t)W * Ring::BYTES + 8 * 32 * 4 + (size_t)W * 8 * 32 * 4 + (size_t)W * S * 8 + W * 8;
 };
 
 template <typename T, int L>
-__global__ void __launch_bounds__(NormsWarpCfg<T, L>::WARPS * 32)
-haar_norms_warp_kernel(const __grid_constant__ CUtensorMap tmx, int N, int C, int H, int W, int tiles_total, int tile_ctas,
-                       float* __restrict__ nrm2, float* __restrict__ amaxpos, const NormsExtra ex, int* __restrict__ status)
+__global__ void __launch_bounds__(NormsTokCfg<T, L>::W * 32, 4)
+haar_norms_token_kernel(const __grid_constant__ CUtensorMap tmx, int N, int C, int H, int W, int tiles_total,
+                        float* __restrict__ nrm2, float* __restrict__ amaxpos, const NormsExtra ex, int* __restrict__ status)
 {
     using TT = HaarTile<L>;
-    using Cfg = NormsWarpCfg<T, L>;
+    using Cfg = NormsTokCfg<T, L>;
     using Ring = typename Cfg::Ring;
-    constexpr int CB = Cfg::CB, S = Cfg::S, U = 4;
+    constexpr int CB = Cfg::CB, S = Cfg::S, NW = Cfg::W;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if ((int)blockIdx.x >= tile_ctas) {                // weight preparation CTAs
-        const int o = ((int)blockIdx.x - tile_ctas) * Cfg::WARPS + warp;
+    if ((int)blockIdx.x >= tiles_total) {              // weight preparation CTAs
+        const int o = ((int)blockIdx.x - tiles_total) * NW + warp;
         if (o < ex.Cout) weight_prep_row(ex.Wt, o, C, ex.kpad, ex.bits, ex.Wq, ex.scale_w);
         return;
     }
-    const int tile = (int)blockIdx.x * Cfg::WARPS + warp;
-    if (tile >= tiles_total) return;                   // warps never meet at a block-wide barrier
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_s = tc::smem_u32(smem_raw);
     uint8_t* sm = smem_raw + (((raw_s + 127u) & ~127u) - raw_s);
     uint8_t* stages = sm + (size_t)warp * Ring::BYTES;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sm + (size_t)Cfg::WARPS * Ring::BYTES) + warp * S;
+    float4* token = reinterpret_cast<float4*>(sm + (size_t)NW * Ring::BYTES);                 // [2][32] float4: 8 sums per lane
+    float* amax_sm = reinterpret_cast<float*>(token + 2 * 32);                                 // [NW][8][32]
+    uint64_t* ring_bars = reinterpret_cast<uint64_t*>(amax_sm + NW * 8 * 32);                   // [NW][S]
+    uint64_t* tok_bars = ring_bars + NW * S;                                                    // [NW]
 
     const int tiles_x = (W + TT::TW - 1) / TT::TW, tiles_y = H / TT::TH;
     int n, ty, tx;
-    tile_coords(tile, tiles_x, tiles_y, n, ty, tx);
+    tile_coords(blockIdx.x, tiles_x, tiles_y, n, ty, tx);
     const LanePos lp = lane_positions<L>(H, W, ty, tx, lane);
     const size_t P = (size_t)H * W;
     const int x0 = tx * TT::TW, y0 = ty * TT::TH;
 
-    Ring ring;
-    ring.init(stages, bars, lane);
     const int rounds = (C + CB - 1) / CB;
+    const int mine = (rounds - warp + NW - 1) / NW;    // boxes of this warp: r = warp + m * NW
+    Ring ring;
+    ring.init(stages, ring_bars + warp * S, lane);
     if (lane == 0) {
 #pragma unroll
-        for (int i = 0; i < S; ++i)
-            if (i < rounds) ring.issue(&tmx, i, x0, y0, i * CB, n);
+        for (int m = 0; m < S; ++m)
+            if (m < mine) ring.issue(&tmx, m, x0, y0, (warp + m * NW) * CB, n);
     }
-    // the transform runs without its halvings (haar_fwd_lanes_raw); one exact multiplication per slot at the end
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int i = 0; i < NW; ++i) tc::mbar_init(tc::smem_u32(&tok_bars[i]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
     float sc[8];
     slot_scales<L>(lane, ring.swap, sc);
-    float nacc[8], amax[8];
+    float amax[8];
 #pragma unroll
-    for (int s = 0; s < 8; ++s) { nacc[s] = 0.0f; amax[s] = 0.0f; }
+    for (int s = 0; s < 8; ++s) amax[s] = 0.0f;
     bool ok = true;
-    for (int r = 0; r < rounds; ++r) {
-        const int stage = r % S;
-        if (ok) ok = ring.wait(stage, (uint32_t)(r / S) & 1u);
+    for (int m = 0; m < mine && ok; ++m) {
+        const int r = warp + m * NW, stage = m % S;
+        ok = ring.wait(stage, (uint32_t)(m / S) & 1u);
+        RawPatch raw[CB];
 #pragma unroll
-        for (int g = 0; g < CB / U; ++g) {
-            float p[U][2][4], o[U][8];
+        for (int d = 0; d < CB; ++d) ring.read_raw(stage, d, raw[d]);      // channels beyond C arrive as zeros: fma(0, 0, acc) = acc
+        if (ex.coef) {                                 // test tap: the plain transform (also gets the signs of zeros right)
 #pragma unroll
-            for (int d = 0; d < U; ++d) {
-                RawPatch raw;
-                ring.read_raw(stage, g * U + d, raw);  // channels beyond C arrive as zeros: fma(0, 0, acc) = acc
-                unpack_patch<T>(raw, p[d]);
-            }
-            haar_fwd_lanes_raw<L, U>(p, o, lane);
-#pragma unroll
-            for (int d = 0; d < U; ++d) {
-                const int c = r * CB + g * U + d;
-                if (ex.coef && c < C) {                // test tap: the plain transform (also gets the signs of zeros right)
-                    RawPatch raw;
+            for (int d = 0; d < CB; ++d) {
+                if (r * CB + d < C) {
+                    RawPatch rw;
                     float pp[2][4], oc[8];
-                    ring.read(stage, g * U + d, raw);
-                    unpack_patch<T>(raw, pp);
+                    ring.read(stage, d, rw);
+                    unpack_patch<T>(rw, pp);
                     haar_fwd_lane<L>(pp, oc, lane);
-                    store_slots<L, true>(ex.coef + ((size_t)n * C + c) * P, lp, oc);
-                }
-#pragma unroll
-                for (int s = 0; s < 8; s += 2) {
-                    const float2 v = make_float2(o[d][s], o[d][s + 1]);
-                    const float2 a = __ffma2_rn(v, v, make_float2(nacc[s], nacc[s + 1]));
-                    nacc[s] = a.x; nacc[s + 1] = a.y;
-                    amax[s] = fmaxf(amax[s], fabsf(v.x));
-                    amax[s + 1] = fmaxf(amax[s + 1], fabsf(v.y));
+                    store_slots<L, true>(ex.coef + ((size_t)n * C + r * CB + d) * P, lp, oc);
                 }
             }
         }
         __syncwarp();                                  // every lane is done reading the stage
-        if (lane == 0 && r + S < rounds) ring.issue(&tmx, stage, x0, y0, (r + S) * CB, n);
-    }
-    if (!__all_sync(0xFFFFFFFFu, ok ? 1 : 0)) { tma_timeout(status); return; }
+        if (lane == 0 && m + S < mine) ring.issue(&tmx, stage, x0, y0, (warp + (m + S) * NW) * CB, n);
+        float o[CB][8];
 #pragma unroll
-    for (int s = 0; s < 8; ++s) {
-        nacc[s] = __fmul_rn(nacc[s], __fmul_rn(sc[s], sc[s]));
-        amax[s] = __fmul_rn(amax[s], fabsf(sc[s]));
-    }
-    store_slots<L, true>(nrm2 + (size_t)n * P, lp, nacc);
-    if (amaxpos) store_slots<L, true>(amaxpos + (size_t)n * P, lp, amax);
-    if (ex.hist1) {                                    // norms are >= +0: key = bits | sign bit, digit = top 11 bits
-        uint32_t* h = ex.hist1 + (size_t)n * 3 * 2048;
+        for (int g = 0; g < CB / 4; ++g) {
+            float p[4][2][4];
 #pragma unroll
-        for (int s = 0; s < 8; ++s) hist_add(h, float_key(nacc[s]) >> 21, lp.ok0);
-    }
-    if (ex.fine) {                                     // 16-bit digits are spread out: plain atomics
-        uint32_t* f = ex.fine + (size_t)n * 65536;
-        if (lp.ok0) {
-#pragma unroll
-            for (int s = 0; s < 8; ++s) atomicAdd(&f[float_key(nacc[s]) >> 16], 1u);
+            for (int d = 0; d < 4; ++d) unpack_patch<T>(raw[g * 4 + d], p[d]);
+            haar_fwd_lanes_raw<L, 4>(p, *reinterpret_cast<float(*)[4][8]>(&o[g * 4]), lane);
         }
+#pragma unroll
+        for (int d = 0; d < CB; ++d)
+#pragma unroll
+            for (int s = 0; s < 8; ++s) amax[s] = fmaxf(amax[s], fabsf(o[d][s]));
+        // the token: partial sums of the boxes before this one
+        float2 acc[4];
+        if (r > 0) {
+            const int waits_before = (warp == 0) ? m - 1 : m;
+            ok = tc::mbar_wait(tc::smem_u32(&tok_bars[warp]), (uint32_t)waits_before & 1u);
+            const float4 t0 = token[lane], t1 = token[32 + lane];
+            acc[0] = make_float2(t0.x, t0.y); acc[1] = make_float2(t0.z, t0.w);
+            acc[2] = make_float2(t1.x, t1.y); acc[3] = make_float2(t1.z, t1.w);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[i] = make_float2(0.0f, 0.0f);
+        }
+#pragma unroll
+        for (int d = 0; d < CB; ++d)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 v = make_float2(o[d][2 * i], o[d][2 * i + 1]);
+                acc[i] = __ffma2_rn(v, v, acc[i]);
+            }
+        if (r + 1 < rounds) {
+            token[lane] = make_float4(acc[0].x, acc[0].y, acc[1].x, acc[1].y);
+            token[32 + lane] = make_float4(acc[2].x, acc[2].y, acc[3].x, acc[3].y);
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(tc::smem_u32(&tok_bars[(warp + 1) % NW]));
+        } else if (ok) {                               // last box: these are the norms
+            float nacc[8];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                nacc[2 * i] = __fmul_rn(acc[i].x, __fmul_rn(sc[2 * i], sc[2 * i]));
+                nacc[2 * i + 1] = __fmul_rn(acc[i].y, __fmul_rn(sc[2 * i + 1], sc[2 * i + 1]));
+            }
+            store_slots<L, true>(nrm2 + (size_t)n * P, lp, nacc);
+            if (ex.hist1) {                            // norms are >= +0: key = bits | sign bit, digit = top 11 bits
+                uint32_t* h = ex.hist1 + (size_t)n * 3 * 2048;
+#pragma unroll
+                for (int s = 0; s < 8; ++s) hist_add(h, float_key(nacc[s]) >> 21, lp.ok0);
+            }
+            if (ex.fine && lp.ok0) {                   // 16-bit digits are spread out: plain atomics
+                uint32_t* f = ex.fine + (size_t)n * 65536;
+#pragma unroll
+                for (int s = 0; s < 8; ++s) atomicAdd(&f[float_key(nacc[s]) >> 16], 1u);
+            }
+        }
+    }
+    if (!__all_sync(0xFFFFFFFFu, ok ? 1 : 0)) tma_timeout(status);
+    // per-position max |coef|: combine the warps' maxima
+#pragma unroll
+    for (int s = 0; s < 8; ++s) amax_sm[(warp * 8 + s) * 32 + lane] = amax[s];
+    __syncthreads();
+    if (warp == 0 && amaxpos) {
+        float am[8];
+#pragma unroll
+        for (int s = 0; s < 8; ++s) {
+            float v = amax_sm[s * 32 + lane];
+#pragma unroll
+            for (int w2 = 1; w2 < NW; ++w2) v = fmaxf(v, amax_sm[(w2 * 8 + s) * 32 + lane]);
+            am[s] = __fmul_rn(v, fabsf(sc[s]));
+        }
+        store_slots<L, true>(amaxpos + (size_t)n * P, lp, am);
     }
 }
 
@@ -1131,18 +1178,16 @@ static wcc_status haar_norms_dispatch(const void* x, int N, int C, int H, int W,
     using TT = HaarTile<L>;
     const long long tiles = (long long)N * ceil_div(W, TT::TW) * (H / TT::TH);
     if (VEC && tc::tma_ok_x(x, (int)sizeof(T), W)) {
-        using Cfg = NormsWarpCfg<T, L>;
+        using Cfg = NormsTokCfg<T, L>;
         CUtensorMap tmx;
         if (!tc::make_map_x(&tmx, x, (int)sizeof(T), N, C, H, W, TT::TW, TT::TH, Cfg::CB)) return WCC_ERR_CUDA;
         int* status = nullptr;
         WCC_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_status));
-        WCC_CUDA_TRY(cudaFuncSetAttribute(haar_norms_warp_kernel<T, L>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM));
-        const long long tile_ctas = (tiles + Cfg::WARPS - 1) / Cfg::WARPS;
-        const long long grid = tile_ctas + (ex.Wt ? ceil_div(ex.Cout, Cfg::WARPS) : 0);
+        WCC_CUDA_TRY(cudaFuncSetAttribute(haar_norms_token_kernel<T, L>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM));
+        const long long grid = tiles + (ex.Wt ? ceil_div(ex.Cout, Cfg::W) : 0);
         if (grid > 0x7FFFFFFFLL) return WCC_ERR_SHAPE;
         ex.tiles = (int)tiles;
-        haar_norms_warp_kernel<T, L><<<(unsigned)grid, Cfg::WARPS * 32, Cfg::SMEM, st>>>(tmx, N, C, H, W, (int)tiles, (int)tile_ctas,
-                                                                                        nrm2, amaxpos, ex, status);
+        haar_norms_token_kernel<T, L><<<(unsigned)grid, Cfg::W * 32, Cfg::SMEM, st>>>(tmx, N, C, H, W, (int)tiles, nrm2, amaxpos, ex, status);
         WCC_LAUNCH_CHECK();
         return WCC_OK;
     }
