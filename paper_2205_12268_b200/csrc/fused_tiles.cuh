@@ -92,14 +92,38 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    const int tiles_x = (pr.W + TT::TW - 1) / TT::TW, tiles_y = pr.H / TT::TH;
     if (is_mma) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(tc::smem_u32(&ctl->tmem_base)), "r"((uint32_t)pr.tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        // Lane w of this warp starts the input ring of compute warp w (barriers and the first S boxes), so that the
+        // compute warps spend the set-up on their own global loads instead of waiting for the first TMA issue.
+        if (lane < C::CWARPS) {
+            const int t2 = lane & 3, q2 = lane >> 2, tile2 = (int)blockIdx.x * TILES + t2;
+            const uint32_t bar2 = tc::smem_u32(ring_bars + lane * C::S);
+            const uint32_t ring2 = tc::smem_u32(sRing + (size_t)lane * Ring::BYTES);
+#pragma unroll
+            for (int i = 0; i < C::S; ++i) tc::mbar_init(bar2 + 8 * i, 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            if (tile2 < pr.tiles_total) {
+                int n2, ty2, tx2;
+                tile_coords(tile2, tiles_x, tiles_y, n2, ty2, tx2);
+                const int boxes2 = ((kchunks - q2 + WPT - 1) / WPT) * C::BPC;
+#pragma unroll
+                for (int m = 0; m < C::S; ++m) {
+                    if (m < boxes2) {
+                        tc::mbar_expect_tx(bar2 + 8 * m, Ring::STAGE_BYTES);
+                        tc::tma_load_4d(ring2 + m * Ring::STAGE_BYTES, &tmx, tx2 * TT::TW, ty2 * TT::TH,
+                                        (q2 + (m / C::BPC) * WPT) * C::CCH + (m % C::BPC) * C::CB, n2, bar2 + 8 * m);
+                    }
+                }
+            }
+        }
+        __syncwarp();
     }
     const int tile = (int)blockIdx.x * TILES + t;
     const bool live = !is_mma && tile < pr.tiles_total;
-    const int tiles_x = (pr.W + TT::TW - 1) / TT::TW, tiles_y = pr.H / TT::TH;
     int n = 0, ty = 0, tx = 0;
     if (live) tile_coords(tile, tiles_x, tiles_y, n, ty, tx);
     const LanePos lp = lane_positions<L>(pr.H, pr.W, ty, tx, lane);
@@ -111,14 +135,7 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
     const int my_boxes = live ? my_chunks * C::BPC : 0;
     auto box_c0 = [&](int m) { return (q + (m / C::BPC) * WPT) * C::CCH + (m % C::BPC) * C::CB; };
     Ring ring;
-    if (!is_mma) {
-        ring.init(sRing + (size_t)warp * Ring::BYTES, ring_bars + warp * C::S, lane);
-        if (lane == 0) {
-#pragma unroll
-            for (int m = 0; m < C::S; ++m)
-                if (m < my_boxes) ring.issue(&tmx, m, x0, y0, box_c0(m), n);
-        }
-    }
+    if (!is_mma) ring.attach(sRing + (size_t)warp * Ring::BYTES, ring_bars + warp * C::S, lane);
     // weights -> B operand (core-matrix layout), all threads
     for (int i = threadIdx.x; i < pr.npad * kchunks; i += C::THREADS) {
         const int row = i / kchunks, j = i - row * kchunks;

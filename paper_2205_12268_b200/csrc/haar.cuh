@@ -827,6 +827,14 @@ struct TileRing {
     int off_a, off_b;            // byte offsets (inside a channel) of the row this lane reads first / second
     bool swap;                   // the first row read is the patch's second row
 
+    // the same without touching the barriers (another thread initializes them and a block-wide barrier follows)
+    __device__ __forceinline__ void attach(uint8_t* stages, uint64_t* bars, int lane)
+    {
+        ring = stages;
+        ring_s = tc::smem_u32(stages);
+        bar_s = tc::smem_u32(bars);
+        set_lane(lane);
+    }
     __device__ __forceinline__ void init(uint8_t* stages, uint64_t* bars, int lane)
     {
         ring = stages;
