@@ -185,7 +185,8 @@ const char* wcc_status_str(wcc_status s);
  * stream around each stage; wcc_profile_read waits for the last recorded call and writes, to the HOST array ms, the
  * milliseconds of, for wcc_forward_staged: 0 Haar transform + norms, 1 top-k select + compaction, 2 weight
  * quantization, 3 gather + quantize, 4 tensor-core contraction, 5 dequantize + scatter + inverse Haar; for wcc_forward:
- * 0 pass 1 (transform + norms, select histograms, weight quantization), 1 select, 2 fused pass 2, 3 to 5 zero.
+ * 0 clearing of the select's histograms (a memset node), 1 pass 1 (transform + norms, select histograms, weight
+ * quantization), 2 select, 3 fused pass 2, 4 and 5 zero.
  * Off by default; not thread-safe.
  */
 #define WCC_NUM_STAGES 6

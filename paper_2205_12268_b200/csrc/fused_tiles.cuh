@@ -235,7 +235,7 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
             if (live) {
                 // all of the chunk's input words first (one wait per box), refill the stages right away, then compute:
                 // the groups of four channels below carry no barrier between them and overlap freely
-                constexpr int HB = (sizeof(T) == 2) ? C::CCH : ((C::CCH < 8) ? C::CCH : 8);   // channels loaded ahead (<= 64 registers)
+                constexpr int HB = (C::CCH < 8) ? C::CCH : 8;     // channels loaded ahead
 #pragma unroll
                 for (int hb = 0; hb < C::CCH / HB; ++hb) {
                     RawPatch rawp[HB];

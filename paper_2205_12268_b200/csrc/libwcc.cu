@@ -218,6 +218,7 @@ static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, i
     // histogram and quantizes the weights in a few extra CTAs.
     const SelectWs sw = carve_select_ws(f.sel, N, P);
     WCC_CUDA_TRY(cudaMemsetAsync(f.fine, 0, f.fine_bytes + sw.zero_bytes, st));   // histograms, max |kept|, barrier counters
+    if ((s = profile_mark(1, st)) != WCC_OK) return s;
     NormsExtra ex = {};
     ex.coef = taps ? taps->coef : nullptr;
     ex.hist1 = sw.hist;
@@ -225,12 +226,12 @@ static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, i
     ex.Wt = Wt; ex.Wq = f.Wq; ex.scale_w = f.scale_w; ex.Cout = Cout; ex.kpad = f.kpad; ex.bits = bits;
     s = launch_haar_norms(x, N, Cin, H, W, L, dt, f.nrm2, f.amaxpos, ex, st);
     if (s != WCC_OK) return s;
-    if ((s = profile_mark(1, st)) != WCC_OK) return s;
+    if ((s = profile_mark(2, st)) != WCC_OK) return s;
     // joint shrinkage: index list, rank map, max |kept|
     s = launch_select(f.nrm2, N, P, k, f.idx, nullptr, f.rank, f.amaxpos, true, f.sel, f.sel_bytes, st, true,
                       f.fine, f.thr, taps != nullptr);
     if (s != WCC_OK) return s;
-    if ((s = profile_mark(2, st)) != WCC_OK) return s;
+    if ((s = profile_mark(3, st)) != WCC_OK) return s;
     // second pass over x: transform, mask + quantize, tensor-core contraction, dequantize, inverse, store
     void* xq_tap = taps ? (bits >= 2 ? static_cast<void*>(taps->Xq) : taps->Xb) : nullptr;
     s = launch_fused_tiles(x, f.Wq, f.rank, f.nrm2, f.thr, f.amax_kept, bits, f.scale_w, N, Cin, Cout, H, W, L, k, f.kpad, dt, y,
@@ -239,7 +240,7 @@ static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, i
         s = launch_fused_pass2(x, f.Wq, f.rank, f.nrm2, f.thr, f.amax_kept, bits, f.scale_w, N, Cin, Cout, H, W, L, k, f.kpad, dt, y,
                                xq_tap, taps ? taps->acc : nullptr, st);
     if (s != WCC_OK) return s;
-    for (int i = 3; i <= WCC_NUM_STAGES; ++i)
+    for (int i = 4; i <= WCC_NUM_STAGES; ++i)
         if ((s = profile_mark(i, st)) != WCC_OK) return s;
 
     if (taps) {

@@ -23,7 +23,7 @@ EXPORTS = ("wcc_staged_workspace_bytes", "wcc_forward_staged", "wcc_workspace_by
            "wcc_profile_enable", "wcc_profile_read", "wcc_kernel_launches", "wcc_select_topk_static")
 STATIC_SCRATCH_BYTES = 512 * 1024
 STAGES = ("haar_fwd_norms", "select_topk", "weight_quant", "gather_quant", "contract", "scatter_inv")   # wcc_forward_staged
-FUSED_STAGES = ("haar_norms", "select_topk", "fused_pass2")                                               # wcc_forward
+FUSED_STAGES = ("clear", "haar_norms", "select_topk", "fused_pass2")                                      # wcc_forward
 
 
 class WccError(RuntimeError):

@@ -91,6 +91,10 @@ SMALL = [  # N, Cin, Cout, H, W, dtype, levels, gamma, bits
     (2, 144, 24, 32, 64, "bf16", 3, 0.5, 0),
     (1, 8, 8, 32, 32, "f32", 2, 0.25, 4),         # fewer bits on the same int8 path
     (1, 8, 8, 32, 32, "f32", 2, 0.25, 2),
+    (1, 40, 24, 8, 96, "bf16", 3, 0.5, 8),        # three tiles: the last group of four is ragged
+    (3, 12, 80, 16, 160, "f32", 2, 0.3, 8),       # output channels in chunks of 32, 32 and 16; 15 tiles
+    (2, 70, 20, 16, 64, "bf16", 3, 0.4, 8),       # three K steps streamed through two operand buffers
+    (1, 20, 100, 24, 64, "bf16", 3, 0.3, 0),      # unquantized, several chunks of output channels, two K steps
 ]
 
 
