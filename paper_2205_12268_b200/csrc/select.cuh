@@ -458,7 +458,7 @@ struct ClusterSmem {
     uint32_t amax;
     uint32_t ncand;                 // candidates of this CTA (keys whose top 16 bits hold the threshold)
     uint32_t cand[CL_CAND_CTA];
-    uint32_t all[CL_CAND_MAX];      // candidates of the whole cluster
+    __align__(16) uint32_t all[CL_CAND_MAX];      // candidates of the whole cluster
     uint32_t thr[3];                // threshold key, ties to keep, ties in total
 };
 
@@ -659,7 +659,13 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
             for (uint32_t i = threadIdx.x; i < M; i += blockDim.x) {
                 const uint32_t ci = sm.all[i];
                 uint32_t g = 0, e = 0;
-                for (uint32_t j = 0; j < M; ++j) { const uint32_t cj = sm.all[j]; g += cj > ci; e += cj == ci; }
+                const uint4* all4 = reinterpret_cast<const uint4*>(sm.all);
+                for (uint32_t j4 = 0; j4 < M / 4; ++j4) {        // four candidates per shared-memory load
+                    const uint4 c = all4[j4];
+                    g += (c.x > ci) + (c.y > ci) + (c.z > ci) + (c.w > ci);
+                    e += (c.x == ci) + (c.y == ci) + (c.z == ci) + (c.w == ci);
+                }
+                for (uint32_t j = M & ~3u; j < M; ++j) { const uint32_t cj = sm.all[j]; g += cj > ci; e += cj == ci; }
                 if (g < k16 && k16 <= g + e) { sm.thr[0] = ci; sm.thr[1] = k16 - g; sm.thr[2] = e; }   // equal keys write equal values
             }
             __syncthreads();
@@ -706,6 +712,10 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
 
     const bool ordered = want_rank || need_eq < total_eq;       // uniform over the cluster
     float amax = 0.0f;
+    // Nobody may leave while a neighbour can still read its shared memory.  When no further exchange follows, every CTA
+    // signals here that it is done reading and only waits for the others at the very end (the wait is hidden behind the
+    // pass over the kept positions).
+    if (!ordered) cluster.barrier_arrive();
     if (!ordered) {
         // every key >= threshold is kept; nobody needs the order
         if (amaxpos) {
@@ -760,7 +770,8 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
         __syncthreads();
         if (threadIdx.x == 0 && sm.amax) atomicMax(reinterpret_cast<uint32_t*>(amax_kept), sm.amax);
     }
-    cluster.sync();                                  // nobody leaves while a neighbour may still read its shared memory
+    if (!ordered) cluster.barrier_wait();
+    else cluster.sync();                             // nobody leaves while a neighbour may still read its shared memory
 }
 
 __global__ void thr_use_rank_kernel(uint32_t* thr, int N)
