@@ -648,11 +648,12 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
         for (int r = 0; r < cs; ++r) { overflow = overflow || sm.tot[r] > CL_CAND_CTA; M += sm.tot[r]; }
         overflow = overflow || M > CL_CAND_MAX;
         if (!overflow) {
-            uint32_t off = 0;
-            for (int r = 0; r < cs; ++r) {
-                const uint32_t* rc = cluster.map_shared_rank(sm.cand, r);
-                for (uint32_t i = threadIdx.x; i < sm.tot[r]; i += blockDim.x) sm.all[off + i] = rc[i];
-                off += sm.tot[r];
+            // one remote load per thread, all in flight together (rank after rank would expose every rank's latency)
+            for (uint32_t g = threadIdx.x; g < M; g += blockDim.x) {
+                uint32_t pre = 0;
+                int r = 0;
+                while (g >= pre + sm.tot[r]) { pre += sm.tot[r]; ++r; }
+                sm.all[g] = cluster.map_shared_rank(sm.cand, r)[g - pre];
             }
             __syncthreads();
             // the k16-th largest candidate, by counting (M is small)
