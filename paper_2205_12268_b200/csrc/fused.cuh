@@ -1,4 +1,7 @@
-// Second pass of the fused layer: for one warp tile of one image, recompute the Haar transform from x, keep the
+// Second pass of the fused layer, one tile per CTA.  wcc_forward uses it for the shapes that the four-tile kernel of
+// fused_tiles.cuh does not cover (input rows that cannot be a TMA map, many output channels together with many K steps);
+// that kernel also borrows the descriptor and TMEM helpers below.
+// For one warp tile of one image, recompute the Haar transform from x, keep the
 // selected positions (zero the others), quantize, run the pointwise convolution on tensor cores, dequantize,
 // apply the inverse transform and store y (steps A, C, D, E of the WCC workflow, Eq. 9 / Alg. 1, with the index
 // set and the activation scale of step B already known).  Neither the coefficient map, nor the compressed matrix,

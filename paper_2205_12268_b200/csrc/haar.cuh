@@ -11,10 +11,11 @@
 //        L>=2, rp even: slot 7 = y2 of level 2, slot 6 = y1 of level 2 (L=2) or one of y1..y4 of level 3,
 //                       by (rp & 2, cg & 1): (0,0) y1, (0,1) y2, (2,0) y3, (2,1) y4
 //        L>=2, rp odd : slot 6 = y3 of level 2, slot 7 = y4 of level 2
-// so the per-position norm accumulators live in registers across the whole channel loop, which keeps the
-// channel order of the fused multiply-add chain fixed (ascending), and nothing is exchanged through
-// shared memory.  Arithmetic follows the order written in wcc.h so that results are bit-identical to a
-// plain fp32 evaluation.
+// In haar_fwd_kernel the per-position norm accumulators live in registers across the whole channel loop, which keeps
+// the channel order of the fused multiply-add chain fixed (ascending); the first pass of the fused layer
+// (haar_norms_token_kernel) keeps that order too while several warps share a tile: the partial sums are handed from
+// warp to warp.  Arithmetic follows the order written in wcc.h so that results are bit-identical to a plain fp32
+// evaluation.
 #pragma once
 
 #include "common.cuh"
@@ -660,7 +661,8 @@ struct PatchRing {
     }
 };
 
-// ---- first pass of the fused layer: norms only (inputs through per-warp cp.async rings) -----------
+// ---- first pass of the fused layer without TMA (rows that are no multiple of 16 bytes, unaligned x) -----------
+// Norms only, inputs through per-warp cp.async rings.
 // One CTA of 4 warps per (image, tile).  The warps split the channels: in every round of 4 * LU channels warp w
 // transforms channels [w * LU, (w + 1) * LU) of the round in registers and hands the slot values over through shared
 // memory; then the 128 threads run the fused multiply-add chain of two positions each (warp w: slots 2w and 2w+1
