@@ -924,7 +924,7 @@ struct NormsTokCfg {
 
 template <typename T, int L>
 __global__ void __launch_bounds__(NormsTokCfg<T, L>::W * 32, 4)
-haar_norms_token_kernel(const __grid_constant__ CUtensorMap tmx, int N, int C, int H, int W, int tiles_total,
+haar_norms_token_kernel(const __grid_constant__ CUtensorMap tmx, int N, int C, int H, int W, int tiles_total, int tile_ctas,
                         float* __restrict__ nrm2, float* __restrict__ amaxpos, const NormsExtra ex, int* __restrict__ status)
 {
     using TT = HaarTile<L>;
@@ -932,8 +932,8 @@ haar_norms_token_kernel(const __grid_constant__ CUtensorMap tmx, int N, int C, i
     using Ring = typename Cfg::Ring;
     constexpr int CB = Cfg::CB, S = Cfg::S, NW = Cfg::W;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if ((int)blockIdx.x >= tiles_total) {              // weight preparation CTAs
-        const int o = ((int)blockIdx.x - tiles_total) * NW + warp;
+    if ((int)blockIdx.x >= tile_ctas) {                // weight preparation CTAs
+        const int o = ((int)blockIdx.x - tile_ctas) * NW + warp;
         if (o < ex.Cout) weight_prep_row(ex.Wt, o, C, ex.kpad, ex.bits, ex.Wq, ex.scale_w);
         return;
     }
@@ -946,21 +946,26 @@ haar_norms_token_kernel(const __grid_constant__ CUtensorMap tmx, int N, int C, i
     uint64_t* ring_bars = reinterpret_cast<uint64_t*>(amax_sm + NW * 8 * 32);                   // [NW][S]
     uint64_t* tok_bars = ring_bars + NW * S;                                                    // [NW]
 
+    // The CTA walks the tiles blockIdx.x, blockIdx.x + tile_ctas, ...; a warp's ring of boxes runs on across tiles, so
+    // the first boxes of the next tile are in flight while the current one is finished.
     const int tiles_x = (W + TT::TW - 1) / TT::TW, tiles_y = H / TT::TH;
-    int n, ty, tx;
-    tile_coords(blockIdx.x, tiles_x, tiles_y, n, ty, tx);
-    const LanePos lp = lane_positions<L>(H, W, ty, tx, lane);
     const size_t P = (size_t)H * W;
-    const int x0 = tx * TT::TW, y0 = ty * TT::TH;
-
+    const int iters = (tiles_total - (int)blockIdx.x + tile_ctas - 1) / tile_ctas;
     const int rounds = (C + CB - 1) / CB;
-    const int mine = (rounds - warp + NW - 1) / NW;    // boxes of this warp: r = warp + m * NW
+    const int mine = (rounds - warp + NW - 1) / NW;    // boxes of this warp per tile: r = warp + m * NW
+    const int total = iters * mine;
     Ring ring;
     ring.init(stages, ring_bars + warp * S, lane);
+    auto issue_box = [&](int mg) {                     // lane 0 only; mg counts this warp's boxes over all its tiles
+        const int it = mg / mine, mi = mg - it * mine;
+        int n_, ty_, tx_;
+        tile_coords((int)blockIdx.x + it * tile_ctas, tiles_x, tiles_y, n_, ty_, tx_);
+        ring.issue(&tmx, mg % S, tx_ * TT::TW, ty_ * TT::TH, (warp + mi * NW) * CB, n_);
+    };
     if (lane == 0) {
 #pragma unroll
         for (int m = 0; m < S; ++m)
-            if (m < mine) ring.issue(&tmx, m, x0, y0, (warp + m * NW) * CB, n);
+            if (m < total) issue_box(m);
     }
     if (threadIdx.x == 0) {
 #pragma unroll
@@ -971,103 +976,111 @@ haar_norms_token_kernel(const __grid_constant__ CUtensorMap tmx, int N, int C, i
 
     float sc[8];
     slot_scales<L>(lane, ring.swap, sc);
-    float amax[8];
-#pragma unroll
-    for (int s = 0; s < 8; ++s) amax[s] = 0.0f;
     bool ok = true;
-    for (int m = 0; m < mine && ok; ++m) {
-        const int r = warp + m * NW, stage = m % S;
-        ok = ring.wait(stage, (uint32_t)(m / S) & 1u);
-        RawPatch raw[CB];
+    int mg = 0, tok_seen = 0;                          // boxes consumed / tokens received so far
+    for (int it = 0; it < iters; ++it) {
+        int n, ty, tx;
+        tile_coords((int)blockIdx.x + it * tile_ctas, tiles_x, tiles_y, n, ty, tx);
+        const LanePos lp = lane_positions<L>(H, W, ty, tx, lane);
+        float amax[8];
 #pragma unroll
-        for (int d = 0; d < CB; ++d) ring.read_raw(stage, d, raw[d]);      // channels beyond C arrive as zeros: fma(0, 0, acc) = acc
-        if (ex.coef) {                                 // test tap: the plain transform (also gets the signs of zeros right)
+        for (int s = 0; s < 8; ++s) amax[s] = 0.0f;
+        for (int m = 0; m < mine && ok; ++m, ++mg) {
+            const int r = warp + m * NW, stage = mg % S;
+            ok = ring.wait(stage, (uint32_t)(mg / S) & 1u);
+            RawPatch raw[CB];
 #pragma unroll
-            for (int d = 0; d < CB; ++d) {
-                if (r * CB + d < C) {
-                    RawPatch rw;
-                    float pp[2][4], oc[8];
-                    ring.read(stage, d, rw);
-                    unpack_patch<T>(rw, pp);
-                    haar_fwd_lane<L>(pp, oc, lane);
-                    store_slots<L, true>(ex.coef + ((size_t)n * C + r * CB + d) * P, lp, oc);
+            for (int d = 0; d < CB; ++d) ring.read_raw(stage, d, raw[d]);      // channels beyond C arrive as zeros: fma(0, 0, acc) = acc
+            if (ex.coef) {                             // test tap: the plain transform (also gets the signs of zeros right)
+#pragma unroll
+                for (int d = 0; d < CB; ++d) {
+                    if (r * CB + d < C) {
+                        RawPatch rw;
+                        float pp[2][4], oc[8];
+                        ring.read(stage, d, rw);
+                        unpack_patch<T>(rw, pp);
+                        haar_fwd_lane<L>(pp, oc, lane);
+                        store_slots<L, true>(ex.coef + ((size_t)n * C + r * CB + d) * P, lp, oc);
+                    }
+                }
+            }
+            __syncwarp();                              // every lane is done reading the stage
+            if (lane == 0 && mg + S < total) issue_box(mg + S);
+            float o[CB][8];
+#pragma unroll
+            for (int g = 0; g < CB / 4; ++g) {
+                float p[4][2][4];
+#pragma unroll
+                for (int d = 0; d < 4; ++d) unpack_patch<T>(raw[g * 4 + d], p[d]);
+                haar_fwd_lanes_raw<L, 4>(p, *reinterpret_cast<float(*)[4][8]>(&o[g * 4]), lane);
+            }
+#pragma unroll
+            for (int d = 0; d < CB; ++d)
+#pragma unroll
+                for (int s = 0; s < 8; ++s) amax[s] = fmaxf(amax[s], fabsf(o[d][s]));
+            // the token: partial sums of the boxes before this one
+            float2 acc[4];
+            if (r > 0) {
+                ok = tc::mbar_wait(tc::smem_u32(&tok_bars[warp]), (uint32_t)tok_seen & 1u);
+                ++tok_seen;
+                const float4 t0 = token[lane], t1 = token[32 + lane];
+                acc[0] = make_float2(t0.x, t0.y); acc[1] = make_float2(t0.z, t0.w);
+                acc[2] = make_float2(t1.x, t1.y); acc[3] = make_float2(t1.z, t1.w);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[i] = make_float2(0.0f, 0.0f);
+            }
+#pragma unroll
+            for (int d = 0; d < CB; ++d)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float2 v = make_float2(o[d][2 * i], o[d][2 * i + 1]);
+                    acc[i] = __ffma2_rn(v, v, acc[i]);
+                }
+            if (r + 1 < rounds) {
+                token[lane] = make_float4(acc[0].x, acc[0].y, acc[1].x, acc[1].y);
+                token[32 + lane] = make_float4(acc[2].x, acc[2].y, acc[3].x, acc[3].y);
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(tc::smem_u32(&tok_bars[(warp + 1) % NW]));
+            } else if (ok) {                           // last box: these are the norms
+                float nacc[8];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    nacc[2 * i] = __fmul_rn(acc[i].x, __fmul_rn(sc[2 * i], sc[2 * i]));
+                    nacc[2 * i + 1] = __fmul_rn(acc[i].y, __fmul_rn(sc[2 * i + 1], sc[2 * i + 1]));
+                }
+                store_slots<L, true>(nrm2 + (size_t)n * P, lp, nacc);
+                if (ex.hist1) {                        // norms are >= +0: key = bits | sign bit, digit = top 11 bits
+                    uint32_t* h = ex.hist1 + (size_t)n * 3 * 2048;
+#pragma unroll
+                    for (int s = 0; s < 8; ++s) hist_add(h, float_key(nacc[s]) >> 21, lp.ok0);
+                }
+                if (ex.fine && lp.ok0) {               // 16-bit digits are spread out: plain atomics
+                    uint32_t* f = ex.fine + (size_t)n * 65536;
+#pragma unroll
+                    for (int s = 0; s < 8; ++s) atomicAdd(&f[float_key(nacc[s]) >> 16], 1u);
                 }
             }
         }
-        __syncwarp();                                  // every lane is done reading the stage
-        if (lane == 0 && m + S < mine) ring.issue(&tmx, stage, x0, y0, (warp + (m + S) * NW) * CB, n);
-        float o[CB][8];
+        // per-position max |coef|: combine the warps' maxima.  The two block-wide barriers also keep every token of
+        // this tile ahead of any token of the next one (a single token buffer is enough).
 #pragma unroll
-        for (int g = 0; g < CB / 4; ++g) {
-            float p[4][2][4];
+        for (int s = 0; s < 8; ++s) amax_sm[(warp * 8 + s) * 32 + lane] = amax[s];
+        __syncthreads();
+        if (warp == 0 && amaxpos) {
+            float am[8];
 #pragma unroll
-            for (int d = 0; d < 4; ++d) unpack_patch<T>(raw[g * 4 + d], p[d]);
-            haar_fwd_lanes_raw<L, 4>(p, *reinterpret_cast<float(*)[4][8]>(&o[g * 4]), lane);
+            for (int s = 0; s < 8; ++s) {
+                float v = amax_sm[s * 32 + lane];
+#pragma unroll
+                for (int w2 = 1; w2 < NW; ++w2) v = fmaxf(v, amax_sm[(w2 * 8 + s) * 32 + lane]);
+                am[s] = __fmul_rn(v, fabsf(sc[s]));
+            }
+            store_slots<L, true>(amaxpos + (size_t)n * P, lp, am);
         }
-#pragma unroll
-        for (int d = 0; d < CB; ++d)
-#pragma unroll
-            for (int s = 0; s < 8; ++s) amax[s] = fmaxf(amax[s], fabsf(o[d][s]));
-        // the token: partial sums of the boxes before this one
-        float2 acc[4];
-        if (r > 0) {
-            const int waits_before = (warp == 0) ? m - 1 : m;
-            ok = tc::mbar_wait(tc::smem_u32(&tok_bars[warp]), (uint32_t)waits_before & 1u);
-            const float4 t0 = token[lane], t1 = token[32 + lane];
-            acc[0] = make_float2(t0.x, t0.y); acc[1] = make_float2(t0.z, t0.w);
-            acc[2] = make_float2(t1.x, t1.y); acc[3] = make_float2(t1.z, t1.w);
-        } else {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) acc[i] = make_float2(0.0f, 0.0f);
-        }
-#pragma unroll
-        for (int d = 0; d < CB; ++d)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float2 v = make_float2(o[d][2 * i], o[d][2 * i + 1]);
-                acc[i] = __ffma2_rn(v, v, acc[i]);
-            }
-        if (r + 1 < rounds) {
-            token[lane] = make_float4(acc[0].x, acc[0].y, acc[1].x, acc[1].y);
-            token[32 + lane] = make_float4(acc[2].x, acc[2].y, acc[3].x, acc[3].y);
-            __syncwarp();
-            if (lane == 0) tc::mbar_arrive(tc::smem_u32(&tok_bars[(warp + 1) % NW]));
-        } else if (ok) {                               // last box: these are the norms
-            float nacc[8];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                nacc[2 * i] = __fmul_rn(acc[i].x, __fmul_rn(sc[2 * i], sc[2 * i]));
-                nacc[2 * i + 1] = __fmul_rn(acc[i].y, __fmul_rn(sc[2 * i + 1], sc[2 * i + 1]));
-            }
-            store_slots<L, true>(nrm2 + (size_t)n * P, lp, nacc);
-            if (ex.hist1) {                            // norms are >= +0: key = bits | sign bit, digit = top 11 bits
-                uint32_t* h = ex.hist1 + (size_t)n * 3 * 2048;
-#pragma unroll
-                for (int s = 0; s < 8; ++s) hist_add(h, float_key(nacc[s]) >> 21, lp.ok0);
-            }
-            if (ex.fine && lp.ok0) {                   // 16-bit digits are spread out: plain atomics
-                uint32_t* f = ex.fine + (size_t)n * 65536;
-#pragma unroll
-                for (int s = 0; s < 8; ++s) atomicAdd(&f[float_key(nacc[s]) >> 16], 1u);
-            }
-        }
+        __syncthreads();
     }
     if (!__all_sync(0xFFFFFFFFu, ok ? 1 : 0)) tma_timeout(status);
-    // per-position max |coef|: combine the warps' maxima
-#pragma unroll
-    for (int s = 0; s < 8; ++s) amax_sm[(warp * 8 + s) * 32 + lane] = amax[s];
-    __syncthreads();
-    if (warp == 0 && amaxpos) {
-        float am[8];
-#pragma unroll
-        for (int s = 0; s < 8; ++s) {
-            float v = amax_sm[s * 32 + lane];
-#pragma unroll
-            for (int w2 = 1; w2 < NW; ++w2) v = fmaxf(v, amax_sm[(w2 * 8 + s) * 32 + lane]);
-            am[s] = __fmul_rn(v, fabsf(sc[s]));
-        }
-        store_slots<L, true>(amaxpos + (size_t)n * P, lp, am);
-    }
 }
 
 // ---- plain inverse -------------------------------------------------------------------------------
@@ -1194,10 +1207,18 @@ static wcc_status haar_norms_dispatch(const void* x, int N, int C, int H, int W,
         int* status = nullptr;
         WCC_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_status));
         WCC_CUDA_TRY(cudaFuncSetAttribute(haar_norms_token_kernel<T, L>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM));
-        const long long grid = tiles + (ex.Wt ? ceil_div(ex.Cout, Cfg::W) : 0);
-        if (grid > 0x7FFFFFFFLL) return WCC_ERR_SHAPE;
+        if (tiles > 0x7FFFFFFFLL) return WCC_ERR_SHAPE;
+        static int sm_count[64] = {0};
+        int dev = 0;
+        WCC_CUDA_TRY(cudaGetDevice(&dev));
+        if (dev < 0 || dev >= 64) return WCC_ERR_CUDA;
+        if (!sm_count[dev]) WCC_CUDA_TRY(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
+        const long long resident = 4LL * sm_count[dev];                 // four CTAs per SM: every tile CTA is resident at once
+        const int tile_ctas = (int)(tiles < resident ? tiles : resident);
+        const long long grid = tile_ctas + (ex.Wt ? ceil_div(ex.Cout, Cfg::W) : 0);
         ex.tiles = (int)tiles;
-        haar_norms_token_kernel<T, L><<<(unsigned)grid, Cfg::W * 32, Cfg::SMEM, st>>>(tmx, N, C, H, W, (int)tiles, nrm2, amaxpos, ex, status);
+        haar_norms_token_kernel<T, L><<<(unsigned)grid, Cfg::W * 32, Cfg::SMEM, st>>>(tmx, N, C, H, W, (int)tiles, tile_ctas, nrm2,
+                                                                                         amaxpos, ex, status);
         WCC_LAUNCH_CHECK();
         return WCC_OK;
     }
