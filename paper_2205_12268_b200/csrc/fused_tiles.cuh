@@ -21,8 +21,6 @@
 // Every mbarrier wait is bounded and reports WCC_ERR_TIMEOUT.
 #pragma once
 
-#include <type_traits>
-
 #include "common.cuh"
 #include "contract.cuh"
 #include "fused.cuh"
@@ -175,9 +173,6 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
 #pragma unroll
         for (int s = 0; s < 8; ++s) mul[s] = __fmul_rn(mul[s], sc[s]);
     }
-    // does the shrinkage keep any level-1 detail coefficient (slots 0..5) of this warp's tile?
-    const bool fine_any = __any_sync(0xFFFFFFFFu, (mul[0] != 0.0f) | (mul[1] != 0.0f) | (mul[2] != 0.0f) | (mul[3] != 0.0f) |
-                                                      (mul[4] != 0.0f) | (mul[5] != 0.0f)) != 0;
     if (I8) {                                          // dequantization factor of every output channel
         const float scale_a = __fdiv_rn(amax, pr.qmax);
         for (int o = threadIdx.x; o < pr.npad; o += C::THREADS) sscale[o] = (o < pr.Cout) ? __fmul_rn(scale_a, pr.scale_w[o]) : 0.0f;
@@ -257,21 +252,18 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
                         for (int bx = hb * (HB / C::CB); bx < (hb + 1) * (HB / C::CB); ++bx)
                             if (m + bx + C::S < my_boxes) ring.issue(&tmx, (m + bx) % C::S, x0, y0, box_c0(m + bx + C::S), n);
                     }
-                    // one group of four channels: transform, keep / drop + quantize, pack.  When the shrinkage keeps no
-                    // level-1 detail coefficient of this tile (fine_any false, the usual case at low keep ratios) only the
-                    // low-pass path is computed and only slots 6 and 7 are quantized; the other codes are zero.
-                    auto do_group = [&](int gg, auto fine_tag) {
-                        constexpr bool FINE = decltype(fine_tag)::value;
+#pragma unroll
+                    for (int gg = 0; gg < HB / 4; ++gg) {
                         const int g = hb * (HB / 4) + gg;
                         float p[4][2][4], o[4][8];
 #pragma unroll
                         for (int d = 0; d < 4; ++d) unpack_patch<T>(rawp[gg * 4 + d], p[d]);
-                        haar_fwd_lanes_raw<L, 4, FINE>(p, o, lane);
+                        haar_fwd_lanes_raw<L, 4>(p, o, lane);
                         uint32_t code[4][8];
 #pragma unroll
                         for (int d = 0; d < 4; ++d) {
 #pragma unroll
-                            for (int s = FINE ? 0 : 6; s < 8; s += 2) {
+                            for (int s = 0; s < 8; s += 2) {
                                 float2 v = mul2(make_float2(o[d][s], o[d][s + 1]), make_float2(mul[s], mul[s + 1]));
                                 // int8: the low byte of (v + 1.5*2^23) is the two's complement code of rint(v).  The sum is
                                 // written as fma(v, 1, 1.5*2^23): the product above keeps its own rounding (a packed add right
@@ -283,10 +275,7 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
                         }
 #pragma unroll
                         for (int s = 0; s < 8; ++s) {
-                            if (!FINE && s < 6) {
-                                if (I8) packed[s][g] = 0u;
-                                else { packed[s][2 * g] = 0u; packed[s][2 * g + 1] = 0u; }
-                            } else if (I8) {
+                            if (I8) {
                                 const uint32_t lo = __byte_perm(code[0][s], code[1][s], 0x0040);
                                 const uint32_t hi = __byte_perm(code[2][s], code[3][s], 0x0040);
                                 packed[s][g] = __byte_perm(lo, hi, 0x5410);
@@ -295,13 +284,6 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
                                 packed[s][2 * g + 1] = pack_bf16x2(__uint_as_float(code[2][s]), __uint_as_float(code[3][s]));
                             }
                         }
-                    };
-                    if (fine_any) {
-#pragma unroll
-                        for (int gg = 0; gg < HB / 4; ++gg) do_group(gg, std::true_type{});
-                    } else {
-#pragma unroll
-                        for (int gg = 0; gg < HB / 4; ++gg) do_group(gg, std::false_type{});
                     }
                 }
                 m += C::BPC;

@@ -321,9 +321,7 @@ __device__ __forceinline__ void slot_scales(int lane, bool swapped, float (&sc)[
     }
 }
 
-// FINE = false: the caller has no use for the level-1 detail coefficients (slots 0..5, e.g. all of them dropped by the
-// shrinkage); only the low-pass path is computed and those slots are returned as zeros.
-template <int L, int U, bool FINE = true>
+template <int L, int U>
 __device__ __forceinline__ void haar_fwd_lanes_raw(const float (&p)[U][2][4], float (&o)[U][8], int lane)
 {
     using T = HaarTile<L>;
@@ -332,16 +330,10 @@ __device__ __forceinline__ void haar_fwd_lanes_raw(const float (&p)[U][2][4], fl
     for (int u = 0; u < U; ++u) {
         const float2 a = make_float2(p[u][0][0], p[u][0][2]), b = make_float2(p[u][0][1], p[u][0][3]);
         const float2 c = make_float2(p[u][1][0], p[u][1][2]), d = make_float2(p[u][1][1], p[u][1][3]);
-        const float2 s0 = add2(a, b), s1 = add2(c, d);
+        const float2 s0 = add2(a, b), d0 = sub2(a, b), s1 = add2(c, d), d1 = sub2(c, d);
         ll[u] = add2(s0, s1);
-        if (FINE) {
-            const float2 d0 = sub2(a, b), d1 = sub2(c, d);
-            const float2 y2 = add2(d0, d1), y3 = sub2(s0, s1), y4 = sub2(d0, d1);
-            o[u][0] = y2.x; o[u][1] = y2.y; o[u][2] = y3.x; o[u][3] = y3.y; o[u][4] = y4.x; o[u][5] = y4.y;
-        } else {
-#pragma unroll
-            for (int s = 0; s < 6; ++s) o[u][s] = 0.0f;
-        }
+        const float2 y2 = add2(d0, d1), y3 = sub2(s0, s1), y4 = sub2(d0, d1);
+        o[u][0] = y2.x; o[u][1] = y2.y; o[u][2] = y3.x; o[u][3] = y3.y; o[u][4] = y4.x; o[u][5] = y4.y;
         if (L == 1) { o[u][6] = ll[u].x; o[u][7] = ll[u].y; }
     }
     if (L == 1) return;
