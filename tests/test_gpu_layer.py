@@ -152,6 +152,36 @@ def test_layer_named_workloads_full_size(wcc, name, staged):
     _run_and_compare(wcc, inputs.make(name), staged=staged)
 
 
+def test_bench_workload_as_cuda_graph_replay(wcc):
+    """The launch configuration the benchmark times: wcc_forward of workload C2 captured once in a CUDA graph and
+    replayed (with the L2 cache overwritten in between); every replay must give the oracle's output bit for bit."""
+    w = inputs.make("C2")
+    x = _x_dev(w)
+    Wt = torch.from_numpy(w.Wt).cuda()
+    y = torch.empty((w.N, w.Cout, w.H, w.W), dtype=x.dtype, device="cuda")
+    ws = wcc.Workspace.for_problem(x, w.Cout, w.levels, w.k, w.bits)
+    wcc.forward(x, Wt, w.levels, w.k, w.bits, y=y, ws=ws)          # sets kernel attributes outside the capture
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        wcc.forward(x, Wt, w.levels, w.k, w.bits, y=y, ws=ws)
+    torch.cuda.current_stream().wait_stream(side)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        wcc.forward(x, Wt, w.levels, w.k, w.bits, y=y, ws=ws)
+    want = oracle.forward(w.x_f32(), w.Wt, w.levels, w.k, w.bits, out_bf16=True)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    for rep in range(3):
+        y.fill_(float("nan"))
+        ws.buf.fill_(0xFF)                                          # nothing may depend on what the last replay left
+        flush.fill_(rep)
+        g.replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(y.float().cpu().numpy().view(np.uint32), want.view(np.uint32))
+    assert wcc.last_status() == 0
+
+
 def test_chain_of_layers_with_relu(wcc):
     """Six pointwise WCC layers 32 -> 192 -> 32 ... with ReLU in between (reduced spatial size); each layer
     is checked against the oracle fed with the GPU's own input to that layer."""
