@@ -152,6 +152,32 @@ def test_layer_named_workloads_full_size(wcc, name, staged):
     _run_and_compare(wcc, inputs.make(name), staged=staged)
 
 
+def _random_shapes(count, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for _ in range(count):
+        L = int(rng.integers(1, 4))
+        unit = 1 << L
+        H = unit * int(rng.integers(1, 6))
+        W = unit * int(rng.integers(1, 24))
+        if L == 1 and rng.random() < 0.7:
+            W = 4 * max(1, W // 4)                                    # mostly the vectorized paths
+        cfg = (int(rng.integers(1, 4)), int(rng.integers(1, 80)), int(rng.integers(1, 100)), H, W,
+               "bf16" if rng.random() < 0.5 else "f32", L, float(rng.choice([0.05, 0.125, 0.25, 0.5, 0.9])),
+               int(rng.choice([8, 8, 8, 0, 5])))
+        out.append(cfg)
+    return out
+
+
+@pytest.mark.parametrize("cfg", _random_shapes(24, 2205), ids=lambda c: "N%d_%dto%d_%dx%d_%s_L%d_g%s_b%d" % c)
+def test_layer_random_shapes(wcc, cfg):
+    """Seeded random small shapes (channel counts, tile counts, levels, types, keep ratios, bit widths drawn at random):
+    every intermediate and the output against the oracle, as for the hand-picked shapes above."""
+    N, Cin, Cout, H, W, dtype, L, gamma, bits = cfg
+    w = inputs.custom("fuzz", 11, N, Cin, Cout, H, W, dtype, L, gamma, bits, n_sin=4, fmax=3.0)
+    _run_and_compare(wcc, w)
+
+
 def test_bench_workload_as_cuda_graph_replay(wcc):
     """The launch configuration the benchmark times: wcc_forward of workload C2 captured once in a CUDA graph and
     replayed (with the L2 cache overwritten in between); every replay must give the oracle's output bit for bit."""
