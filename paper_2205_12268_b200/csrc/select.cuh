@@ -602,7 +602,8 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
     auto valid = [&](int i) { return i < kpt && base + i < P; };
 
     for (int i = threadIdx.x; i < SEL_BINS; i += blockDim.x) sm.hist[i] = 0u;
-    if (threadIdx.x == 0) { sm.amax = 0u; sm.ncand = 0u; }
+    if (threadIdx.x == 0) { sm.amax = 0u; sm.ncand = 0u; sm.thr[0] = 0xFFFFFFFFu; sm.thr[1] = 0u; sm.thr[2] = 0u; }   // thr: keep nothing
+                                                       // unless a candidate is found (histograms that do not match the keys)
     __syncthreads();
 
     uint32_t tkey = 0, need_eq = 0, total_eq = 0, ranked = 0;    // ranked: candidates counted through (diagnostic)
@@ -750,10 +751,10 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
             const bool keep = is_gt || (is_eq && eq_before < need_eq);
             const uint32_t pos = gt_before + min(eq_before, need_eq);
             if (keep) {
-                if (idx) idx[(size_t)n * k + pos] = base + i;
+                if (idx && pos < (uint32_t)k) idx[(size_t)n * k + pos] = base + i;
                 if (amaxpos) amax = fmaxf(amax, amaxpos[(size_t)n * P + base + i]);
             }
-            if (rank) rank[(size_t)n * P + base + i] = keep ? (int32_t)pos : -1;
+            if (rank) rank[(size_t)n * P + base + i] = (keep && pos < (uint32_t)k) ? (int32_t)pos : -1;
             gt_before += is_gt;
             eq_before += is_eq;
         }
