@@ -751,10 +751,10 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
             const bool keep = is_gt || (is_eq && eq_before < need_eq);
             const uint32_t pos = gt_before + min(eq_before, need_eq);
             if (keep) {
-                if (idx && pos < (uint32_t)k) idx[(size_t)n * k + pos] = base + i;
+                if (idx) idx[(size_t)n * k + pos] = base + i;
                 if (amaxpos) amax = fmaxf(amax, amaxpos[(size_t)n * P + base + i]);
             }
-            if (rank) rank[(size_t)n * P + base + i] = (keep && pos < (uint32_t)k) ? (int32_t)pos : -1;
+            if (rank) rank[(size_t)n * P + base + i] = keep ? (int32_t)pos : -1;
             gt_before += is_gt;
             eq_before += is_eq;
         }
