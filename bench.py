@@ -204,6 +204,83 @@ def whole_job_gpix(world: int, pixels_per_rank: int, ms_per_step: float) -> floa
 
 
 # ------------------------------------------------------------------------------------------------ our arm
+L2_BYTES = 126 << 20
+NOMINAL_HBM_GBS = 8000.0
+CONTEXT_WORKLOADS = ("C1", "C2", "C3", "C3u", "C4", "C4b", "C5a", "C5b")
+
+
+def layer_bytes(w):
+    """Compulsory bytes of one layer (x once, y once) and the two-pass bound (the selection forces a second look at
+    x; norms and per-position maxima written once and read once)."""
+    s = 2 if w.dtype == "bf16" else 4
+    NP = w.N * w.P
+    b_min = s * NP * (w.Cin + w.Cout)
+    return b_min, b_min + s * NP * w.Cin + 8 * NP
+
+
+class Case:
+    """One workload resident on the device: buffers, workspace, and the CUDA graph of one wcc_forward."""
+
+    def __init__(self, wcc, torch, np, w, dev, staged=False, graph=True):
+        self.wcc, self.torch, self.w, self.staged = wcc, torch, w, staged
+        if w.dtype == "bf16":
+            self.x_host = torch.from_numpy(w.x.view(np.int16)).view(torch.bfloat16).pin_memory()
+        else:
+            self.x_host = torch.from_numpy(w.x).pin_memory()
+        self.x = self.x_host.to(dev)
+        self.Wt = torch.from_numpy(w.Wt).to(dev)
+        self.y = torch.empty((w.N, w.Cout, w.H, w.W), dtype=self.x.dtype, device=dev)
+        self.y_host = torch.empty(self.y.shape, dtype=self.y.dtype).pin_memory()
+        self.ws = wcc.Workspace.for_problem(self.x, w.Cout, w.levels, w.k, w.bits, staged=staged)
+        self.pixels = w.N * w.H * w.W
+        l0 = wcc.kernel_launches()
+        self.eager()                                    # sets kernel attributes, counts launches
+        self.launches_per_step = wcc.kernel_launches() - l0
+        torch.cuda.synchronize()
+        assert wcc.last_status() == 0
+        self.graph = None
+        if graph:
+            try:
+                side = torch.cuda.Stream()
+                side.wait_stream(torch.cuda.current_stream())
+                with torch.cuda.stream(side):
+                    self.eager()
+                torch.cuda.current_stream().wait_stream(side)
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    self.eager()
+                self.graph = g
+            except Exception as e:                      # keep going eagerly, and say so
+                print("graph capture failed, timing eager launches: %r" % (e,), file=sys.stderr)
+                self.graph = None
+                torch.cuda.synchronize()
+        self.step = self.graph.replay if self.graph is not None else self.eager
+
+    def eager(self):
+        w = self.w
+        self.wcc.forward(self.x, self.Wt, w.levels, w.k, w.bits, y=self.y, ws=self.ws, staged=self.staged)
+
+    def e2e(self):
+        w = self.w
+        self.x.copy_(self.x_host, non_blocking=True)
+        self.wcc.forward(self.x, self.Wt, w.levels, w.k, w.bits, y=self.y, ws=self.ws, staged=self.staged)
+        self.y_host.copy_(self.y, non_blocking=True)
+
+    def stage_times(self, flush, steps):
+        """Mean device time of every stage, from CUDA events recorded inside eager calls (L2 flushed before each)."""
+        wcc = self.wcc
+        names = wcc.STAGES if self.staged else wcc.FUSED_STAGES
+        acc = [0.0] * len(wcc.STAGES)
+        wcc.profile_enable(True)
+        for _ in range(steps):
+            flush.fill_(1)
+            self.eager()
+            for i, v in enumerate(wcc.profile_read()):
+                acc[i] += v
+        wcc.profile_enable(False)
+        return {n: acc[i] / steps for i, n in enumerate(names)}
+
+
 def run_ours(args):
     import numpy as np
     import torch
@@ -231,61 +308,23 @@ def run_ours(args):
 
     over = {"N": args.batch} if args.batch else {}
     w = inputs.make(args.workload, seed=rank_seed(rank), **over)
-    if w.dtype == "bf16":
-        x_host = torch.from_numpy(w.x.view(np.int16)).view(torch.bfloat16).pin_memory()
-    else:
-        x_host = torch.from_numpy(w.x).pin_memory()
-    x = x_host.to(dev)
-    Wt = torch.from_numpy(w.Wt).to(dev)
-    y = torch.empty((w.N, w.Cout, w.H, w.W), dtype=x.dtype, device=dev)
-    y_host = torch.empty(y.shape, dtype=y.dtype).pin_memory()
-    ws = wcc.Workspace.for_problem(x, w.Cout, w.levels, w.k, w.bits, staged=args.staged)
+    case = Case(wcc, torch, np, w, dev, staged=args.staged, graph=not args.no_graph)
     flush = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device=dev)
-    pixels = w.N * w.H * w.W
+    warmup = max(3, args.warmup)
 
-    def step_eager():
-        wcc.forward(x, Wt, w.levels, w.k, w.bits, y=y, ws=ws, staged=args.staged)
-
-    # one eager call first: sets kernel attributes, counts launches
-    l0 = wcc.kernel_launches()
-    step_eager()
-    launches_per_step = wcc.kernel_launches() - l0
-    torch.cuda.synchronize()
-    assert wcc.last_status() == 0
-
-    graph = None
-    if not args.no_graph:
-        try:
-            side = torch.cuda.Stream()
-            side.wait_stream(torch.cuda.current_stream())
-            with torch.cuda.stream(side):
-                step_eager()
-            torch.cuda.current_stream().wait_stream(side)
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g):
-                step_eager()
-            graph = g
-        except Exception as e:                          # keep going eagerly, and say so
-            print("graph capture failed, timing eager launches: %r" % (e,), file=sys.stderr)
-            graph = None
-            torch.cuda.synchronize()
-    step = graph.replay if graph is not None else step_eager
-
-    def timed_loop(fn, steps, pre=None):
+    def timed_loop(fn, steps):
         ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
         for a, b in ev:
             flush.fill_(1)                              # evict x, y and the scratch from L2
-            if pre:
-                pre()
             a.record()
             fn()
             b.record()
         torch.cuda.synchronize()
         return [a.elapsed_time(b) for a, b in ev]
 
-    for _ in range(max(3, args.warmup)):
+    for _ in range(warmup):
         flush.fill_(1)
-        step()
+        case.step()
     torch.cuda.synchronize()
 
     sampler = ClockSampler(_physical_gpu_index(local_rank))
@@ -294,18 +333,19 @@ def run_ours(args):
         dist.barrier()
     torch.cuda.synchronize()
     t_wall0 = time.perf_counter()
-    ms = timed_loop(step, args.steps)
+    ms = timed_loop(case.step, args.steps)
     torch.cuda.synchronize()
     if dist:
         dist.barrier()
     t_wall = time.perf_counter() - t_wall0
-    clocks = sampler.stop()
+    n_timed_samples = len(sampler.samples)
     assert wcc.last_status() == 0
     total_ms = max_over_ranks(dist, float(sum(ms)), dev)
     ms_per_step = total_ms / args.steps
-    value = whole_job_gpix(world, pixels, ms_per_step)
+    value = whole_job_gpix(world, case.pixels, ms_per_step)
 
     if args.lean:                                       # profiling runs: the timed loop only
+        sampler.stop()
         if rank == 0:
             print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "ms_per_step": ms_per_step, "lean": True,
                               "config": _config_dict(w, args)}))
@@ -314,59 +354,91 @@ def run_ours(args):
         return 0
 
     # end to end through the public call: host input -> device, layer, device -> host output, every step
-    def e2e_step():
-        x.copy_(x_host, non_blocking=True)
-        wcc.forward(x, Wt, w.levels, w.k, w.bits, y=y, ws=ws, staged=args.staged)
-        y_host.copy_(y, non_blocking=True)
-
     e2e_steps = min(args.steps, 200)
     for _ in range(3):
-        e2e_step()
+        case.e2e()
     torch.cuda.synchronize()
-    e_ms = timed_loop(e2e_step, e2e_steps)
+    e_ms = timed_loop(case.e2e, e2e_steps)
     e_total = max_over_ranks(dist, float(sum(e_ms)), dev)
-    e2e_val = whole_job_gpix(world, pixels, e_total / e2e_steps)
+    e2e_val = whole_job_gpix(world, case.pixels, e_total / e2e_steps)
 
-    # per-stage device times with CUDA events recorded inside the call, same launch configuration (eager)
-    wcc.profile_enable(True)
-    prof_steps = min(args.steps, 200)
-    names = wcc.STAGES if args.staged else wcc.FUSED_STAGES
-    acc = [0.0] * len(wcc.STAGES)
-    for _ in range(prof_steps):
-        flush.fill_(1)
-        step_eager()
-        for i, v in enumerate(wcc.profile_read()):
-            acc[i] += v
-    wcc.profile_enable(False)
-    stage_ms = {n: acc[i] / prof_steps for i, n in enumerate(names)}
-    dom = max((n for n in stage_ms if n != "clear"), key=stage_ms.get)      # the memset node is not one of our kernels
+    # per-stage device times with CUDA events recorded inside the call (eager launches of the same configuration)
     peak, peak_kind = _peaks()
+    stage_ms = case.stage_times(flush, max(50, min(args.steps, 200)))
+    dom = max((n for n in stage_ms if n != "clear"), key=stage_ms.get)      # a memset node is not one of our kernels
     achieved = stage_bytes(w, dom) / (stage_ms[dom] * 1e-3) / 1e9
     tr = NCU_TRAFFIC.get((w.name, dom))
-    traffic = tr["bytes"] if tr and tr.get("src") == _source_hash() else None
-    layer_min_bytes = (2 if w.dtype == "bf16" else 4) * w.N * w.P * (w.Cin + w.Cout)
+    traffic = tr["bytes"] if tr and tr.get("src") == _source_hash() and not args.batch else None
+    b_min, b_2p = layer_bytes(w)
+    gbs = lambda nbytes, t_ms: nbytes / (t_ms * 1e-3) / 1e9
+    x_bytes = (2 if w.dtype == "bf16" else 4) * w.N * w.P * w.Cin
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": traffic, "peak_kind": "%s HBM copy bandwidth" % peak_kind,
                 "algorithmic_bytes_per_launch": stage_bytes(w, dom),
                 "stage_ms": stage_ms,
-                "stage_frac_of_peak": {n: stage_bytes(w, n) / (stage_ms[n] * 1e-3) / 1e9 / peak for n in stage_ms},
-                "layer": {"compulsory_bytes": layer_min_bytes,
-                          "frac_of_peak": layer_min_bytes / (ms_per_step * 1e-3) / 1e9 / peak}}
+                "stage_frac_of_peak": {n: gbs(stage_bytes(w, n), stage_ms[n]) / peak for n in stage_ms if stage_ms[n] > 0},
+                "x_fits_l2": x_bytes < L2_BYTES,
+                "note": ("x (%.0f MB) is smaller than the 126 MB L2, so part of the second pass's re-read of x can be served "
+                         "from L2: its fraction is algorithmic bytes over time, not DRAM throughput" % (x_bytes / 1e6))
+                        if x_bytes < L2_BYTES else "x is larger than L2: both passes stream it from DRAM",
+                "layer": {"compulsory_bytes": b_min, "two_pass_bytes": b_2p,
+                          "frac_of_peak": gbs(b_min, ms_per_step) / peak,
+                          "frac_of_two_pass_bound": gbs(b_2p, ms_per_step) / peak,
+                          "frac_of_nominal_8TBs": gbs(b_min, ms_per_step) / NOMINAL_HBM_GBS,
+                          "two_pass_frac_of_nominal_8TBs": gbs(b_2p, ms_per_step) / NOMINAL_HBM_GBS}}
 
     if rank != 0:
+        sampler.stop()
         if dist:
             dist.destroy_process_group()
         return 0
 
     # dense 1x1 convolution on the uncompressed map (library kernel), for context
-    dense_ms = None
-    try:
-        xd = x.reshape(w.N, w.Cin, w.P)
-        Wd = Wt.to(x.dtype)
-        torch.matmul(Wd, xd)
-        dense_ms = statistics.median(timed_loop(lambda: torch.matmul(Wd, xd), 50))
-    except Exception:
-        pass
+    def dense_ms_of(c):
+        try:
+            xd = c.x.reshape(c.w.N, c.w.Cin, c.w.P)
+            Wd = c.Wt.to(c.x.dtype)
+            torch.matmul(Wd, xd)
+            return statistics.median(timed_loop(lambda: torch.matmul(Wd, xd), 50))
+        except Exception:
+            return None
+
+    dense_ms = dense_ms_of(case)
+
+    # every other workload, briefly: graph replay time, stage times, fractions (single GPU context, not the headline)
+    workloads = {}
+    if not args.batch and not args.no_context:
+        ctx_steps = 200
+        for name in CONTEXT_WORKLOADS:
+            if name == w.name and not args.staged:
+                c, c_ms = case, ms
+            else:
+                c = Case(wcc, torch, np, inputs.make(name), dev, graph=not args.no_graph)
+                for _ in range(3):
+                    flush.fill_(1)
+                    c.step()
+                c_ms = timed_loop(c.step, ctx_steps)
+            t = sum(c_ms) / len(c_ms)
+            st = stage_ms if c is case else c.stage_times(flush, 100)
+            bm, b2 = layer_bytes(c.w)
+            workloads[name] = {
+                "config": _config_dict(c.w, args)["workload"], "steps": len(c_ms), "ms_per_step": t,
+                "Gpix/s": c.pixels / (t * 1e-3) / 1e9,
+                "layer_frac_of_peak": gbs(bm, t) / peak, "layer_frac_of_two_pass_bound": gbs(b2, t) / peak,
+                "layer_frac_of_nominal_8TBs": gbs(bm, t) / NOMINAL_HBM_GBS,
+                "stage_ms": st,
+                "stage_frac_of_peak": {n: gbs(stage_bytes(c.w, n), st[n]) / peak for n in st if st[n] > 0},
+                "dense_1x1_matmul_ms": dense_ms if c is case else dense_ms_of(c),
+                "x_fits_l2": (2 if c.w.dtype == "bf16" else 4) * c.w.N * c.w.P * c.w.Cin < L2_BYTES}
+            if c is not case:
+                del c
+                torch.cuda.empty_cache()
+        assert wcc.last_status() == 0
+    clocks_all = sampler.stop()
+    timed = sampler.samples[:max(1, n_timed_samples)]
+    clocks = {"sm_mhz": (statistics.median(timed) if timed else None), "sm_max_mhz": clocks_all["sm_max_mhz"],
+              "reasons": clocks_all["reasons"], "samples": len(timed),
+              "whole_run": {"sm_mhz": clocks_all["sm_mhz"], "samples": clocks_all["samples"]}}
 
     # the oracle on the host cores: a bounded sample of the same workload
     import oracle
@@ -380,24 +452,24 @@ def run_ours(args):
     for _ in range(reps):
         oracle.forward(xo, w.Wt, w.levels, w.k, w.bits, out_bf16=(w.dtype == "bf16"))
     t_cpu = (time.perf_counter() - t0) / reps
-    cpu = {"value": pixels / t_cpu / 1e9, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+    cpu = {"value": case.pixels / t_cpu / 1e9, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
            "sample": "the full workload, %d repetitions (%.1f s of CPU work)" % (reps, t_cpu * reps)}
 
-    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
            "dtype": "f32 transform, int8 x int8 -> int32 contraction" if w.bits else "f32 transform, bf16 contraction",
            "data": "synthetic",
            "config": _config_dict(w, args, l2="flushed before every step by a %d MiB write outside the step's events" % (FLUSH_BYTES >> 20),
-                                  launch=("CUDA graph replay of one %s" if graph is not None else "eager %s") % (
+                                  launch=("CUDA graph replay of one %s" if case.graph is not None else "eager %s") % (
                                       "wcc_forward_staged" if args.staged else "wcc_forward"),
                                   wall_s_timed_region=t_wall),
            "clocks": clocks,
-           "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": x_host.numel() * x_host.element_size(),
-                   "d2h_bytes_per_step": y_host.numel() * y_host.element_size(), "steps": e2e_steps},
-           "gpu_launches": int(launches_per_step * args.steps),
+           "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": case.x_host.numel() * case.x_host.element_size(),
+                   "d2h_bytes_per_step": case.y_host.numel() * case.y_host.element_size(), "steps": e2e_steps},
+           "gpu_launches": int(case.launches_per_step * args.steps),
            "roofline": roofline, "cpu_baseline": cpu,
            "context": {"dense_1x1_matmul_ms": dense_ms, "ms_per_step_median": statistics.median(ms),
-                       "ms_per_step_min": min(ms)}}
+                       "ms_per_step_min": min(ms), "workloads": workloads}}
     print(json.dumps(out))
     if dist:
         dist.destroy_process_group()
@@ -409,11 +481,12 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="C2")
+    ap.add_argument("--workload", default="C4")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="time eager wcc_forward calls instead of a graph replay")
     ap.add_argument("--batch", type=int, default=0, help="override the number of images per GPU")
     ap.add_argument("--lean", action="store_true", help="timed loop only (for runs under a profiler)")
+    ap.add_argument("--no-context", action="store_true", help="skip the brief runs of the other workloads")
     ap.add_argument("--staged", action="store_true", help="time wcc_forward_staged (every intermediate in memory)")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -61,7 +61,7 @@ size_t wcc_select_workspace_bytes(int N, int P);
 
 /*
  * Forward Haar transform, all levels, of every (n, c) plane (Eq. 3, 5, 6), and in the same pass the
- * feature norm across channels of every position (Alg. 1, "vector norm along the channel dimension").
+ * per-position l2 norm over the channels (Alg. 1, norm step).
  *   x     in : [N][C][H][Wd] of dt
  *   coef  out: fp32 [N][C][H][Wd], quadrant layout.  Arithmetic is fp32: per 2x2 block a,b / c,d:
  *              s0=a+b d0=a-b s1=c+d d1=c-d; y1=(s0+s1)/2 y2=(d0+d1)/2 y3=(s0-s1)/2 y4=(d0-d1)/2.
@@ -81,7 +81,7 @@ wcc_status wcc_haar_inv(const float* coef, int N, int C, int H, int Wd, int leve
                         void* x_out, void* stream);
 
 /*
- * Joint shrinkage T (Eq. 7; Alg. 1 "top ceil(gamma n_w n_h) vectors by norm"): for each image the k
+ * Joint shrinkage T (Eq. 7; Alg. 1, index-set step): for each image the k = ceil(gamma * H * Wd)
  * positions of largest norm.  Ties at the k-th value go to the lowest position.  -0 ranks equal to +0;
  * the order of NaNs is unspecified.
  *   nrm2 in : fp32 [N][P]
@@ -179,6 +179,19 @@ wcc_status wcc_forward_staged(const void* x, const float* Wt, int N, int Cin, in
 wcc_status wcc_last_status(void* stream);
 
 const char* wcc_status_str(wcc_status s);
+
+/*
+ * Test hooks for the device-side timeout contract (no counterpart in the paper).  Every wait inside a kernel (on an
+ * mbarrier of a TMA ring, of the tensor-core pipeline, on the arrival counter of the cooperative select) polls a
+ * bounded number of times, then the kernel records WCC_ERR_TIMEOUT, lets its copies in flight land, frees its TMEM
+ * and returns; nothing traps or faults.
+ *   wcc_debug_set_wait_limit  sets the number of polls (each suspends for up to about a microsecond) on the current
+ *                             device; 0 restores the default (2,000,000).  Synchronous.
+ *   wcc_debug_wait_selftest   enqueues one warp that waits on a barrier nobody arrives on; with a small limit it
+ *                             returns within a millisecond and wcc_last_status then reports WCC_ERR_TIMEOUT.
+ */
+wcc_status wcc_debug_set_wait_limit(unsigned polls);
+wcc_status wcc_debug_wait_selftest(void* stream);
 
 /*
  * Measurement helpers (no counterpart in the paper).  With profiling on, wcc_forward records CUDA events on its

@@ -151,8 +151,7 @@ void SUF(orc_concat_order)(const REAL *coef, int H, int W, int levels, REAL *vec
 }
 
 /*
- * Feature norm across channels at every wavelet-domain position (Alg. 1, "vector norm
- * along the channel dimension"): the squared l2 norm, accumulated as one fused
+ * Feature norm across channels at every wavelet-domain position (Alg. 1, norm step): the squared l2 norm, accumulated as one fused
  * multiply-add per channel in ascending channel order starting from +0.
  * Ranking by the squared norm equals ranking by the norm.
  */
@@ -171,8 +170,8 @@ void SUF(orc_norms)(const REAL *coef, int N, int C, long P, REAL *nrm2)
 }
 
 /*
- * Joint shrinkage T (Eq. 7 with the joint rule of Sec. 4; Alg. 1 "top ceil(gamma n_w n_h)
- * vectors by norm"): for every image, order the positions by (norm descending, position
+ * Joint shrinkage T (Eq. 7 with the joint rule of Sec. 4; Alg. 1, index-set step with
+ * k = ceil(gamma n_w n_h)): for every image, order the positions by (norm descending, position
  * ascending), keep the first k, and report them in ascending position.  tau[n] is the
  * k-th largest norm.  A full sort: nothing clever.
  */

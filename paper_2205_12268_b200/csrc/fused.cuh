@@ -357,6 +357,30 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
 
 static inline size_t vmax(size_t a, size_t b) { return a > b ? a : b; }
 
+// Host-side plan of the one-tile kernel (pure arithmetic; ok = the problem fits its shared memory).
+struct FzPlan { int npad, nchunk, tmem_cols, a_ksteps; size_t smem; bool ok; };
+
+static FzPlan fz_plan(int esz, int Cout, int kpad, int bits)
+{
+    FzPlan p = {};
+    const bool i8 = bits >= 2;
+    const int es = i8 ? 1 : 2;
+    p.npad = ceil_div(Cout, 16) * 16;
+    p.nchunk = p.npad < 64 ? p.npad : 64;
+    p.tmem_cols = 32;
+    while (p.tmem_cols < 2 * p.nchunk) p.tmem_cols <<= 1;
+    const int kchunks = kpad * es / 16;
+    const int ksteps = kpad * es / 32;
+    // two K halves when that brings A down enough for a fourth CTA per SM (single chunk of output channels only)
+    p.a_ksteps = (p.npad <= p.nchunk && ksteps >= 4) ? (ksteps + 1) / 2 : ksteps;
+    const size_t stage_bytes = (size_t)((esz == 2) ? 4 : 2) * 2 * 32 * 4 * esz;          // PatchRing<T>::STAGE_BYTES
+    const size_t region = vmax((size_t)fz::SUB * 8 * 32 * 4, (size_t)4 * fz::RING2 * stage_bytes);
+    p.smem = 128 + (size_t)p.a_ksteps * 2 * fz::ROWS * 16 + (size_t)kchunks * p.npad * 16 + 8 * 32 * 4 + sizeof(fz::Ctl) +
+             region + 16;
+    p.ok = p.smem <= 200 * 1024 && (kpad * es) % 32 == 0;
+    return p;
+}
+
 template <typename T, int L, bool VEC>
 static wcc_status fused_pass2_dispatch(const void* x, const void* Wq, const int32_t* rank, const float* nrm2,
                                        const uint32_t* thr, const float* amax_kept, int bits,
@@ -364,20 +388,12 @@ static wcc_status fused_pass2_dispatch(const void* x, const void* Wq, const int3
                                        void* y, void* xq_tap, int32_t* acc_tap, cudaStream_t st)
 {
     using TT = HaarTile<L>;
+    static_assert(PatchRing<T>::STAGE_BYTES == ((sizeof(T) == 2) ? 4 : 2) * 2 * 32 * 4 * (int)sizeof(T), "fz_plan mirrors PatchRing");
     const bool i8 = bits >= 2;
-    const int es = i8 ? 1 : 2;
-    const int npad = ceil_div(Cout, 16) * 16;
-    const int nchunk = npad < 64 ? npad : 64;
-    int tmem_cols = 32;
-    while (tmem_cols < 2 * nchunk) tmem_cols <<= 1;
-    const int kchunks = kpad * es / 16;
-    const int ksteps = kpad * es / 32;
-    // two K halves when that brings A down enough for a fourth CTA per SM (single chunk of output channels only)
-    const int a_ksteps = (npad <= nchunk && ksteps >= 4) ? (ksteps + 1) / 2 : ksteps;
-    const size_t region = vmax((size_t)fz::SUB * 8 * 32 * 4, (size_t)4 * fz::RING2 * PatchRing<T>::STAGE_BYTES);
-    const size_t smem = 128 + (size_t)a_ksteps * 2 * fz::ROWS * 16 + (size_t)kchunks * npad * 16 + 8 * 32 * 4 + sizeof(fz::Ctl) +
-                        region + 16;
-    if (smem > 200 * 1024 || (kpad * es) % 32 != 0) return WCC_ERR_SHAPE;
+    const FzPlan plan = fz_plan((int)sizeof(T), Cout, kpad, bits);
+    if (!plan.ok) return WCC_ERR_SHAPE;
+    const int npad = plan.npad, nchunk = plan.nchunk, tmem_cols = plan.tmem_cols, a_ksteps = plan.a_ksteps;
+    const size_t smem = plan.smem;
     const float qmax = i8 ? (float)((1 << (bits - 1)) - 1) : 1.0f;
     int* status = nullptr;
     WCC_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_status));

@@ -391,6 +391,32 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
 
 }  // namespace ft
 
+// Host-side plan of the four-tile kernel: how the output channels are chunked, how many operand buffers and TMEM
+// columns it takes, and whether the problem fits at all (ok).  Pure arithmetic: callers decide before anything is launched.
+struct FtPlan { int npad, nchunk, nn, nbuf, na, tmem_cols; size_t smem; bool ok; };
+
+static FtPlan ft_plan(const void* x, int esz, int W, int Cout, int kpad, int bits)
+{
+    constexpr int WPT = 2, S = 4;                     // as instantiated below (Cfg<T, I8, 2>::S)
+    FtPlan p = {};
+    const bool i8 = bits >= 2;
+    const int es = i8 ? 1 : 2;
+    if ((W % 4) != 0 || !tc::tma_ok_x(x, esz, W) || (kpad * es) % 32 != 0) return p;
+    p.npad = ceil_div(Cout, 16) * 16;
+    const int kchunks = kpad * es / 16, ksteps = kpad * es / 32;
+    if (p.npad <= 64) { p.nchunk = p.npad; p.nn = 1; p.nbuf = 1; p.na = ksteps < 2 ? ksteps : 2; }
+    else { p.nchunk = 32; p.nn = ceil_div(p.npad, 32); p.nbuf = 2; p.na = ksteps; }
+    if (p.na > ft::MAX_NA) return p;
+    p.tmem_cols = 32;
+    while (p.tmem_cols < 8 * p.nchunk * p.nbuf) p.tmem_cols <<= 1;
+    if (p.tmem_cols > 512) return p;
+    const size_t ring_bytes = (size_t)ft::TILES * WPT * S * 4096;
+    p.smem = 128 + (size_t)p.na * ft::KSTEP_BYTES + ring_bytes + (size_t)kchunks * p.npad * 16 +
+             (size_t)ft::TILES * WPT * 8 * 8 + sizeof(ft::Ctl) + (size_t)p.npad * 4 + 64;
+    p.ok = p.smem <= 227 * 1024;
+    return p;
+}
+
 // Returns WCC_ERR_SHAPE when this kernel does not cover the problem (the caller then uses fused_pass2_kernel).
 template <typename T, int L>
 static wcc_status fused_tiles_dispatch(const void* x, const void* Wq, const int32_t* rank, const float* nrm2, const uint32_t* thr,
@@ -399,22 +425,13 @@ static wcc_status fused_tiles_dispatch(const void* x, const void* Wq, const int3
 {
     using TT = HaarTile<L>;
     constexpr int WPT = 2;
+    static_assert(ft::Cfg<T, true, WPT>::S == 4 && ft::Cfg<T, false, WPT>::S == 4, "ft_plan assumes four boxes per ring");
     const bool i8 = bits >= 2;
-    const int es = i8 ? 1 : 2;
-    if (!tc::tma_ok_x(x, (int)sizeof(T), W) || (kpad * es) % 32 != 0) return WCC_ERR_SHAPE;
+    const FtPlan plan = ft_plan(x, (int)sizeof(T), W, Cout, kpad, bits);
+    if (!plan.ok) return WCC_ERR_SHAPE;
     ft::Params pr = {};
-    pr.npad = ceil_div(Cout, 16) * 16;
-    const int kchunks = kpad * es / 16, ksteps = kpad * es / 32;
-    if (pr.npad <= 64) { pr.nchunk = pr.npad; pr.nn = 1; pr.nbuf = 1; pr.na = ksteps < 2 ? ksteps : 2; }
-    else { pr.nchunk = 32; pr.nn = ceil_div(pr.npad, 32); pr.nbuf = 2; pr.na = ksteps; }
-    if (pr.na > ft::MAX_NA) return WCC_ERR_SHAPE;
-    pr.tmem_cols = 32;
-    while (pr.tmem_cols < 8 * pr.nchunk * pr.nbuf) pr.tmem_cols <<= 1;
-    if (pr.tmem_cols > 512) return WCC_ERR_SHAPE;
-    const size_t ring_bytes = (size_t)ft::TILES * WPT * (i8 ? ft::Cfg<T, true, WPT>::S : ft::Cfg<T, false, WPT>::S) * 4096;
-    const size_t smem = 128 + (size_t)pr.na * ft::KSTEP_BYTES + ring_bytes + (size_t)kchunks * pr.npad * 16 +
-                        (size_t)ft::TILES * WPT * 8 * 8 + sizeof(ft::Ctl) + (size_t)pr.npad * 4 + 64;
-    if (smem > 227 * 1024) return WCC_ERR_SHAPE;
+    pr.npad = plan.npad; pr.nchunk = plan.nchunk; pr.nn = plan.nn; pr.nbuf = plan.nbuf; pr.na = plan.na; pr.tmem_cols = plan.tmem_cols;
+    const size_t smem = plan.smem;
     const long long tiles = (long long)N * ceil_div(W, TT::TW) * (H / TT::TH);
     if (tiles > 0x7FFFFFFFLL) return WCC_ERR_SHAPE;
     CUtensorMap tmx;

@@ -1021,7 +1021,7 @@ haar_norms_token_kernel(const __grid_constant__ CUtensorMap tmx, int N, int C, i
             // the token: partial sums of the boxes before this one
             float2 acc[4];
             if (r > 0) {
-                ok = tc::mbar_wait(tc::smem_u32(&tok_bars[warp]), (uint32_t)tok_seen & 1u);
+                ok = ok && tc::mbar_wait(tc::smem_u32(&tok_bars[warp]), (uint32_t)tok_seen & 1u);
                 ++tok_seen;
                 const float4 t0 = token[lane], t1 = token[32 + lane];
                 acc[0] = make_float2(t0.x, t0.y); acc[1] = make_float2(t0.z, t0.w);

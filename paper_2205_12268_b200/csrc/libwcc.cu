@@ -33,6 +33,23 @@ static wcc_status check_forward_args(int N, int Cin, int Cout, int H, int W, int
     return WCC_OK;
 }
 
+// Can one of the two fused second-pass kernels run this problem?  (x only enters through its alignment.)
+static bool fused_fits(const void* x, int Cout, int W, int bits, wcc_dtype dt, int Cin)
+{
+    const int esz = (dt == WCC_BF16) ? 2 : 4, kpad = wcc_kpad(Cin, bits);
+    return ft_plan(x, esz, W, Cout, kpad, bits).ok || fz_plan(esz, Cout, kpad, bits).ok;
+}
+
+// Can the staged contraction kernel run it?  (Mirrors launch_contract.)
+static bool staged_fits(int Cin, int Cout, int bits)
+{
+    const int krow_bytes = wcc_kpad(Cin, bits) * (bits >= 2 ? 1 : 2);
+    const int katoms = ceil_div(krow_bytes, tc::ATOM_BYTES), npad = ceil_div(Cout, 16) * 16;
+    if (katoms > tc::MAX_KATOMS || npad > 256 || (krow_bytes % 32) != 0) return false;
+    const size_t smem = 1024 + (size_t)katoms * npad * tc::ATOM_BYTES + (size_t)tc::STAGES * katoms * tc::A_ATOM_BYTES + sizeof(tc::SmemCtl) + 16;
+    return smem <= 200 * 1024;
+}
+
 struct FwdWs {
     float* coef; float* nrm2; float* amaxpos; int32_t* rank; int32_t* idx; void* sel; size_t sel_bytes;
     float* amax_kept; void* Xq; void* Wq; float* scale_w; int32_t* acc;
@@ -103,6 +120,20 @@ static wcc_status profile_mark(int i, cudaStream_t st)
     return WCC_OK;
 }
 
+// One warp waits on an mbarrier that nobody ever arrives on: the bounded wait runs out, the kernel records
+// WCC_ERR_TIMEOUT in the status word and returns normally (no trap, no fault).
+__global__ void wait_selftest_kernel(int* status)
+{
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        tc::mbar_init(tc::smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    const bool ok = tc::mbar_wait(tc::smem_u32(&bar), 0u);
+    if (!__all_sync(0xFFFFFFFFu, ok ? 1 : 0) && threadIdx.x == 0) atomicExch(status, (int)WCC_ERR_TIMEOUT);
+}
+
 __global__ void scale_tap_kernel(const float* amax_kept, float qmax, float* out) { *out = __fdiv_rn(*amax_kept, qmax); }
 
 static wcc_status staged_impl(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int W,
@@ -113,6 +144,7 @@ static wcc_status staged_impl(const void* x, const float* Wt, int N, int Cin, in
     wcc_status s = check_forward_args(N, Cin, Cout, H, W, L, k, bits, dt);
     if (s != WCC_OK) return s;
     if (!aligned16(x) || !aligned16(Wt) || !aligned16(y) || (reinterpret_cast<uintptr_t>(ws) & 255u)) return WCC_ERR_ALIGN;
+    if (!staged_fits(Cin, Cout, bits)) return WCC_ERR_SHAPE;          // decided before anything is launched
     const FwdWs f = carve_forward_ws(ws, N, Cin, Cout, H, W, k, bits);
     if (ws_bytes < f.total) return WCC_ERR_WORKSPACE;
     const int P = H * W, M = N * k;
@@ -208,6 +240,7 @@ static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, i
     if (!aligned16(x) || !aligned16(Wt) || !aligned16(y) || (reinterpret_cast<uintptr_t>(ws) & 255u)) return WCC_ERR_ALIGN;
     if (taps && (!aligned16(taps->coef) || !aligned16(taps->Xq) || !aligned16(taps->Xb) || !aligned16(taps->acc)))
         return WCC_ERR_ALIGN;
+    if (!fused_fits(x, Cout, W, bits, dt, Cin)) return WCC_ERR_SHAPE;   // decided before anything is launched
     const FusedWs f = carve_fused_ws(ws, N, Cin, Cout, H, W, k, bits);
     if (ws_bytes < f.total) return WCC_ERR_WORKSPACE;
     const int P = H * W, M = N * k;
@@ -274,12 +307,14 @@ int wcc_kpad(int Cin, int bits)
 size_t wcc_workspace_bytes(int N, int Cin, int Cout, int H, int Wd, int levels, int k, int bits, wcc_dtype dt)
 {
     if (check_forward_args(N, Cin, Cout, H, Wd, levels, k, bits, dt) != WCC_OK) return 0;
+    if (!fused_fits(nullptr, Cout, Wd, bits, dt, Cin)) return 0;
     return carve_fused_ws(nullptr, N, Cin, Cout, H, Wd, k, bits).total;
 }
 
 size_t wcc_staged_workspace_bytes(int N, int Cin, int Cout, int H, int Wd, int levels, int k, int bits, wcc_dtype dt)
 {
     if (check_forward_args(N, Cin, Cout, H, Wd, levels, k, bits, dt) != WCC_OK) return 0;
+    if (!staged_fits(Cin, Cout, bits)) return 0;
     return carve_forward_ws(nullptr, N, Cin, Cout, H, Wd, k, bits).total;
 }
 
@@ -369,6 +404,22 @@ wcc_status wcc_last_status(void* stream)
         if (cudaMemcpyToSymbol(g_status, &zero, sizeof(int)) != cudaSuccess) return WCC_ERR_CUDA;
     }
     return static_cast<wcc_status>(v);
+}
+
+wcc_status wcc_debug_set_wait_limit(unsigned polls)
+{
+    const uint32_t v = polls ? (uint32_t)polls : tc::WAIT_LIMIT_DEFAULT;
+    if (cudaMemcpyToSymbol(tc::c_wait_limit, &v, sizeof(v)) != cudaSuccess) return WCC_ERR_CUDA;
+    return WCC_OK;
+}
+
+wcc_status wcc_debug_wait_selftest(void* stream)
+{
+    int* status = nullptr;
+    WCC_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_status));
+    wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(status);
+    WCC_LAUNCH_CHECK();
+    return WCC_OK;
 }
 
 wcc_status wcc_profile_enable(int on)

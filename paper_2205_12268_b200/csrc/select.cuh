@@ -13,6 +13,7 @@
 #include <cooperative_groups.h>
 
 #include "common.cuh"
+#include "tma.cuh"
 
 namespace wcc {
 namespace cg = cooperative_groups;
@@ -296,7 +297,6 @@ select_compact_kernel(const float* __restrict__ nrm2, int P, int k, const uint32
 // All phases in one launch; the CTAs of an image meet at per-image barriers (an arrival counter in global memory,
 // a bounded spin).  The launch is cooperative, so every CTA is resident and the barriers can complete.  The keys
 // stay in registers across the phases.
-constexpr uint32_t SEL_SPIN_LIMIT = 4000000u;
 
 __device__ __forceinline__ bool image_barrier(uint32_t* counter, uint32_t target)
 {
@@ -306,7 +306,8 @@ __device__ __forceinline__ bool image_barrier(uint32_t* counter, uint32_t target
         __threadfence();
         atomicAdd(counter, 1u);
         int ok = 0;
-        for (uint32_t it = 0; it < SEL_SPIN_LIMIT; ++it) {
+        const uint32_t limit = 2u * tc::c_wait_limit;               // polls of >= 40 ns
+        for (uint32_t it = 0; it < limit; ++it) {
             if (*reinterpret_cast<volatile uint32_t*>(counter) >= target) { ok = 1; break; }
             __nanosleep(40);
         }
@@ -357,7 +358,10 @@ select_coop_kernel(const float* __restrict__ nrm2, int P, int k, uint32_t* __res
 #pragma unroll
     for (int i = 0; i < SEL_KPT; ++i) hist_add(sh, key[i] >> 21, okk[i]);
     flush_hist<SEL_BINS>(sh, hn);
-    bool good = image_barrier(barn, chunks);
+    // A barrier that ran out leaves the histograms incomplete: report it and leave at once (the decision is uniform
+    // over the block), so that nothing is derived from them and no index is written.
+    auto give_up = [&]() { if (threadIdx.x == 0) atomicExch(status, (int)WCC_ERR_TIMEOUT); };
+    if (!image_barrier(barn, chunks)) { give_up(); return; }
     // round 2
     uint32_t b1, above;
     find_bin<SEL_BINS>(hn, (uint32_t)k, sh_scan, sh_res, b1, above);
@@ -365,7 +369,7 @@ select_coop_kernel(const float* __restrict__ nrm2, int P, int k, uint32_t* __res
 #pragma unroll
     for (int i = 0; i < SEL_KPT; ++i) hist_add(sh, (key[i] >> 10) & 0x7FFu, okk[i] && (key[i] >> 21) == b1);
     flush_hist<SEL_BINS>(sh, hn + SEL_BINS);
-    good = image_barrier(barn, 2 * chunks) && good;
+    if (!image_barrier(barn, 2 * chunks)) { give_up(); return; }
     // round 3
     uint32_t b2;
     find_bin<SEL_BINS>(hn + SEL_BINS, k1, sh_scan, sh_res, b2, above);
@@ -374,7 +378,7 @@ select_coop_kernel(const float* __restrict__ nrm2, int P, int k, uint32_t* __res
 #pragma unroll
     for (int i = 0; i < SEL_KPT; ++i) hist_add(sh, key[i] & 0x3FFu, okk[i] && (key[i] >> 10) == prefix);
     flush_hist<1024>(sh, hn + 2 * SEL_BINS);
-    good = image_barrier(barn, 3 * chunks) && good;
+    if (!image_barrier(barn, 3 * chunks)) { give_up(); return; }
     // threshold, chunk counts
     uint32_t b3;
     find_bin<1024>(hn + 2 * SEL_BINS, k2, sh_scan, sh_res, b3, above);
@@ -392,7 +396,7 @@ select_coop_kernel(const float* __restrict__ nrm2, int P, int k, uint32_t* __res
     const uint32_t eq_local = block_exclusive_scan(eq, sh_scan, &tot_eq);
     uint32_t* cc = chunkcnt + (size_t)n * chunks * 2;
     if (threadIdx.x == 0) { cc[2 * blockIdx.x] = tot_gt; cc[2 * blockIdx.x + 1] = tot_eq; }
-    good = image_barrier(barn, 4 * chunks) && good;
+    if (!image_barrier(barn, 4 * chunks)) { give_up(); return; }
     // ordered compaction
     {
         uint32_t g = 0, e = 0;
@@ -416,7 +420,7 @@ select_coop_kernel(const float* __restrict__ nrm2, int P, int k, uint32_t* __res
         const bool is_gt = key[i] > tkey, is_eq = key[i] == tkey;
         const bool keep = is_gt || (is_eq && eq_before < need_eq);
         const uint32_t pos = gt_before + min(eq_before, need_eq);
-        if (keep) {
+        if (keep && pos < (uint32_t)k) {
             idx[(size_t)n * k + pos] = base + i;
             if (amaxpos) amax = fmaxf(amax, amaxpos[(size_t)n * P + base + i]);
         }
@@ -431,7 +435,6 @@ select_coop_kernel(const float* __restrict__ nrm2, int P, int k, uint32_t* __res
         __syncthreads();
         if (threadIdx.x == 0 && sh_amax) atomicMax(reinterpret_cast<uint32_t*>(amax_kept), sh_amax);
     }
-    if (!good && threadIdx.x == 0) atomicExch(status, (int)WCC_ERR_TIMEOUT);
 }
 
 // ---- the select as one thread-block cluster per image -------------------------------------------------

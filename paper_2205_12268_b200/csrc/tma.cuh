@@ -9,7 +9,11 @@
 namespace wcc {
 namespace tc {
 
-constexpr uint32_t WAIT_LIMIT = 2000000u;       // polls of <= ~1 us each
+// Every device-side wait polls at most c_wait_limit times (each poll suspends for up to ~1 us), then gives up and the
+// kernel reports WCC_ERR_TIMEOUT.  A constant-bank word so that reading it costs nothing on the fast path; the host
+// can lower it (wcc_debug_set_wait_limit) to exercise the timeout path in a millisecond.
+constexpr uint32_t WAIT_LIMIT_DEFAULT = 2000000u;
+__constant__ uint32_t c_wait_limit = WAIT_LIMIT_DEFAULT;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -38,7 +42,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 // Bounded wait.  Returns false when the limit ran out or another role already gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
 {
-    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+    const uint32_t limit = c_wait_limit;
+    for (uint32_t it = 0; it < limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
     }
@@ -57,7 +62,8 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm,
 // Same bounded wait without an abort flag (a warp that waits only for its own copies).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 {
-    for (uint32_t it = 0; it < WAIT_LIMIT; ++it)
+    const uint32_t limit = c_wait_limit;
+    for (uint32_t it = 0; it < limit; ++it)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }

@@ -20,7 +20,8 @@ _STATUS = {0: "ok", 1: "null pointer", 2: "bad shape", 3: "k out of range", 4: "
 
 EXPORTS = ("wcc_staged_workspace_bytes", "wcc_forward_staged", "wcc_workspace_bytes", "wcc_select_workspace_bytes", "wcc_haar_fwd", "wcc_haar_inv", "wcc_select_topk",
            "wcc_forward", "wcc_forward_debug", "wcc_kpad", "wcc_last_status", "wcc_status_str",
-           "wcc_profile_enable", "wcc_profile_read", "wcc_kernel_launches", "wcc_select_topk_static")
+           "wcc_profile_enable", "wcc_profile_read", "wcc_kernel_launches", "wcc_select_topk_static",
+           "wcc_debug_set_wait_limit", "wcc_debug_wait_selftest")
 STATIC_SCRATCH_BYTES = 512 * 1024
 STAGES = ("haar_fwd_norms", "select_topk", "weight_quant", "gather_quant", "contract", "scatter_inv")   # wcc_forward_staged
 FUSED_STAGES = ("clear", "haar_norms", "select_topk", "fused_pass2")                                      # wcc_forward
@@ -79,6 +80,10 @@ def lib() -> C.CDLL:
         L.wcc_profile_read.argtypes = [C.POINTER(C.c_float)]
         L.wcc_kernel_launches.restype = C.c_ulonglong
         L.wcc_kernel_launches.argtypes = []
+        L.wcc_debug_set_wait_limit.restype = i
+        L.wcc_debug_set_wait_limit.argtypes = [C.c_uint]
+        L.wcc_debug_wait_selftest.restype = i
+        L.wcc_debug_wait_selftest.argtypes = [vp]
         L.wcc_status_str.restype = C.c_char_p
         L.wcc_status_str.argtypes = [i]
         _lib = L
@@ -233,6 +238,16 @@ def forward(x: torch.Tensor, Wt: torch.Tensor, levels: int, k: int, bits: int = 
 def last_status() -> int:
     """Synchronises the current stream and returns (and clears) the device status word."""
     return int(lib().wcc_last_status(_stream()))
+
+
+def debug_set_wait_limit(polls: int):
+    """Polls every device-side wait makes before it gives up (0 restores the default)."""
+    _check(lib().wcc_debug_set_wait_limit(int(polls)), "wcc_debug_set_wait_limit")
+
+
+def debug_wait_selftest():
+    """Enqueues one warp that waits on a barrier nobody arrives on (it gives up after the wait limit)."""
+    _check(lib().wcc_debug_wait_selftest(_stream()), "wcc_debug_wait_selftest")
 
 
 def profile_enable(on: bool):

@@ -208,10 +208,7 @@ def test_bench_workload_as_cuda_graph_replay(wcc):
     assert wcc.last_status() == 0
 
 
-def test_chain_of_layers_with_relu(wcc):
-    """Six pointwise WCC layers 32 -> 192 -> 32 ... with ReLU in between (reduced spatial size); each layer
-    is checked against the oracle fed with the GPU's own input to that layer."""
-    N, H, W, L, gamma = 2, 64, 128, 3, 0.25
+def _chain(wcc, N, H, W, L, gamma):
     first = inputs.custom("chain", 0, N, 32, 192, H, W, "bf16", L, gamma, 8, n_sin=16, fmax=8.0)
     x = _x_dev(first)
     chans = [32, 192, 32, 192, 32, 192, 32]
@@ -219,9 +216,51 @@ def test_chain_of_layers_with_relu(wcc):
         Wt_np = inputs.weights(100 + i, chans[i + 1], chans[i])
         y = wcc.forward(x, torch.from_numpy(Wt_np).cuda(), L, first.k, 8)
         want = oracle.forward(x.float().cpu().numpy(), Wt_np, L, first.k, 8, out_bf16=True)
-        assert np.array_equal(y.float().cpu().numpy().view(np.uint32), want.view(np.uint32))
+        assert np.array_equal(y.float().cpu().numpy().view(np.uint32), want.view(np.uint32)), i
         x = torch.relu(y)
     assert wcc.last_status() == 0
+
+
+def test_chain_of_layers_with_relu(wcc):
+    """Six pointwise WCC layers 32 -> 192 -> 32 ... with ReLU in between (reduced spatial size); each layer
+    is checked against the oracle fed with the GPU's own input to that layer."""
+    _chain(wcc, 2, 64, 128, 3, 0.25)
+
+
+def test_chain_of_layers_with_relu_full_size(wcc):
+    """The same chain at the benchmark's size (2 x 256 x 512)."""
+    _chain(wcc, 2, 256, 512, 3, 0.25)
+
+
+_C5_CACHE = {}
+
+
+def _c5_workload(cin, cout):
+    """The two layer shapes of the six-layer chain workload at full size (inputs generated once per shape)."""
+    if (cin, cout) not in _C5_CACHE:
+        _C5_CACHE[(cin, cout)] = inputs.custom("C5", 0, 2, cin, cout, 256, 512, "bf16", 3, 0.25, 8, n_sin=16, fmax=8.0)
+    return _C5_CACHE[(cin, cout)]
+
+
+@pytest.mark.parametrize("gamma", [0.5, 0.25, 0.125, 0.0625], ids=lambda g: "g%s" % g)
+@pytest.mark.parametrize("L", [1, 2, 3], ids=lambda l: "L%d" % l)
+@pytest.mark.parametrize("shape", [(32, 192), (192, 32)], ids=lambda c: "%dto%d" % c)
+def test_layer_config5_sweep_full_size(wcc, shape, L, gamma):
+    """Every (levels, keep ratio) point of the chain workload's sweep, both layer shapes, 2 x 256 x 512 bf16: output
+    bit for bit against the oracle; at the 1/16 points also every intermediate (many accumulator chunks per tile group
+    at one and two levels, where a tile is a thin strip of the image)."""
+    import copy
+    w = copy.copy(_c5_workload(*shape))
+    w.levels = L
+    w.k = inputs.keep_count(gamma, w.P)
+    if gamma == 0.0625:
+        _run_and_compare(wcc, w)
+        return
+    x = _x_dev(w)
+    y = wcc.forward(x, torch.from_numpy(w.Wt).cuda(), L, w.k, 8)
+    assert wcc.last_status() == 0
+    want = oracle.forward(w.x_f32(), w.Wt, L, w.k, 8, out_bf16=True)
+    assert np.array_equal(y.float().cpu().numpy().view(np.uint32), want.view(np.uint32))
 
 
 def test_workspace_too_small_is_rejected(wcc):
