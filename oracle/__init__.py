@@ -36,6 +36,7 @@ def _L():
     if _lib is None:
         _lib = C.CDLL(build())
         _lib.orc_quantize.restype = C.c_float
+        _lib.orc_quantize_alpha.restype = C.c_float
     return _lib
 
 
@@ -137,9 +138,20 @@ def round_bf16(a: np.ndarray) -> np.ndarray:
     return out
 
 
+def quantize_alpha(x: np.ndarray, alpha: float, bits: int = 8):
+    """The same quantizer with a given clipping parameter (values beyond +-alpha clip) -> (int8 codes, scale)."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    q = np.empty(x.shape, dtype=np.int8)
+    s = _L().orc_quantize_alpha(_p(x, C.c_float), C.c_long(x.size), bits, C.c_float(alpha), _p(q, C.c_int8))
+    return q, np.float32(s)
+
+
 def forward(x: np.ndarray, Wt: np.ndarray, levels: int, k: int, bits: int, out_bf16: bool = False,
-            idx_in: np.ndarray | None = None, taps: bool = False):
-    """The WCC layer in fp32.  Returns y, or (y, dict of taps) when ``taps`` is set."""
+            idx_in: np.ndarray | None = None, taps: bool = False, wbits: int | None = None, alpha: float = 0.0,
+            residual: np.ndarray | None = None, relu: bool = False):
+    """The WCC layer in fp32.  Returns y, or (y, dict of taps) when ``taps`` is set.
+    Options: ``wbits`` bits of the weight codes (default: ``bits``), ``alpha`` > 0 a given clipping parameter of the
+    activation quantizer (default: the largest kept magnitude), ``residual`` a map added to the output, ``relu``."""
     x = np.ascontiguousarray(x, dtype=np.float32)
     Wt = np.ascontiguousarray(Wt, dtype=np.float32)
     N, Cin, H, W = x.shape
@@ -158,15 +170,34 @@ def forward(x: np.ndarray, Wt: np.ndarray, levels: int, k: int, bits: int, out_b
     if idx_in is not None:
         idx_in = np.ascontiguousarray(idx_in, dtype=np.int32)
         assert idx_in.shape == (N, k)
-    rc = _L().orc_forward_f32(
-        _p(x, C.c_float), _p(Wt, C.c_float), N, Cin, Cout, H, W, levels, k, bits, int(out_bf16),
+    if residual is not None:
+        residual = np.ascontiguousarray(residual, dtype=np.float32)
+        assert residual.shape == y.shape
+    rc = _L().orc_forward_ex_f32(
+        _p(x, C.c_float), _p(Wt, C.c_float), N, Cin, Cout, H, W, levels, k, bits, bits if wbits is None else wbits,
+        C.c_float(alpha), _p(residual, C.c_float), int(relu), int(out_bf16),
         _p(idx_in, C.c_int32), _p(y, C.c_float),
         _p(t.get("coef"), C.c_float), _p(t.get("nrm2"), C.c_float), _p(t.get("idx"), C.c_int32),
         _p(t.get("Xq"), C.c_int8), _p(t.get("scale_a"), C.c_float), _p(t.get("Wq"), C.c_int8),
         _p(t.get("scale_w"), C.c_float), _p(t.get("acc"), C.c_int32))
     if rc:
-        raise ValueError("orc_forward_f32 rc=%d" % rc)
+        raise ValueError("orc_forward_ex_f32 rc=%d" % rc)
     return (y, t) if taps else y
+
+
+def chain(x: np.ndarray, weights, levels: int, k: int, bits: int = 8, out_bf16: bool = False, relu_last: bool = False,
+          alphas=None):
+    """A chain of pointwise WCC layers with a ReLU after every layer but (unless ``relu_last``) the last: layer i maps
+    the previous layer's output with ``weights[i]`` ([Cout_i][Cin_i]).  ``alphas[i]`` > 0 gives layer i a fixed
+    clipping parameter.  Nothing but a loop over ``forward``.  Returns the list of the layers' outputs."""
+    outs = []
+    cur = np.ascontiguousarray(x, dtype=np.float32)
+    for i, Wt in enumerate(weights):
+        last = i == len(weights) - 1
+        cur = forward(cur, Wt, levels, k, bits, out_bf16=out_bf16, relu=(relu_last or not last),
+                      alpha=0.0 if alphas is None else float(alphas[i]))
+        outs.append(cur)
+    return outs
 
 
 def forward_f64(x: np.ndarray, Wt: np.ndarray, levels: int, k: int, idx_in: np.ndarray | None = None,

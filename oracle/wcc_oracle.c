@@ -65,14 +65,26 @@ void orc_round_bf16(const float *in, long n, float *out)
  * multiplication by inv = qmax/alpha; round is to nearest, ties to even.
  * Returns the step (scale); codes are written to q.
  */
+float orc_quantize_alpha(const float *x, long n, int bits, float alpha, int8_t *q);
+
 float orc_quantize(const float *x, long n, int bits, int8_t *q)
 {
-    const float qmax = (float)((1 << (bits - 1)) - 1);
     float amax = 0.0f;
     for (long i = 0; i < n; ++i) {
         const float a = fabsf(x[i]);
         if (a > amax) amax = a;
     }
+    return orc_quantize_alpha(x, n, bits, amax, q);
+}
+
+/*
+ * The same quantizer with the clipping parameter given (Eq. 2: alpha is a parameter of the layer, learned during
+ * training; here it is an argument).  Values beyond +-alpha are clipped: their codes are +-qmax.
+ */
+float orc_quantize_alpha(const float *x, long n, int bits, float alpha, int8_t *q)
+{
+    const float qmax = (float)((1 << (bits - 1)) - 1);
+    const float amax = alpha;
     const float inv = (amax > 0.0f) ? qmax / amax : 0.0f;
     for (long i = 0; i < n; ++i) {
         float r = nearbyintf(x[i] * inv);
@@ -83,7 +95,7 @@ float orc_quantize(const float *x, long n, int bits, int8_t *q)
     return amax / qmax;
 }
 
-/* Weights: one clipping parameter per output channel (row of Wt[Cout][Cin]). */
+/* Weights: one clipping parameter per output channel (row of Wt[Cout][Cin]), the row's largest magnitude. */
 void orc_quantize_weights(const float *Wt, int Cout, int Cin, int bits, int8_t *Wq, float *scale_w)
 {
     for (int o = 0; o < Cout; ++o)
@@ -103,14 +115,41 @@ void orc_quantize_weights(const float *Wt, int Cout, int Cin, int bits, int8_t *
  * Optional taps (NULL to skip): coef [N][Cin][P], nrm2 [N][P], idx [N][k], Xq int8 [N][k][Cin],
  *  scale_a [1], Wq int8 [Cout][Cin], scale_w [Cout], acc int32 [N][k][Cout].
  */
+int orc_forward_ex_f32(const float *x, const float *Wt, int N, int Cin, int Cout, int H, int W,
+                       int levels, int k, int bits, int wbits, float alpha, const float *residual, int relu,
+                       int out_bf16, const int32_t *idx_in, float *y,
+                       float *coef_tap, float *nrm2_tap, int32_t *idx_tap, int8_t *Xq_tap,
+                       float *scale_a_tap, int8_t *Wq_tap, float *scale_w_tap, int32_t *acc_tap);
+
 int orc_forward_f32(const float *x, const float *Wt, int N, int Cin, int Cout, int H, int W,
                     int levels, int k, int bits, int out_bf16, const int32_t *idx_in, float *y,
                     float *coef_tap, float *nrm2_tap, int32_t *idx_tap, int8_t *Xq_tap,
                     float *scale_a_tap, int8_t *Wq_tap, float *scale_w_tap, int32_t *acc_tap)
 {
+    return orc_forward_ex_f32(x, Wt, N, Cin, Cout, H, W, levels, k, bits, bits, 0.0f, NULL, 0, out_bf16, idx_in, y,
+                              coef_tap, nrm2_tap, idx_tap, Xq_tap, scale_a_tap, Wq_tap, scale_w_tap, acc_tap);
+}
+
+/*
+ * The layer with the options a network built from it uses:
+ *  wbits     bits of the weight codes (the paper also runs 4-bit weights with 8-bit activations, Tables 1-2)
+ *  alpha     > 0: the clipping parameter of the activation quantizer (Eq. 2), one for the whole layer (Sec. 4);
+ *            <= 0: the largest kept magnitude of this call
+ *  residual  NULL, or a map [N][Cout][H][W] added to the layer's output (the skip connection of the inverted
+ *            residual block, Eq. 13): one fp32 addition per element, after the inverse transform
+ *  relu      non-zero: max(., 0) after the addition (the non-linearity between chained layers)
+ * The output is rounded to bf16 last, when asked.
+ */
+int orc_forward_ex_f32(const float *x, const float *Wt, int N, int Cin, int Cout, int H, int W,
+                       int levels, int k, int bits, int wbits, float alpha, const float *residual, int relu,
+                       int out_bf16, const int32_t *idx_in, float *y,
+                       float *coef_tap, float *nrm2_tap, int32_t *idx_tap, int8_t *Xq_tap,
+                       float *scale_a_tap, int8_t *Wq_tap, float *scale_w_tap, int32_t *acc_tap)
+{
     const long P = (long)H * W;
     if (k < 1 || k > P) return -1;
     if (!(bits == 0 || (bits >= 2 && bits <= 8))) return -1;
+    if (bits > 0 && !(wbits >= 2 && wbits <= 8)) return -1;
     const size_t nk = (size_t)N * k;
     float *coef = (float *)malloc(sizeof(float) * (size_t)N * Cin * P);
     float *nrm2 = (float *)malloc(sizeof(float) * (size_t)N * P);
@@ -139,8 +178,9 @@ int orc_forward_f32(const float *x, const float *Wt, int N, int Cin, int Cout, i
 
     /* C: the 1x1 convolution on the compressed columns */
     if (bits > 0) {
-        const float scale_a = orc_quantize(Xc, (long)(nk * Cin), bits, Xq);   /* one alpha for the layer */
-        orc_quantize_weights(Wt, Cout, Cin, bits, Wq, scale_w);
+        const float scale_a = (alpha > 0.0f) ? orc_quantize_alpha(Xc, (long)(nk * Cin), bits, alpha, Xq)
+                                             : orc_quantize(Xc, (long)(nk * Cin), bits, Xq);   /* one alpha for the layer */
+        orc_quantize_weights(Wt, Cout, Cin, wbits, Wq, scale_w);
 #pragma omp parallel for schedule(static)
         for (long r = 0; r < (long)nk; ++r)
             for (int o = 0; o < Cout; ++o) {
@@ -173,6 +213,10 @@ int orc_forward_f32(const float *x, const float *Wt, int N, int Cin, int Cout, i
     /* E: inverse Haar transform */
     rc = orc_haar_inv_f32(Ywt, N, Cout, H, W, levels, y);
     if (rc) goto done;
+    if (residual)
+        for (size_t i = 0; i < (size_t)N * Cout * P; ++i) y[i] = y[i] + residual[i];
+    if (relu)
+        for (size_t i = 0; i < (size_t)N * Cout * P; ++i) y[i] = (y[i] > 0.0f) ? y[i] : 0.0f;
     if (out_bf16) orc_round_bf16(y, (long)N * Cout * P, y);
 
     if (coef_tap) memcpy(coef_tap, coef, sizeof(float) * (size_t)N * Cin * P);
