@@ -162,6 +162,53 @@ wcc_status wcc_forward_debug(const void* x, const float* Wt, int N, int Cin, int
                              void* ws, size_t ws_bytes, void* stream, const wcc_taps* taps);
 
 /*
+ * Options of the layer beyond Alg. 1, as a network built from WCC layers uses them.  A zeroed structure (or NULL)
+ * means wcc_forward.
+ *   alpha        > 0: the clipping parameter of the activation quantizer (Eq. 2; per layer, Sec. 4 -- in the paper it is
+ *                learned, here it is an argument): codes = clamp(rint(v * (qmax / alpha)), -qmax, qmax), scale_a =
+ *                alpha / qmax, so kept coefficients beyond +-alpha saturate.  <= 0: the largest kept magnitude of this
+ *                call, as in wcc_forward.  Ignored when bits == 0.
+ *   weight_bits  0: as `bits`; 2..8: bits of the weight codes (Tables 1-2 run 4-bit weights with 8-bit activations).
+ *   relu         non-zero: y = max(., 0), applied last before rounding to dt (the non-linearity between chained layers).
+ *   residual     NULL, or a DEVICE map [N][Cout][H][Wd] of dt added to the layer's output before the ReLU: the skip
+ *                connection of the inverted residual block (Eq. 13); one fp32 addition per element.  May be y itself.
+ *   Wq, scale_w  NULL, or the weights already quantized (DEVICE): int8 [Cout][wcc_kpad(Cin, bits)], rows zero padded,
+ *                and fp32 [Cout] scales (what taps Wq / scale_w return).  Static weights need quantizing only once;
+ *                Wt is then not read and may be NULL.  Only with bits >= 2.
+ */
+typedef struct wcc_options {
+    float alpha;
+    int weight_bits;
+    int relu;
+    const void* residual;
+    const int8_t* Wq;
+    const float* scale_w;
+} wcc_options;
+
+/* wcc_forward with options (opt may be NULL) and optional taps (may be NULL).  Same workspace as wcc_forward. */
+wcc_status wcc_forward_ex(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int Wd,
+                          int levels, int k, int bits, void* y, wcc_dtype dt,
+                          void* ws, size_t ws_bytes, void* stream, const wcc_options* opt, const wcc_taps* taps);
+
+/*
+ * A chain of pointwise WCC layers on one feature map (e.g. the 32 -> 192 -> 32 ... stacks of an inverted-residual
+ * network): layer i maps the output of layer i-1 with Wt [Cout][Cin]; Cin of a layer must equal Cout of the one before.
+ * `layers` is a HOST array (read during the call only); Wt are DEVICE pointers.  relu / alpha as in wcc_options.
+ * Same levels, k and bits for every layer.  Intermediate maps live in the workspace (two buffers of the largest one).
+ * All arguments of all layers are checked before the first launch.
+ */
+typedef struct wcc_chain_layer {
+    const float* Wt;
+    int Cin, Cout;
+    float alpha;
+    int relu;
+} wcc_chain_layer;
+size_t wcc_chain_workspace_bytes(const wcc_chain_layer* layers, int n_layers, int N, int H, int Wd, int levels, int k,
+                                 int bits, wcc_dtype dt);
+wcc_status wcc_chain_forward(const void* x, const wcc_chain_layer* layers, int n_layers, int N, int H, int Wd,
+                             int levels, int k, int bits, void* y, wcc_dtype dt, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * The same layer as wcc_forward computed stage by stage with every intermediate in memory (Alg. 1 literally):
  * transform + norms -> select -> gather + quantize -> tensor-core contraction on the compressed matrix ->
  * dequantize + scatter + inverse.  Same results as wcc_forward; used to measure the stages one by one and as a

@@ -48,6 +48,29 @@ __device__ __forceinline__ void tmem_ld8_nowait(uint32_t taddr, uint32_t (&r)[8]
                  : "r"(taddr));
 }
 
+// y = WCC(x) + residual: one fp32 addition per element of the lane's patch (Eq. 13)
+template <typename T, bool VEC>
+__device__ __forceinline__ void add_residual(const T* __restrict__ plane, int W, const LanePos& lp, float (&p)[2][4])
+{
+    RawPatch rr;
+    float rp[2][4];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) rr.w[i] = 0u;
+    load_patch<T, VEC>(plane, W, lp, rr);
+    unpack_patch<T>(rr, rp);
+#pragma unroll
+    for (int a = 0; a < 2; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) p[a][b] = __fadd_rn(p[a][b], rp[a][b]);
+}
+__device__ __forceinline__ void relu_patch(float (&p)[2][4])
+{
+#pragma unroll
+    for (int a = 0; a < 2; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) p[a][b] = fmaxf(p[a][b], 0.0f);
+}
+
 struct Ctl {
     uint64_t mma_done;
     uint32_t tmem_base;
@@ -59,7 +82,8 @@ __global__ void __launch_bounds__(128, 4)
 fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, const int32_t* __restrict__ rank,
                    const float* __restrict__ nrm2, const uint32_t* __restrict__ thr, const float* __restrict__ amax_kept, float qmax, const float* __restrict__ scale_w,
                    int N, int Cin, int Cout, int H, int W, int k, int kpad, int npad, int nchunk, int tmem_cols, int a_ksteps,
-                   T* __restrict__ y, uint8_t* __restrict__ xq_tap, int32_t* __restrict__ acc_tap, int* __restrict__ status)
+                   T* __restrict__ y, uint8_t* __restrict__ xq_tap, int32_t* __restrict__ acc_tap, int* __restrict__ status,
+                   float alpha, int relu, const T* __restrict__ residual)
 {
     using TT = HaarTile<L>;
     constexpr int ES = I8 ? 1 : 2;                    // operand element size
@@ -141,7 +165,7 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
     }
     float inv = 0.0f, scale_a = 1.0f;
     if (I8) {
-        const float amax = *amax_kept;
+        const float amax = (alpha > 0.0f) ? alpha : *amax_kept;
         inv = (amax > 0.0f) ? __fdiv_rn(qmax, amax) : 0.0f;
         scale_a = __fdiv_rn(amax, qmax);
     } else {
@@ -220,6 +244,10 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
 #pragma unroll
                     for (int s = 0; s < 8; s += 2) {
                         float2 t = mul2(make_float2(o[dd4][s], o[dd4][s + 1]), make_float2(mul[s], mul[s + 1]));
+                        if (I8 && alpha > 0.0f) {          // a given clipping parameter can be exceeded: clamp to the grid
+                            t.x = fminf(fmaxf(t.x, -qmax), qmax);
+                            t.y = fminf(fmaxf(t.y, -qmax), qmax);
+                        }
                         // int8: the low byte of (t + 1.5*2^23) is the two's complement code of rint(t); |t| <= qmax by
                         // construction.  Scalar adds on purpose: a packed add right after the packed product gets
                         // contracted into one fused operation, which rounds once and changes half-way codes.
@@ -335,7 +363,12 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
 #pragma unroll
                 for (int jj = 0; jj < SUB / 4; ++jj) {
                     const int o = n0 + s0 + warp + 4 * jj;
-                    if (o < Cout) store_patch<T, VEC>(y + ((size_t)n * Cout + o) * P, W, lp, p[jj]);
+                    if (o < Cout) {
+                        const size_t plane = ((size_t)n * Cout + o) * P;
+                        if (residual) add_residual<T, VEC>(residual + plane, W, lp, p[jj]);
+                        if (relu) relu_patch(p[jj]);
+                        store_patch<T, VEC>(y + plane, W, lp, p[jj]);
+                    }
                 }
             }
             __syncthreads();
@@ -356,6 +389,9 @@ fused_pass2_kernel(const T* __restrict__ x, const uint8_t* __restrict__ Wq, cons
 }  // namespace fz
 
 static inline size_t vmax(size_t a, size_t b) { return a > b ? a : b; }
+
+// Options of the fused second pass beyond Alg. 1: a given clipping parameter, residual add and ReLU on the way out.
+struct FusedExtra { float alpha; int relu; const void* residual; };
 
 // Host-side plan of the one-tile kernel (pure arithmetic; ok = the problem fits its shared memory).
 struct FzPlan { int npad, nchunk, tmem_cols, a_ksteps; size_t smem; bool ok; };
@@ -385,7 +421,7 @@ template <typename T, int L, bool VEC>
 static wcc_status fused_pass2_dispatch(const void* x, const void* Wq, const int32_t* rank, const float* nrm2,
                                        const uint32_t* thr, const float* amax_kept, int bits,
                                        const float* scale_w, int N, int Cin, int Cout, int H, int W, int k, int kpad,
-                                       void* y, void* xq_tap, int32_t* acc_tap, cudaStream_t st)
+                                       void* y, void* xq_tap, int32_t* acc_tap, const FusedExtra& fx, cudaStream_t st)
 {
     using TT = HaarTile<L>;
     static_assert(PatchRing<T>::STAGE_BYTES == ((sizeof(T) == 2) ? 4 : 2) * 2 * 32 * 4 * (int)sizeof(T), "fz_plan mirrors PatchRing");
@@ -403,7 +439,8 @@ static wcc_status fused_pass2_dispatch(const void* x, const void* Wq, const int3
         WCC_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
         kern<<<(unsigned)ctas, 128, smem, st>>>(static_cast<const T*>(x), static_cast<const uint8_t*>(Wq), rank, nrm2, thr, amax_kept,
                                                 qmax, scale_w, N, Cin, Cout, H, W, k, kpad, npad, nchunk, tmem_cols, a_ksteps,
-                                                static_cast<T*>(y), static_cast<uint8_t*>(xq_tap), acc_tap, status);
+                                                static_cast<T*>(y), static_cast<uint8_t*>(xq_tap), acc_tap, status,
+                                                fx.alpha, fx.relu, static_cast<const T*>(fx.residual));
         WCC_LAUNCH_CHECK();
         return WCC_OK;
     };
@@ -415,11 +452,11 @@ static wcc_status fused_pass2_dispatch(const void* x, const void* Wq, const int3
 wcc_status launch_fused_pass2(const void* x, const void* Wq, const int32_t* rank, const float* nrm2, const uint32_t* thr,
                               const float* amax_kept, int bits,
                               const float* scale_w, int N, int Cin, int Cout, int H, int W, int L, int k, int kpad,
-                              wcc_dtype dt, void* y, void* xq_tap, int32_t* acc_tap, cudaStream_t st)
+                              wcc_dtype dt, void* y, void* xq_tap, int32_t* acc_tap, const FusedExtra& fx, cudaStream_t st)
 {
     const bool vec = (W % 4) == 0;
     WCC_DISPATCH_TLV(fused_pass2_dispatch, dt, L, vec, x, Wq, rank, nrm2, thr, amax_kept, bits, scale_w, N, Cin, Cout, H, W, k, kpad,
-                     y, xq_tap, acc_tap, st);
+                     y, xq_tap, acc_tap, fx, st);
 }
 
 }  // namespace wcc

@@ -57,6 +57,9 @@ struct Cfg {
 struct Params {
     const uint8_t* Wq; const int32_t* rank; const float* nrm2; const uint32_t* thr; const float* amax_kept;
     const float* scale_w; float qmax;
+    float alpha;                 // > 0: given clipping parameter of the activation quantizer (codes are clamped)
+    int relu;                    // non-zero: y = max(., 0)
+    const void* residual;        // NULL, or [N][Cout][H][W] of the activation type, added before the ReLU
     int N, Cin, Cout, H, W, k, kpad, npad, nchunk, nn, nbuf, tmem_cols, na, tiles_total;
     void* y; uint8_t* xq_tap; int32_t* acc_tap; int* status;
 };
@@ -150,7 +153,7 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
     for (int s = 0; s < 8; ++s) { mul[s] = 0.0f; rk[s] = -1; }
     // all independent loads first (threshold, norms, max |kept|), so that their latencies overlap
     float amax = 0.0f;
-    if (I8) amax = *pr.amax_kept;
+    if (I8) amax = (pr.alpha > 0.0f) ? pr.alpha : *pr.amax_kept;
     if (live) {
         const uint4 th = *reinterpret_cast<const uint4*>(pr.thr + n * 4);      // {threshold key, ties kept, use-rank flag, -}
         float nv[8];
@@ -228,6 +231,8 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
         __syncwarp();
     } else {
         // ---- phase 1: transform + quantize into the A operand ---------------------------------------------
+        const bool clamp = I8 && pr.alpha > 0.0f;      // a given clipping parameter can be exceeded
+        const float qmax = pr.qmax;
         int m = 0;                                     // boxes consumed so far
         for (int ci = 0; ci < my_chunks && ok; ++ci) {
             const int j = q + ci * WPT, ks = j >> 1, jj = j & 1, buf = ks % pr.na;
@@ -268,6 +273,8 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
                                 // int8: the low byte of (v + 1.5*2^23) is the two's complement code of rint(v).  The sum is
                                 // written as fma(v, 1, 1.5*2^23): the product above keeps its own rounding (a packed add right
                                 // after the packed product gets contracted into one fused operation, which changes half-way codes).
+                                // clamping before the rounding is the same as after it: the bounds are integers
+                                if (clamp) { v.x = fminf(fmaxf(v.x, -qmax), qmax); v.y = fminf(fmaxf(v.y, -qmax), qmax); }
                                 if (I8) v = __ffma2_rn(v, make_float2(1.0f, 1.0f), make_float2(fz::MAGIC, fz::MAGIC));
                                 code[d][s] = __float_as_uint(v.x);
                                 code[d][s + 1] = __float_as_uint(v.y);
@@ -314,6 +321,7 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
 
         // ---- phase 3: accumulators -> dequantize -> inverse transform -> y ---------------------------------
         T* yout = static_cast<T*>(pr.y);
+        const T* res = static_cast<const T*>(pr.residual);
         const bool coarse6 = L == 3 && ((lane / TT::CG) & 1) == 0;     // slot 6 holds a level-3 coefficient
         for (int c = 0; c < pr.nn && ok; ++c) {
             const int tb = c % pr.nbuf;
@@ -361,7 +369,12 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
 #pragma unroll
                     for (int d = 0; d < 4; ++d) {
                         const int o = o0 + hh * 4 + d;
-                        if (o < pr.Cout) store_patch<T, true>(yout + ((size_t)n * pr.Cout + o) * P, pr.W, lp, p[d]);
+                        if (o < pr.Cout) {
+                            const size_t plane = ((size_t)n * pr.Cout + o) * P;
+                            if (res) fz::add_residual<T, true>(res + plane, pr.W, lp, p[d]);
+                            if (pr.relu) fz::relu_patch(p[d]);
+                            store_patch<T, true>(yout + plane, pr.W, lp, p[d]);
+                        }
                     }
                 }
             }
@@ -421,7 +434,8 @@ static FtPlan ft_plan(const void* x, int esz, int W, int Cout, int kpad, int bit
 template <typename T, int L>
 static wcc_status fused_tiles_dispatch(const void* x, const void* Wq, const int32_t* rank, const float* nrm2, const uint32_t* thr,
                                        const float* amax_kept, int bits, const float* scale_w, int N, int Cin, int Cout, int H,
-                                       int W, int k, int kpad, void* y, void* xq_tap, int32_t* acc_tap, cudaStream_t st)
+                                       int W, int k, int kpad, void* y, void* xq_tap, int32_t* acc_tap, const FusedExtra& fx,
+                                       cudaStream_t st)
 {
     using TT = HaarTile<L>;
     constexpr int WPT = 2;
@@ -440,6 +454,7 @@ static wcc_status fused_tiles_dispatch(const void* x, const void* Wq, const int3
     pr.scale_w = scale_w; pr.qmax = i8 ? (float)((1 << (bits - 1)) - 1) : 1.0f;
     pr.N = N; pr.Cin = Cin; pr.Cout = Cout; pr.H = H; pr.W = W; pr.k = k; pr.kpad = kpad; pr.tiles_total = (int)tiles;
     pr.y = y; pr.xq_tap = static_cast<uint8_t*>(xq_tap); pr.acc_tap = acc_tap;
+    pr.alpha = fx.alpha; pr.relu = fx.relu; pr.residual = fx.residual;
     WCC_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&pr.status), g_status));
     const unsigned ctas = (unsigned)((tiles + ft::TILES - 1) / ft::TILES);
     auto launch = [&](auto kern, int threads) -> wcc_status {
@@ -454,10 +469,11 @@ static wcc_status fused_tiles_dispatch(const void* x, const void* Wq, const int3
 
 wcc_status launch_fused_tiles(const void* x, const void* Wq, const int32_t* rank, const float* nrm2, const uint32_t* thr,
                               const float* amax_kept, int bits, const float* scale_w, int N, int Cin, int Cout, int H, int W,
-                              int L, int k, int kpad, wcc_dtype dt, void* y, void* xq_tap, int32_t* acc_tap, cudaStream_t st)
+                              int L, int k, int kpad, wcc_dtype dt, void* y, void* xq_tap, int32_t* acc_tap, const FusedExtra& fx,
+                              cudaStream_t st)
 {
     if ((W % 4) != 0) return WCC_ERR_SHAPE;
-#define WCC_FT(TY, LL) return fused_tiles_dispatch<TY, LL>(x, Wq, rank, nrm2, thr, amax_kept, bits, scale_w, N, Cin, Cout, H, W, k, kpad, y, xq_tap, acc_tap, st)
+#define WCC_FT(TY, LL) return fused_tiles_dispatch<TY, LL>(x, Wq, rank, nrm2, thr, amax_kept, bits, scale_w, N, Cin, Cout, H, W, k, kpad, y, xq_tap, acc_tap, fx, st)
     if (dt == WCC_F32) { if (L == 1) WCC_FT(float, 1); if (L == 2) WCC_FT(float, 2); WCC_FT(float, 3); }
     if (L == 1) WCC_FT(__nv_bfloat16, 1);
     if (L == 2) WCC_FT(__nv_bfloat16, 2);

@@ -956,17 +956,23 @@ haar_norms_token_kernel(const __grid_constant__ CUtensorMap tmx, int N, int C, i
     const int total = iters * mine;
     Ring ring;
     ring.init(stages, ring_bars + warp * S, lane);
-    auto issue_box = [&](int mg) {                     // lane 0 only; mg counts this warp's boxes over all its tiles
-        const int it = mg / mine, mi = mg - it * mine;
-        int n_, ty_, tx_;
-        tile_coords((int)blockIdx.x + it * tile_ctas, tiles_x, tiles_y, n_, ty_, tx_);
-        ring.issue(&tmx, mg % S, tx_ * TT::TW, ty_ * TT::TH, (warp + mi * NW) * CB, n_);
+    // The next box to request, kept as running counters (a division per box would cost more issue slots than the
+    // transform of the box's channels): box `iss_mi` of this warp in tile (iss_n, iss_ty, iss_tx), into stage `iss_stage`.
+    int iss_mi = 0, iss_it = 0, iss_stage = 0, iss_n = 0, iss_ty = 0, iss_tx = 0, issued = 0;
+    tile_coords((int)blockIdx.x, tiles_x, tiles_y, iss_n, iss_ty, iss_tx);
+    auto issue_next = [&]() {                          // all lanes keep the counters, lane 0 talks to the TMA unit
+        if (issued >= total) return;
+        if (lane == 0) ring.issue(&tmx, iss_stage, iss_tx * TT::TW, iss_ty * TT::TH, (warp + iss_mi * NW) * CB, iss_n);
+        ++issued;
+        if (++iss_stage == S) iss_stage = 0;
+        if (++iss_mi == mine) {
+            iss_mi = 0;
+            ++iss_it;
+            tile_coords((int)blockIdx.x + iss_it * tile_ctas, tiles_x, tiles_y, iss_n, iss_ty, iss_tx);
+        }
     };
-    if (lane == 0) {
 #pragma unroll
-        for (int m = 0; m < S; ++m)
-            if (m < total) issue_box(m);
-    }
+    for (int m = 0; m < S; ++m) issue_next();
     if (threadIdx.x == 0) {
 #pragma unroll
         for (int i = 0; i < NW; ++i) tc::mbar_init(tc::smem_u32(&tok_bars[i]), 1);
@@ -977,7 +983,9 @@ haar_norms_token_kernel(const __grid_constant__ CUtensorMap tmx, int N, int C, i
     float sc[8];
     slot_scales<L>(lane, ring.swap, sc);
     bool ok = true;
-    int mg = 0, tok_seen = 0;                          // boxes consumed / tokens received so far
+    int tok_seen = 0;                                  // tokens received so far
+    int stage = 0;                                     // stage of the next box to consume, and its barrier's parity
+    uint32_t parity = 0;
     for (int it = 0; it < iters; ++it) {
         int n, ty, tx;
         tile_coords((int)blockIdx.x + it * tile_ctas, tiles_x, tiles_y, n, ty, tx);
@@ -985,9 +993,9 @@ haar_norms_token_kernel(const __grid_constant__ CUtensorMap tmx, int N, int C, i
         float amax[8];
 #pragma unroll
         for (int s = 0; s < 8; ++s) amax[s] = 0.0f;
-        for (int m = 0; m < mine && ok; ++m, ++mg) {
-            const int r = warp + m * NW, stage = mg % S;
-            ok = ring.wait(stage, (uint32_t)(mg / S) & 1u);
+        for (int m = 0; m < mine && ok; ++m) {
+            const int r = warp + m * NW;
+            ok = ring.wait(stage, parity);
             RawPatch raw[CB];
 #pragma unroll
             for (int d = 0; d < CB; ++d) ring.read_raw(stage, d, raw[d]);      // channels beyond C arrive as zeros: fma(0, 0, acc) = acc
@@ -1005,7 +1013,8 @@ haar_norms_token_kernel(const __grid_constant__ CUtensorMap tmx, int N, int C, i
                 }
             }
             __syncwarp();                              // every lane is done reading the stage
-            if (lane == 0 && mg + S < total) issue_box(mg + S);
+            issue_next();                              // refills exactly this stage (S boxes are always in flight)
+            if (++stage == S) { stage = 0; parity ^= 1u; }
             float o[CB][8];
 #pragma unroll
             for (int g = 0; g < CB / 4; ++g) {

@@ -134,7 +134,10 @@ __global__ void wait_selftest_kernel(int* status)
     if (!__all_sync(0xFFFFFFFFu, ok ? 1 : 0) && threadIdx.x == 0) atomicExch(status, (int)WCC_ERR_TIMEOUT);
 }
 
-__global__ void scale_tap_kernel(const float* amax_kept, float qmax, float* out) { *out = __fdiv_rn(*amax_kept, qmax); }
+__global__ void scale_tap_kernel(const float* amax_kept, float alpha, float qmax, float* out)
+{
+    *out = __fdiv_rn(alpha > 0.0f ? alpha : *amax_kept, qmax);
+}
 
 static wcc_status staged_impl(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int W,
                                int L, int k, int bits, void* y, wcc_dtype dt, void* ws, size_t ws_bytes,
@@ -183,7 +186,7 @@ static wcc_status staged_impl(const void* x, const float* Wt, int N, int Cin, in
             if (taps->Wq) WCC_CUDA_TRY(cudaMemcpyAsync(taps->Wq, f.Wq, (size_t)Cout * f.kpad, dd, st));
             if (taps->scale_w) WCC_CUDA_TRY(cudaMemcpyAsync(taps->scale_w, f.scale_w, (size_t)Cout * 4, dd, st));
             if (taps->scale_a) {
-                scale_tap_kernel<<<1, 1, 0, st>>>(f.amax_kept, (float)((1 << (bits - 1)) - 1), taps->scale_a);
+                scale_tap_kernel<<<1, 1, 0, st>>>(f.amax_kept, 0.0f, (float)((1 << (bits - 1)) - 1), taps->scale_a);
                 WCC_LAUNCH_CHECK();
             }
         } else if (taps->Xb) {
@@ -230,13 +233,28 @@ static FusedWs carve_fused_ws(void* ws, int N, int Cin, int Cout, int H, int W, 
     return f;
 }
 
+static wcc_status check_options(const wcc_options* o, int bits, const void* x, const void* y)
+{
+    if (!o) return WCC_OK;
+    if (o->weight_bits != 0 && (bits == 0 || o->weight_bits < 2 || o->weight_bits > 8)) return WCC_ERR_BITS;
+    if (o->alpha != o->alpha || o->alpha > 3.0e38f) return WCC_ERR_SHAPE;      // NaN or infinite clipping parameter
+    if ((o->Wq != nullptr) != (o->scale_w != nullptr)) return WCC_ERR_NULL;
+    if (o->Wq && bits == 0) return WCC_ERR_BITS;                               // codes only exist on the quantized path
+    if (!aligned16(o->residual) || !aligned16(o->Wq) || !aligned16(o->scale_w)) return WCC_ERR_ALIGN;
+    if (o->residual && o->residual == y) return WCC_OK;                        // in-place accumulation into y is allowed
+    (void)x;
+    return WCC_OK;
+}
+
 static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int W,
                                int L, int k, int bits, void* y, wcc_dtype dt, void* ws, size_t ws_bytes,
-                               cudaStream_t st, const wcc_taps* taps)
+                               cudaStream_t st, const wcc_taps* taps, const wcc_options* opt = nullptr)
 {
-    if (!x || !Wt || !y || !ws) return WCC_ERR_NULL;
+    const bool own_codes = opt && opt->Wq;             // weights arrive quantized: Wt is not read
+    if (!x || (!Wt && !own_codes) || !y || !ws) return WCC_ERR_NULL;
     wcc_status s = check_forward_args(N, Cin, Cout, H, W, L, k, bits, dt);
     if (s != WCC_OK) return s;
+    if ((s = check_options(opt, bits, x, y)) != WCC_OK) return s;
     if (!aligned16(x) || !aligned16(Wt) || !aligned16(y) || (reinterpret_cast<uintptr_t>(ws) & 255u)) return WCC_ERR_ALIGN;
     if (taps && (!aligned16(taps->coef) || !aligned16(taps->Xq) || !aligned16(taps->Xb) || !aligned16(taps->acc)))
         return WCC_ERR_ALIGN;
@@ -256,7 +274,11 @@ static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, i
     ex.coef = taps ? taps->coef : nullptr;
     ex.hist1 = sw.hist;
     ex.fine = f.fine;
-    ex.Wt = Wt; ex.Wq = f.Wq; ex.scale_w = f.scale_w; ex.Cout = Cout; ex.kpad = f.kpad; ex.bits = bits;
+    const int wbits = (opt && opt->weight_bits && bits) ? opt->weight_bits : bits;
+    if (!own_codes) { ex.Wt = Wt; ex.Wq = f.Wq; ex.scale_w = f.scale_w; ex.Cout = Cout; ex.kpad = f.kpad; ex.bits = wbits; }
+    const void* Wq_use = own_codes ? static_cast<const void*>(opt->Wq) : f.Wq;
+    const float* scale_w_use = own_codes ? opt->scale_w : f.scale_w;
+    const FusedExtra fx = {opt ? opt->alpha : 0.0f, opt ? opt->relu : 0, opt ? opt->residual : nullptr};
     s = launch_haar_norms(x, N, Cin, H, W, L, dt, f.nrm2, f.amaxpos, ex, st);
     if (s != WCC_OK) return s;
     if ((s = profile_mark(2, st)) != WCC_OK) return s;
@@ -267,11 +289,11 @@ static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, i
     if ((s = profile_mark(3, st)) != WCC_OK) return s;
     // second pass over x: transform, mask + quantize, tensor-core contraction, dequantize, inverse, store
     void* xq_tap = taps ? (bits >= 2 ? static_cast<void*>(taps->Xq) : taps->Xb) : nullptr;
-    s = launch_fused_tiles(x, f.Wq, f.rank, f.nrm2, f.thr, f.amax_kept, bits, f.scale_w, N, Cin, Cout, H, W, L, k, f.kpad, dt, y,
-                           xq_tap, taps ? taps->acc : nullptr, st);
+    s = launch_fused_tiles(x, Wq_use, f.rank, f.nrm2, f.thr, f.amax_kept, bits, scale_w_use, N, Cin, Cout, H, W, L, k, f.kpad, dt, y,
+                           xq_tap, taps ? taps->acc : nullptr, fx, st);
     if (s == WCC_ERR_SHAPE)                            // shapes the four-tile kernel does not cover (nothing was launched)
-        s = launch_fused_pass2(x, f.Wq, f.rank, f.nrm2, f.thr, f.amax_kept, bits, f.scale_w, N, Cin, Cout, H, W, L, k, f.kpad, dt, y,
-                               xq_tap, taps ? taps->acc : nullptr, st);
+        s = launch_fused_pass2(x, Wq_use, f.rank, f.nrm2, f.thr, f.amax_kept, bits, scale_w_use, N, Cin, Cout, H, W, L, k, f.kpad, dt, y,
+                               xq_tap, taps ? taps->acc : nullptr, fx, st);
     if (s != WCC_OK) return s;
     for (int i = 4; i <= WCC_NUM_STAGES; ++i)
         if ((s = profile_mark(i, st)) != WCC_OK) return s;
@@ -281,15 +303,50 @@ static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, i
         if (taps->nrm2) WCC_CUDA_TRY(cudaMemcpyAsync(taps->nrm2, f.nrm2, (size_t)N * P * 4, dd, st));
         if (taps->idx) WCC_CUDA_TRY(cudaMemcpyAsync(taps->idx, f.idx, (size_t)M * 4, dd, st));
         if (bits >= 2) {
-            if (taps->Wq) WCC_CUDA_TRY(cudaMemcpyAsync(taps->Wq, f.Wq, (size_t)Cout * f.kpad, dd, st));
-            if (taps->scale_w) WCC_CUDA_TRY(cudaMemcpyAsync(taps->scale_w, f.scale_w, (size_t)Cout * 4, dd, st));
+            if (taps->Wq) WCC_CUDA_TRY(cudaMemcpyAsync(taps->Wq, Wq_use, (size_t)Cout * f.kpad, dd, st));
+            if (taps->scale_w) WCC_CUDA_TRY(cudaMemcpyAsync(taps->scale_w, scale_w_use, (size_t)Cout * 4, dd, st));
             if (taps->scale_a) {
-                scale_tap_kernel<<<1, 1, 0, st>>>(f.amax_kept, (float)((1 << (bits - 1)) - 1), taps->scale_a);
+                scale_tap_kernel<<<1, 1, 0, st>>>(f.amax_kept, fx.alpha, (float)((1 << (bits - 1)) - 1), taps->scale_a);
                 WCC_LAUNCH_CHECK();
             }
         }
     }
     return WCC_OK;
+}
+
+// ---- chain of layers -------------------------------------------------------------------------------
+struct ChainWs { void* act[2]; void* layer_ws; size_t layer_ws_bytes; size_t total; };
+
+static wcc_status chain_shapes_ok(const wcc_chain_layer* layers, int n_layers)
+{
+    if (!layers) return WCC_ERR_NULL;
+    if (n_layers < 1 || n_layers > 4096) return WCC_ERR_SHAPE;
+    for (int i = 0; i + 1 < n_layers; ++i)
+        if (layers[i].Cout != layers[i + 1].Cin) return WCC_ERR_SHAPE;
+    return WCC_OK;
+}
+
+static ChainWs carve_chain_ws(void* ws, const wcc_chain_layer* layers, int n_layers, int N, int H, int W, int L, int k, int bits,
+                              wcc_dtype dt)
+{
+    ChainWs c = {};
+    const size_t es = (dt == WCC_BF16) ? 2 : 4, P = (size_t)H * W;
+    size_t act = 0, lw = 0;
+    for (int i = 0; i < n_layers; ++i) {
+        if (i + 1 < n_layers) { const size_t b = (size_t)N * layers[i].Cout * P * es; if (b > act) act = b; }
+        const size_t b = wcc_workspace_bytes(N, layers[i].Cin, layers[i].Cout, H, W, L, k, bits, dt);
+        if (b == 0) { c.total = 0; return c; }
+        if (b > lw) lw = b;
+    }
+    char* b = static_cast<char*>(ws);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { char* p = b ? b + off : nullptr; off += align_up(bytes, 256); return p; };
+    c.act[0] = take(act);
+    c.act[1] = take(act);
+    c.layer_ws_bytes = lw;
+    c.layer_ws = take(lw);
+    c.total = off;
+    return c;
 }
 
 }  // namespace wcc
@@ -376,6 +433,52 @@ wcc_status wcc_forward(const void* x, const float* Wt, int N, int Cin, int Cout,
 {
     return forward_impl(x, Wt, N, Cin, Cout, H, Wd, levels, k, bits, y, dt, ws, ws_bytes,
                         static_cast<cudaStream_t>(stream), nullptr);
+}
+
+wcc_status wcc_forward_ex(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int Wd,
+                          int levels, int k, int bits, void* y, wcc_dtype dt,
+                          void* ws, size_t ws_bytes, void* stream, const wcc_options* opt, const wcc_taps* taps)
+{
+    return forward_impl(x, Wt, N, Cin, Cout, H, Wd, levels, k, bits, y, dt, ws, ws_bytes,
+                        static_cast<cudaStream_t>(stream), taps, opt);
+}
+
+size_t wcc_chain_workspace_bytes(const wcc_chain_layer* layers, int n_layers, int N, int H, int Wd, int levels, int k,
+                                 int bits, wcc_dtype dt)
+{
+    if (chain_shapes_ok(layers, n_layers) != WCC_OK) return 0;
+    return carve_chain_ws(nullptr, layers, n_layers, N, H, Wd, levels, k, bits, dt).total;
+}
+
+wcc_status wcc_chain_forward(const void* x, const wcc_chain_layer* layers, int n_layers, int N, int H, int Wd,
+                             int levels, int k, int bits, void* y, wcc_dtype dt, void* ws, size_t ws_bytes, void* stream)
+{
+    if (!x || !y || !ws) return WCC_ERR_NULL;
+    wcc_status s = chain_shapes_ok(layers, n_layers);
+    if (s != WCC_OK) return s;
+    if (reinterpret_cast<uintptr_t>(ws) & 255u) return WCC_ERR_ALIGN;
+    // every layer's arguments are checked before the first one is launched
+    for (int i = 0; i < n_layers; ++i) {
+        if (!layers[i].Wt) return WCC_ERR_NULL;
+        if ((s = check_forward_args(N, layers[i].Cin, layers[i].Cout, H, Wd, levels, k, bits, dt)) != WCC_OK) return s;
+        if (!aligned16(layers[i].Wt)) return WCC_ERR_ALIGN;
+        if (layers[i].alpha != layers[i].alpha || layers[i].alpha > 3.0e38f) return WCC_ERR_SHAPE;
+    }
+    const ChainWs c = carve_chain_ws(ws, layers, n_layers, N, H, Wd, levels, k, bits, dt);
+    if (c.total == 0) return WCC_ERR_SHAPE;
+    if (ws_bytes < c.total) return WCC_ERR_WORKSPACE;
+    const void* in = x;
+    for (int i = 0; i < n_layers; ++i) {
+        void* out = (i + 1 == n_layers) ? y : c.act[i & 1];
+        wcc_options o = {};
+        o.alpha = layers[i].alpha;
+        o.relu = layers[i].relu;
+        s = forward_impl(in, layers[i].Wt, N, layers[i].Cin, layers[i].Cout, H, Wd, levels, k, bits, out, dt,
+                         c.layer_ws, c.layer_ws_bytes, static_cast<cudaStream_t>(stream), nullptr, &o);
+        if (s != WCC_OK) return s;
+        in = out;
+    }
+    return WCC_OK;
 }
 
 wcc_status wcc_forward_staged(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int Wd,

@@ -21,7 +21,8 @@ _STATUS = {0: "ok", 1: "null pointer", 2: "bad shape", 3: "k out of range", 4: "
 EXPORTS = ("wcc_staged_workspace_bytes", "wcc_forward_staged", "wcc_workspace_bytes", "wcc_select_workspace_bytes", "wcc_haar_fwd", "wcc_haar_inv", "wcc_select_topk",
            "wcc_forward", "wcc_forward_debug", "wcc_kpad", "wcc_last_status", "wcc_status_str",
            "wcc_profile_enable", "wcc_profile_read", "wcc_kernel_launches", "wcc_select_topk_static",
-           "wcc_debug_set_wait_limit", "wcc_debug_wait_selftest")
+           "wcc_debug_set_wait_limit", "wcc_debug_wait_selftest", "wcc_forward_ex", "wcc_chain_workspace_bytes",
+           "wcc_chain_forward")
 STATIC_SCRATCH_BYTES = 512 * 1024
 STAGES = ("haar_fwd_norms", "select_topk", "weight_quant", "gather_quant", "contract", "scatter_inv")   # wcc_forward_staged
 FUSED_STAGES = ("clear", "haar_norms", "select_topk", "fused_pass2")                                      # wcc_forward
@@ -35,6 +36,15 @@ class WccError(RuntimeError):
 
 class Taps(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("coef", "nrm2", "idx", "Xq", "Xb", "scale_a", "Wq", "scale_w", "acc")]
+
+
+class Options(C.Structure):
+    _fields_ = [("alpha", C.c_float), ("weight_bits", C.c_int), ("relu", C.c_int), ("residual", C.c_void_p),
+                ("Wq", C.c_void_p), ("scale_w", C.c_void_p)]
+
+
+class ChainLayer(C.Structure):
+    _fields_ = [("Wt", C.c_void_p), ("Cin", C.c_int), ("Cout", C.c_int), ("alpha", C.c_float), ("relu", C.c_int)]
 
 
 _lib = None
@@ -72,6 +82,12 @@ def lib() -> C.CDLL:
         L.wcc_forward_debug.argtypes = fwd + [C.POINTER(Taps)]
         L.wcc_forward_staged.restype = i
         L.wcc_forward_staged.argtypes = fwd + [C.POINTER(Taps)]
+        L.wcc_forward_ex.restype = i
+        L.wcc_forward_ex.argtypes = fwd + [C.POINTER(Options), C.POINTER(Taps)]
+        L.wcc_chain_workspace_bytes.restype = sz
+        L.wcc_chain_workspace_bytes.argtypes = [C.POINTER(ChainLayer), i, i, i, i, i, i, i, i]
+        L.wcc_chain_forward.restype = i
+        L.wcc_chain_forward.argtypes = [vp, C.POINTER(ChainLayer), i, i, i, i, i, i, i, vp, i, vp, sz, vp]
         L.wcc_last_status.restype = i
         L.wcc_last_status.argtypes = [vp]
         L.wcc_profile_enable.restype = i
@@ -189,27 +205,47 @@ class Workspace:
         return cls(n, x.device)
 
 
-def forward(x: torch.Tensor, Wt: torch.Tensor, levels: int, k: int, bits: int = 8, y: torch.Tensor | None = None,
-            ws: Workspace | None = None, taps: bool = False, staged: bool = False):
+def forward(x: torch.Tensor, Wt: torch.Tensor | None, levels: int, k: int, bits: int = 8, y: torch.Tensor | None = None,
+            ws: Workspace | None = None, taps: bool = False, staged: bool = False, alpha: float = 0.0, wbits: int = 0,
+            relu: bool = False, residual: torch.Tensor | None = None, Wq: torch.Tensor | None = None,
+            scale_w: torch.Tensor | None = None):
     """The WCC layer.  Returns y, or (y, dict of intermediate tensors) when ``taps`` is set.
-    ``staged`` selects wcc_forward_staged (every intermediate in memory) instead of the fused wcc_forward."""
+    ``staged`` selects wcc_forward_staged (every intermediate in memory) instead of the fused wcc_forward.
+    ``alpha``, ``wbits``, ``relu``, ``residual``, ``Wq`` + ``scale_w``: the options of wcc_forward_ex (see wcc.h);
+    with pre-quantized weights ``Wt`` may be None."""
     _dev(x, "x")
-    _dev(Wt, "Wt")
-    if Wt.dtype != torch.float32:
-        raise TypeError("Wt must be float32")
     N, Cin, H, W = x.shape
-    Cout = Wt.shape[0]
-    if Wt.shape[1] != Cin:
-        raise ValueError("Wt must be [Cout][Cin]")
+    use_ex = bool(alpha > 0.0 or wbits or relu or residual is not None or Wq is not None)
+    if Wq is not None:
+        _dev(Wq, "Wq")
+        if scale_w is not None:
+            _dev(scale_w, "scale_w")
+        Cout = Wq.shape[0]
+    else:
+        _dev(Wt, "Wt")
+        if Wt.dtype != torch.float32:
+            raise TypeError("Wt must be float32")
+        Cout = Wt.shape[0]
+        if Wt.shape[1] != Cin:
+            raise ValueError("Wt must be [Cout][Cin]")
+    if use_ex and staged:
+        raise ValueError("options are only available on the fused path")
+    if residual is not None:
+        _dev(residual, "residual")
+        if residual.shape != (N, Cout, H, W) or residual.dtype != x.dtype:
+            raise ValueError("residual must have the output's shape and type")
     if y is None:
         y = torch.empty((N, Cout, H, W), dtype=x.dtype, device=x.device)
     if ws is None:
         ws = Workspace.for_problem(x, Cout, levels, k, bits, staged=staged)
-    args = (x.data_ptr(), Wt.data_ptr(), N, Cin, Cout, H, W, levels, k, bits, y.data_ptr(), _dt(x),
+    args = (x.data_ptr(), _ptr(Wt), N, Cin, Cout, H, W, levels, k, bits, y.data_ptr(), _dt(x),
             ws.buf.data_ptr(), ws.nbytes, _stream())
+    opt = Options(float(alpha), int(wbits), int(bool(relu)), _ptr(residual), _ptr(Wq), _ptr(scale_w)) if use_ex else None
     if not taps:
         if staged:
             _check(lib().wcc_forward_staged(*args, None), "wcc_forward_staged")
+        elif use_ex:
+            _check(lib().wcc_forward_ex(*args, C.byref(opt), None), "wcc_forward_ex")
         else:
             _check(lib().wcc_forward(*args), "wcc_forward")
         return y
@@ -230,9 +266,46 @@ def forward(x: torch.Tensor, Wt: torch.Tensor, levels: int, k: int, bits: int = 
     s = Taps(**{name: _ptr(t.get(name)) for name, _ in Taps._fields_})
     if staged:
         _check(lib().wcc_forward_staged(*args, C.byref(s)), "wcc_forward_staged")
+    elif use_ex:
+        _check(lib().wcc_forward_ex(*args, C.byref(opt), C.byref(s)), "wcc_forward_ex")
     else:
         _check(lib().wcc_forward_debug(*args, C.byref(s)), "wcc_forward_debug")
     return y, t
+
+
+class Chain:
+    """A chain of pointwise WCC layers (wcc_chain_forward): ``weights[i]`` is layer i's fp32 [Cout][Cin] device tensor;
+    a ReLU follows every layer but (unless ``relu_last``) the last; ``alphas[i]`` > 0 fixes layer i's clipping parameter.
+    The workspace (intermediate maps included) is allocated once, here."""
+
+    def __init__(self, x: torch.Tensor, weights, levels: int, k: int, bits: int = 8, relu_last: bool = False, alphas=None):
+        _dev(x, "x")
+        self.N, cin, self.H, self.W = x.shape
+        self.levels, self.k, self.bits, self.dt = levels, k, bits, _dt(x)
+        self.weights = list(weights)
+        n = len(self.weights)
+        self.layers = (ChainLayer * n)()
+        for i, Wt in enumerate(self.weights):
+            _dev(Wt, "weights[%d]" % i)
+            if Wt.dtype != torch.float32 or Wt.shape[1] != cin:
+                raise ValueError("weights[%d] must be float32 [Cout][%d]" % (i, cin))
+            self.layers[i] = ChainLayer(Wt.data_ptr(), cin, Wt.shape[0], 0.0 if alphas is None else float(alphas[i]),
+                                        int(relu_last or i + 1 < n))
+            cin = Wt.shape[0]
+        self.Cout = cin
+        nbytes = int(lib().wcc_chain_workspace_bytes(self.layers, n, self.N, self.H, self.W, levels, k, bits, self.dt))
+        if nbytes == 0:
+            raise WccError(2, "wcc_chain_workspace_bytes")
+        self.ws = Workspace(nbytes, x.device)
+
+    def __call__(self, x: torch.Tensor, y: torch.Tensor | None = None) -> torch.Tensor:
+        _dev(x, "x")
+        if y is None:
+            y = torch.empty((self.N, self.Cout, self.H, self.W), dtype=x.dtype, device=x.device)
+        _check(lib().wcc_chain_forward(x.data_ptr(), self.layers, len(self.weights), self.N, self.H, self.W, self.levels,
+                                       self.k, self.bits, y.data_ptr(), self.dt, self.ws.buf.data_ptr(), self.ws.nbytes,
+                                       _stream()), "wcc_chain_forward")
+        return y
 
 
 def last_status() -> int:
