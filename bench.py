@@ -281,6 +281,72 @@ class Case:
         return {n: acc[i] / steps for i, n in enumerate(names)}
 
 
+def chain_context(wcc, torch, np, inputs, dev, flush, peak, use_graph, steps=100):
+    """The six-layer chain workload 32 -> 192 -> 32 ... with ReLU between the layers (2 x 256 x 512, bf16), every point of
+    the sweep levels {1,2,3} x keep ratio {1/2,1/4,1/8,1/16}: one wcc_chain_forward per step (a CUDA graph replay, L2
+    flushed before every step), beside the dense 1x1 bf16 chain (library matmul + ReLU) as the keep-everything reference."""
+    N, H, W = 2, 256, 512
+    chans = [32, 192, 32, 192, 32, 192, 32]
+    first = inputs.custom("C5", 0, N, 32, 192, H, W, "bf16", 3, 0.25, 8, n_sin=16, fmax=8.0)
+    x = torch.from_numpy(first.x.view(np.int16)).view(torch.bfloat16).to(dev)
+    Ws = [torch.from_numpy(inputs.weights(100 + i, chans[i + 1], chans[i])).to(dev) for i in range(6)]
+    y = torch.empty((N, 32, H, W), dtype=torch.bfloat16, device=dev)
+    P = H * W
+    b_min = sum(2 * N * P * (chans[i] + chans[i + 1]) for i in range(6))           # every layer: input once, output once
+
+    def timed(fn, n):
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+        for a, b in ev:
+            flush.fill_(1)
+            a.record()
+            fn()
+            b.record()
+        torch.cuda.synchronize()
+        t = [a.elapsed_time(b) for a, b in ev]
+        return sum(t) / len(t)
+
+    def graphed(fn):
+        fn()
+        torch.cuda.synchronize()
+        if not use_graph:
+            return fn
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            fn()
+        torch.cuda.current_stream().wait_stream(side)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn()
+        return g.replay
+
+    Wb = [w.to(torch.bfloat16) for w in Ws]
+
+    def dense():
+        cur = x.reshape(N, 32, P)
+        for i in range(6):
+            cur = torch.matmul(Wb[i], cur)
+            if i < 5:
+                cur = torch.relu_(cur)
+        return cur
+
+    dense_ms = timed(graphed(dense), steps)
+    out = {"workload": "C5 chain: 6 layers 32->192->32..., ReLU between, N=2 H=256 W=512 bf16, bits=8",
+           "compulsory_bytes": b_min, "dense_1x1_bf16_chain_ms": dense_ms, "steps": steps, "sweep": {}}
+    for L in (1, 2, 3):
+        for gamma in (0.5, 0.25, 0.125, 0.0625):
+            k = inputs.keep_count(gamma, P)
+            ch = wcc.Chain(x, Ws, L, k, 8)
+            t = timed(graphed(lambda: ch(x, y)), steps)
+            out["sweep"]["L%d_g%s" % (L, gamma)] = {
+                "levels": L, "keep": gamma, "k": k, "ms": t, "Gpix/s_per_layer": 6 * N * P / (t * 1e-3) / 1e9,
+                "frac_of_peak": b_min / (t * 1e-3) / 1e9 / peak, "frac_of_nominal_8TBs": b_min / (t * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+                "vs_dense_chain": t / dense_ms}
+            del ch
+    assert wcc.last_status() == 0
+    return out
+
+
 def run_ours(args):
     import numpy as np
     import torch
@@ -434,6 +500,9 @@ def run_ours(args):
                 del c
                 torch.cuda.empty_cache()
         assert wcc.last_status() == 0
+    chain = None
+    if not args.batch and not args.no_context:
+        chain = chain_context(wcc, torch, np, inputs, dev, flush, peak, not args.no_graph)
     clocks_all = sampler.stop()
     timed = sampler.samples[:max(1, n_timed_samples)]
     clocks = {"sm_mhz": (statistics.median(timed) if timed else None), "sm_max_mhz": clocks_all["sm_max_mhz"],
@@ -469,7 +538,7 @@ def run_ours(args):
            "gpu_launches": int(case.launches_per_step * args.steps),
            "roofline": roofline, "cpu_baseline": cpu,
            "context": {"dense_1x1_matmul_ms": dense_ms, "ms_per_step_median": statistics.median(ms),
-                       "ms_per_step_min": min(ms), "workloads": workloads}}
+                       "ms_per_step_min": min(ms), "workloads": workloads, "chain": chain}}
     print(json.dumps(out))
     if dist:
         dist.destroy_process_group()

@@ -716,13 +716,13 @@ __device__ __forceinline__ void norms_finish(const LanePos& lp, int warp, int n,
     }
     if (ex.hist1) {                                    // norms are >= +0: key = bits | sign bit, digit = top 11 bits
         uint32_t* h = ex.hist1 + (size_t)n * 3 * 2048;
-        hist_add(h, float_key(n0) >> 21, ok0);
-        hist_add(h, float_key(n1) >> 21, ok1);
+        hist_add(h, float_key(n0) >> 21, ok0 && n0 != 0.0f);          // zero norms are not counted (see the token kernel)
+        hist_add(h, float_key(n1) >> 21, ok1 && n1 != 0.0f);
     }
     if (ex.fine) {                                     // 16-bit digits are spread out: plain atomics
         uint32_t* f = ex.fine + (size_t)n * 65536;
-        if (ok0) atomicAdd(&f[float_key(n0) >> 16], 1u);
-        if (ok1) atomicAdd(&f[float_key(n1) >> 16], 1u);
+        if (ok0 && n0 != 0.0f) atomicAdd(&f[float_key(n0) >> 16], 1u);
+        if (ok1 && n1 != 0.0f) atomicAdd(&f[float_key(n1) >> 16], 1u);
     }
 }
 
@@ -1059,15 +1059,19 @@ haar_norms_token_kernel(const __grid_constant__ CUtensorMap tmx, int N, int C, i
                     nacc[2 * i + 1] = __fmul_rn(acc[i].y, __fmul_rn(sc[2 * i + 1], sc[2 * i + 1]));
                 }
                 store_slots<L, true>(nrm2 + (size_t)n * P, lp, nacc);
+                // Norms that are exactly zero are not counted: after a ReLU whole regions of a map are zero, and their
+                // positions would all hit one bin (thousands of atomics on one address).  The selection knows the number
+                // of positions, so the zeros are what the bins leave out; they rank below everything else.
                 if (ex.hist1) {                        // norms are >= +0: key = bits | sign bit, digit = top 11 bits
                     uint32_t* h = ex.hist1 + (size_t)n * 3 * 2048;
 #pragma unroll
-                    for (int s = 0; s < 8; ++s) hist_add(h, float_key(nacc[s]) >> 21, lp.ok0);
+                    for (int s = 0; s < 8; ++s) hist_add(h, float_key(nacc[s]) >> 21, lp.ok0 && nacc[s] != 0.0f);
                 }
-                if (ex.fine && lp.ok0) {               // 16-bit digits are spread out: plain atomics
+                if (ex.fine && lp.ok0) {               // 16-bit digits of non-zero norms are spread out: plain atomics
                     uint32_t* f = ex.fine + (size_t)n * 65536;
 #pragma unroll
-                    for (int s = 0; s < 8; ++s) atomicAdd(&f[float_key(nacc[s]) >> 16], 1u);
+                    for (int s = 0; s < 8; ++s)
+                        if (nacc[s] != 0.0f) atomicAdd(&f[float_key(nacc[s]) >> 16], 1u);
                 }
             }
         }

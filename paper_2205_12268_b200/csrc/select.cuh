@@ -553,7 +553,7 @@ __device__ __forceinline__ void cluster_find_bin(cg::cluster_group& cluster, Clu
 // Find the bin of a complete 2048-bin histogram in global memory that holds the krem-th key from the top; block of
 // 256, 512 or 1024 threads, every thread returns the same values.
 __device__ __forceinline__ void block_find_bin_2048(const uint32_t* __restrict__ h, uint32_t krem, ClusterSmem& sm,
-                                                    uint32_t& bin, uint32_t& above)
+                                                    uint32_t& bin, uint32_t& above, uint32_t& tot)
 {
     const int per = SEL_BINS / (int)blockDim.x;            // 8, 4 or 2
     const int top = SEL_BINS - 1 - (int)threadIdx.x * per;
@@ -563,7 +563,6 @@ __device__ __forceinline__ void block_find_bin_2048(const uint32_t* __restrict__
         c[i] = (i < per) ? __ldcg(&h[top - i]) : 0u;
         mysum += c[i];
     }
-    uint32_t tot;
     const uint32_t before = block_scan_1024(mysum, sm.warp_sums, &tot);
     if (before < krem && krem <= before + mysum) {
         uint32_t a = before;
@@ -611,10 +610,26 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
 
     uint32_t tkey = 0, need_eq = 0, total_eq = 0, ranked = 0;    // ranked: candidates counted through (diagnostic)
     bool found = false;
+    // The supplied histograms count the non-zero norms only; the zeros are the positions they leave out and rank
+    // below everything else.  More kept positions than non-zero norms: the threshold is zero.
+    bool zero_thr = false;
+    uint32_t b1h = 0, aboveh = 0;
     if (hist1 && fine) {
-        // the 11-bit bin, then the 16-bit bin inside it (32 fine bins, one per lane of warp 0, top bin in lane 0)
-        uint32_t b1, above;
-        block_find_bin_2048(hist1 + (size_t)n * 3 * SEL_BINS, (uint32_t)k, sm, b1, above);
+        // the 11-bit bin of the threshold
+        uint32_t nonzero;
+        if (threadIdx.x == 0) { sm.res[0] = 0u; sm.res[1] = 0u; sm.res[2] = 0u; }      // (a barrier follows inside)
+        block_find_bin_2048(hist1 + (size_t)n * 3 * SEL_BINS, (uint32_t)k, sm, b1h, aboveh, nonzero);
+        zero_thr = (uint32_t)k > nonzero;              // the same in every CTA of the cluster
+        if (zero_thr) {
+            tkey = 0x80000000u;                        // key of +0
+            need_eq = (uint32_t)k - nonzero;
+            total_eq = (uint32_t)P - nonzero;
+            found = true;
+        }
+    }
+    if (hist1 && fine && !zero_thr) {
+        // the 16-bit bin inside the 11-bit bin (32 fine bins, one per lane of warp 0, top bin in lane 0)
+        const uint32_t b1 = b1h, above = aboveh;
         const uint32_t k1 = (uint32_t)k - above;
         if (threadIdx.x < 32) {
             const uint32_t f = __ldcg(&fine[(size_t)n * FINE_BINS + (b1 << 5) + 31u - (uint32_t)lane]);
@@ -683,7 +698,8 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
         // round 1: top 11 bits (only the bin search when the producer of the norms histogrammed them)
         uint32_t b1, above;
         if (hist1) {
-            block_find_bin_2048(hist1 + (size_t)n * 3 * SEL_BINS, (uint32_t)k, sm, b1, above);
+            uint32_t nonzero;
+            block_find_bin_2048(hist1 + (size_t)n * 3 * SEL_BINS, (uint32_t)k, sm, b1, above, nonzero);
         } else {
 #pragma unroll
             for (int i = 0; i < CL_MAXKPT; ++i)
@@ -715,7 +731,10 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
     }
     if (tau && crank == 0 && threadIdx.x == 0) tau[n] = key_float(tkey);
 
-    const bool ordered = want_rank || need_eq < total_eq;       // uniform over the cluster
+    // Ties kept in part need the order of positions, except ties at zero: a position whose norm is zero holds only zero
+    // coefficients, so keeping more of them than asked changes nothing downstream (consumers that get the threshold
+    // alone keep every position with key >= threshold).
+    const bool ordered = want_rank || (need_eq < total_eq && !zero_thr);       // uniform over the cluster
     float amax = 0.0f;
     // Nobody may leave while a neighbour can still read its shared memory.  When no further exchange follows, every CTA
     // signals here that it is done reading and only waits for the others at the very end (the wait is hidden behind the
