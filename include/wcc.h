@@ -93,6 +93,17 @@ wcc_status wcc_select_topk(const float* nrm2, int N, int P, int k, int32_t* idx,
                            void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * The same selection reported as a bitmap instead of an index list (Sec. 4 lets the shared index set be kept as "a
+ * single index list or a bit-map"; one bit per position serves all channels): bit (p % 32) of word p / 32 of image n
+ * is set when position p is kept.
+ *   bitmap out: uint32 [N][ceil(P / 32)]; bits beyond P are zero
+ *   ws        : scratch of at least wcc_select_bitmap_workspace_bytes(N, P, k) bytes, 256-byte aligned
+ */
+size_t wcc_select_bitmap_workspace_bytes(int N, int P, int k);
+wcc_status wcc_select_topk_bitmap(const float* nrm2, int N, int P, int k, uint32_t* bitmap, float* tau,
+                                  void* ws, size_t ws_bytes, void* stream);
+
+/*
  * wcc_select_topk without a scratch argument (the paper has no counterpart: this is a packaging variant).
  * For callers that have no way to obtain scratch memory: code that runs where cudaMalloc must not be called
  * (a latency-critical loop in which the allocator's implicit device synchronisation is unacceptable, or a host
@@ -160,6 +171,20 @@ int wcc_kpad(int Cin, int bits);
 wcc_status wcc_forward_debug(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int Wd,
                              int levels, int k, int bits, void* y, wcc_dtype dt,
                              void* ws, size_t ws_bytes, void* stream, const wcc_taps* taps);
+
+/*
+ * The layer on maps whose sides are no multiples of 2^levels (the paper's segmentation networks have 513 x 1025 maps,
+ * App. C; it does not say how they are transformed).  Reading taken here: the map is zero-padded at the bottom and on
+ * the right to the next multiples Hp, Wp of 2^levels, the layer runs on the padded map, and the output is cropped
+ * back to H x Wd.  k counts kept positions of the PADDED map (1 <= k <= Hp * Wp).  With everything kept and no
+ * quantization the result is still the dense 1x1 convolution of x: zero padding commutes with a pointwise convolution
+ * that has no bias.  ws: at least wcc_padded_workspace_bytes(...) bytes (padded input and output plus the layer's own
+ * workspace).  Sizes that need no padding run wcc_forward directly.
+ */
+size_t wcc_padded_workspace_bytes(int N, int Cin, int Cout, int H, int Wd, int levels, int k, int bits, wcc_dtype dt);
+wcc_status wcc_forward_padded(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int Wd,
+                              int levels, int k, int bits, void* y, wcc_dtype dt,
+                              void* ws, size_t ws_bytes, void* stream);
 
 /*
  * Options of the layer beyond Alg. 1, as a network built from WCC layers uses them.  A zeroed structure (or NULL)

@@ -200,6 +200,30 @@ def chain(x: np.ndarray, weights, levels: int, k: int, bits: int = 8, out_bf16: 
     return outs
 
 
+def bitmap_of(idx: np.ndarray, P: int) -> np.ndarray:
+    """Index lists [N][k] -> bitmaps uint32 [N][ceil(P/32)]: bit p % 32 of word p // 32 set for every kept p
+    (the kept set in the other of the two forms Sec. 4 names)."""
+    N = idx.shape[0]
+    words = (P + 31) // 32
+    out = np.zeros((N, words), dtype=np.uint32)
+    for n in range(N):
+        for p in idx[n]:
+            out[n, p >> 5] |= np.uint32(1) << np.uint32(p & 31)
+    return out
+
+
+def forward_padded(x: np.ndarray, Wt: np.ndarray, levels: int, k: int, bits: int, out_bf16: bool = False):
+    """The layer on a map whose sides are no multiples of 2^levels: zero padding at the bottom and on the right up to
+    the next multiples, the layer on the padded map (k counts padded positions), cropping."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    N, Cin, H, W = x.shape
+    unit = 1 << levels
+    Hp, Wp = -(-H // unit) * unit, -(-W // unit) * unit
+    xp = np.zeros((N, Cin, Hp, Wp), dtype=np.float32)
+    xp[:, :, :H, :W] = x
+    return np.ascontiguousarray(forward(xp, Wt, levels, k, bits, out_bf16=out_bf16)[:, :, :H, :W])
+
+
 def forward_f64(x: np.ndarray, Wt: np.ndarray, levels: int, k: int, idx_in: np.ndarray | None = None,
                 taps: bool = False):
     """The unquantized layer entirely in double (invariant tests)."""

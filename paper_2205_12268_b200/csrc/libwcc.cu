@@ -314,6 +314,82 @@ static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, i
     return WCC_OK;
 }
 
+// ---- kept set as a bitmap ---------------------------------------------------------------------------
+// bit p % 32 of word p / 32 of image n is set when position p is kept (rank map >= 0)
+__global__ void __launch_bounds__(256)
+rank_to_bitmap_kernel(const int32_t* __restrict__ rank, int N, int P, int words, uint32_t* __restrict__ bitmap)
+{
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;          // one thread per position, padded to words * 32
+    const long long per = (long long)words * 32;
+    if (i >= (long long)N * per) return;                                            // (whole warps leave together)
+    const int n = (int)(i / per), p = (int)(i - (long long)n * per);
+    const bool kept = p < P && rank[(size_t)n * P + p] >= 0;
+    const unsigned m = __ballot_sync(0xFFFFFFFFu, kept);
+    if ((threadIdx.x & 31) == 0) bitmap[(size_t)n * words + (p >> 5)] = m;
+}
+
+struct BitmapWs { int32_t* rank; int32_t* idx; void* sel; size_t sel_bytes; size_t total; };
+
+static BitmapWs carve_bitmap_ws(void* ws, int N, int P, int k)
+{
+    BitmapWs b = {};
+    char* base = static_cast<char*>(ws);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { char* p = base ? base + off : nullptr; off += align_up(bytes, 256); return p; };
+    b.rank = reinterpret_cast<int32_t*>(take((size_t)N * P * 4));
+    b.idx = reinterpret_cast<int32_t*>(take((size_t)N * k * 4));
+    b.sel_bytes = select_ws_bytes(N, P);
+    b.sel = take(b.sel_bytes);
+    b.total = off;
+    return b;
+}
+
+// ---- maps whose sides are no multiples of 2^levels: zero padding at the bottom and on the right -------------------
+template <typename E>
+__global__ void __launch_bounds__(256)
+pad_planes_kernel(const E* __restrict__ src, long long planes, int H, int W, int Hp, int Wp, E* __restrict__ dst)
+{
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= planes * Hp * Wp) return;
+    const int c = (int)(i % Wp);
+    const long long t = i / Wp;
+    const int r = (int)(t % Hp);
+    const long long pl = t / Hp;
+    dst[i] = (r < H && c < W) ? src[(pl * H + r) * W + c] : E(0);
+}
+template <typename E>
+__global__ void __launch_bounds__(256)
+crop_planes_kernel(const E* __restrict__ src, long long planes, int H, int W, int Hp, int Wp, E* __restrict__ dst)
+{
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= planes * H * W) return;
+    const int c = (int)(i % W);
+    const long long t = i / W;
+    const int r = (int)(t % H);
+    const long long pl = t / H;
+    dst[i] = src[(pl * Hp + r) * Wp + c];
+}
+
+struct PaddedWs { void* xp; void* yp; void* inner; size_t inner_bytes; size_t total; int Hp, Wp; };
+
+static PaddedWs carve_padded_ws(void* ws, int N, int Cin, int Cout, int H, int W, int L, int k, int bits, wcc_dtype dt)
+{
+    PaddedWs p = {};
+    const int unit = 1 << L;
+    p.Hp = ceil_div(H, unit) * unit;
+    p.Wp = ceil_div(W, unit) * unit;
+    const size_t es = (dt == WCC_BF16) ? 2 : 4;
+    char* base = static_cast<char*>(ws);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { char* q = base ? base + off : nullptr; off += align_up(bytes, 256); return q; };
+    p.xp = take((size_t)N * Cin * p.Hp * p.Wp * es);
+    p.yp = take((size_t)N * Cout * p.Hp * p.Wp * es);
+    p.inner_bytes = wcc_workspace_bytes(N, Cin, Cout, p.Hp, p.Wp, L, k, bits, dt);
+    p.inner = take(p.inner_bytes);
+    p.total = p.inner_bytes ? off : 0;
+    return p;
+}
+
 // ---- chain of layers -------------------------------------------------------------------------------
 struct ChainWs { void* act[2]; void* layer_ws; size_t layer_ws_bytes; size_t total; };
 
@@ -441,6 +517,70 @@ wcc_status wcc_forward_ex(const void* x, const float* Wt, int N, int Cin, int Co
 {
     return forward_impl(x, Wt, N, Cin, Cout, H, Wd, levels, k, bits, y, dt, ws, ws_bytes,
                         static_cast<cudaStream_t>(stream), taps, opt);
+}
+
+size_t wcc_select_bitmap_workspace_bytes(int N, int P, int k)
+{
+    if (N <= 0 || P <= 0 || k < 1 || k > P) return 0;
+    return carve_bitmap_ws(nullptr, N, P, k).total;
+}
+
+wcc_status wcc_select_topk_bitmap(const float* nrm2, int N, int P, int k, uint32_t* bitmap, float* tau,
+                                  void* ws, size_t ws_bytes, void* stream)
+{
+    if (!nrm2 || !bitmap || !ws) return WCC_ERR_NULL;
+    if (N <= 0 || P <= 0 || N > 65535 || P > (1 << 30)) return WCC_ERR_SHAPE;
+    if (k < 1 || k > P) return WCC_ERR_K;
+    if (!aligned16(nrm2) || !aligned16(bitmap) || (reinterpret_cast<uintptr_t>(ws) & 255u)) return WCC_ERR_ALIGN;
+    const BitmapWs b = carve_bitmap_ws(ws, N, P, k);
+    if (ws_bytes < b.total) return WCC_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    wcc_status s = launch_select(nrm2, N, P, k, b.idx, tau, b.rank, nullptr, false, b.sel, b.sel_bytes, st);
+    if (s != WCC_OK) return s;
+    const int words = ceil_div(P, 32);
+    const long long threads = (long long)N * words * 32;
+    rank_to_bitmap_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(b.rank, N, P, words, bitmap);
+    WCC_LAUNCH_CHECK();
+    return WCC_OK;
+}
+
+size_t wcc_padded_workspace_bytes(int N, int Cin, int Cout, int H, int Wd, int levels, int k, int bits, wcc_dtype dt)
+{
+    if (N <= 0 || Cin <= 0 || Cout <= 0 || H <= 0 || Wd <= 0 || levels < 1 || levels > 3) return 0;
+    return carve_padded_ws(nullptr, N, Cin, Cout, H, Wd, levels, k, bits, dt).total;
+}
+
+wcc_status wcc_forward_padded(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int Wd,
+                              int levels, int k, int bits, void* y, wcc_dtype dt,
+                              void* ws, size_t ws_bytes, void* stream)
+{
+    if (!x || !Wt || !y || !ws) return WCC_ERR_NULL;
+    if (N <= 0 || Cin <= 0 || Cout <= 0 || H <= 0 || Wd <= 0 || levels < 1 || levels > 3) return WCC_ERR_SHAPE;
+    if (dt != WCC_F32 && dt != WCC_BF16) return WCC_ERR_DTYPE;
+    if (!aligned16(x) || !aligned16(Wt) || !aligned16(y) || (reinterpret_cast<uintptr_t>(ws) & 255u)) return WCC_ERR_ALIGN;
+    const PaddedWs p = carve_padded_ws(ws, N, Cin, Cout, H, Wd, levels, k, bits, dt);
+    wcc_status s = check_forward_args(N, Cin, Cout, p.Hp, p.Wp, levels, k, bits, dt);       // k counts padded positions
+    if (s != WCC_OK) return s;
+    if (p.total == 0) return WCC_ERR_SHAPE;
+    if (ws_bytes < p.total) return WCC_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (p.Hp == H && p.Wp == Wd)                       // nothing to pad: the plain layer
+        return forward_impl(x, Wt, N, Cin, Cout, H, Wd, levels, k, bits, y, dt, p.inner, p.inner_bytes, st, nullptr);
+    const long long in_planes = (long long)N * Cin, out_planes = (long long)N * Cout;
+    const long long n_in = in_planes * p.Hp * p.Wp, n_out = out_planes * H * Wd;
+    if (dt == WCC_BF16)
+        pad_planes_kernel<uint16_t><<<(unsigned)((n_in + 255) / 256), 256, 0, st>>>(static_cast<const uint16_t*>(x), in_planes, H, Wd, p.Hp, p.Wp, static_cast<uint16_t*>(p.xp));
+    else
+        pad_planes_kernel<uint32_t><<<(unsigned)((n_in + 255) / 256), 256, 0, st>>>(static_cast<const uint32_t*>(x), in_planes, H, Wd, p.Hp, p.Wp, static_cast<uint32_t*>(p.xp));
+    WCC_LAUNCH_CHECK();
+    s = forward_impl(p.xp, Wt, N, Cin, Cout, p.Hp, p.Wp, levels, k, bits, p.yp, dt, p.inner, p.inner_bytes, st, nullptr);
+    if (s != WCC_OK) return s;
+    if (dt == WCC_BF16)
+        crop_planes_kernel<uint16_t><<<(unsigned)((n_out + 255) / 256), 256, 0, st>>>(static_cast<const uint16_t*>(p.yp), out_planes, H, Wd, p.Hp, p.Wp, static_cast<uint16_t*>(y));
+    else
+        crop_planes_kernel<uint32_t><<<(unsigned)((n_out + 255) / 256), 256, 0, st>>>(static_cast<const uint32_t*>(p.yp), out_planes, H, Wd, p.Hp, p.Wp, static_cast<uint32_t*>(y));
+    WCC_LAUNCH_CHECK();
+    return WCC_OK;
 }
 
 size_t wcc_chain_workspace_bytes(const wcc_chain_layer* layers, int n_layers, int N, int H, int Wd, int levels, int k,

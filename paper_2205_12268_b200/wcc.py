@@ -22,7 +22,8 @@ EXPORTS = ("wcc_staged_workspace_bytes", "wcc_forward_staged", "wcc_workspace_by
            "wcc_forward", "wcc_forward_debug", "wcc_kpad", "wcc_last_status", "wcc_status_str",
            "wcc_profile_enable", "wcc_profile_read", "wcc_kernel_launches", "wcc_select_topk_static",
            "wcc_debug_set_wait_limit", "wcc_debug_wait_selftest", "wcc_forward_ex", "wcc_chain_workspace_bytes",
-           "wcc_chain_forward")
+           "wcc_chain_forward", "wcc_select_bitmap_workspace_bytes", "wcc_select_topk_bitmap",
+           "wcc_padded_workspace_bytes", "wcc_forward_padded")
 STATIC_SCRATCH_BYTES = 512 * 1024
 STAGES = ("haar_fwd_norms", "select_topk", "weight_quant", "gather_quant", "contract", "scatter_inv")   # wcc_forward_staged
 FUSED_STAGES = ("clear", "haar_norms", "select_topk", "fused_pass2")                                      # wcc_forward
@@ -84,6 +85,14 @@ def lib() -> C.CDLL:
         L.wcc_forward_staged.argtypes = fwd + [C.POINTER(Taps)]
         L.wcc_forward_ex.restype = i
         L.wcc_forward_ex.argtypes = fwd + [C.POINTER(Options), C.POINTER(Taps)]
+        L.wcc_select_bitmap_workspace_bytes.restype = sz
+        L.wcc_select_bitmap_workspace_bytes.argtypes = [i, i, i]
+        L.wcc_select_topk_bitmap.restype = i
+        L.wcc_select_topk_bitmap.argtypes = [vp, i, i, i, vp, vp, vp, sz, vp]
+        L.wcc_padded_workspace_bytes.restype = sz
+        L.wcc_padded_workspace_bytes.argtypes = [i] * 9
+        L.wcc_forward_padded.restype = i
+        L.wcc_forward_padded.argtypes = fwd
         L.wcc_chain_workspace_bytes.restype = sz
         L.wcc_chain_workspace_bytes.argtypes = [C.POINTER(ChainLayer), i, i, i, i, i, i, i, i]
         L.wcc_chain_forward.restype = i
@@ -174,6 +183,36 @@ def select_topk(nrm2: torch.Tensor, k: int):
     _check(lib().wcc_select_topk(nrm2.data_ptr(), N, P, k, idx.data_ptr(), tau.data_ptr(), ws.data_ptr(), nbytes, _stream()),
            "wcc_select_topk")
     return idx, tau
+
+
+def select_topk_bitmap(nrm2: torch.Tensor, k: int):
+    """nrm2 fp32 [N][P] -> (bitmap int32 [N][ceil(P/32)] with bit p % 32 of word p // 32 set for kept p, tau fp32 [N])."""
+    _dev(nrm2, "nrm2")
+    N, P = nrm2.shape
+    bitmap = torch.empty((N, (P + 31) // 32), dtype=torch.int32, device=nrm2.device)
+    tau = torch.empty((N,), dtype=torch.float32, device=nrm2.device)
+    nbytes = int(lib().wcc_select_bitmap_workspace_bytes(N, P, k))
+    ws = torch.empty((max(nbytes, 256),), dtype=torch.uint8, device=nrm2.device)
+    _check(lib().wcc_select_topk_bitmap(nrm2.data_ptr(), N, P, k, bitmap.data_ptr(), tau.data_ptr(), ws.data_ptr(), nbytes,
+                                        _stream()), "wcc_select_topk_bitmap")
+    return bitmap, tau
+
+
+def forward_padded(x: torch.Tensor, Wt: torch.Tensor, levels: int, k: int, bits: int = 8) -> torch.Tensor:
+    """The layer on a map whose sides need not be multiples of 2^levels (zero padding, see wcc_forward_padded);
+    k counts positions of the padded map."""
+    _dev(x, "x")
+    _dev(Wt, "Wt")
+    N, Cin, H, W = x.shape
+    Cout = Wt.shape[0]
+    nbytes = int(lib().wcc_padded_workspace_bytes(N, Cin, Cout, H, W, levels, k, bits, _dt(x)))
+    if nbytes == 0:
+        raise WccError(2, "wcc_padded_workspace_bytes")
+    ws = torch.empty((nbytes,), dtype=torch.uint8, device=x.device)
+    y = torch.empty((N, Cout, H, W), dtype=x.dtype, device=x.device)
+    _check(lib().wcc_forward_padded(x.data_ptr(), Wt.data_ptr(), N, Cin, Cout, H, W, levels, k, bits, y.data_ptr(), _dt(x),
+                                    ws.data_ptr(), nbytes, _stream()), "wcc_forward_padded")
+    return y
 
 
 def select_topk_static(nrm2: torch.Tensor, k: int, idx: torch.Tensor, tau: torch.Tensor):

@@ -109,3 +109,28 @@ def test_chain_is_a_loop_of_single_layers():
             cur = np.maximum(cur, np.float32(0))
         assert np.array_equal(cur, outs[i])
     assert outs[0].min() >= 0 and outs[2].min() < 0                # ReLU between the layers, none after the last
+
+
+def test_padded_layer_with_everything_kept_is_the_dense_conv():
+    """Zero padding commutes with a pointwise convolution that has no bias: on a 13 x 27 map, everything kept and no
+    quantization, the padded layer cropped back equals the dense 1x1 convolution of the original map."""
+    rng = np.random.default_rng(11)
+    x = rng.standard_normal((2, 5, 13, 27)).astype(np.float32)
+    Wt = rng.standard_normal((4, 5)).astype(np.float32)
+    y = oracle.forward_padded(x, Wt, 3, 16 * 32, 0)
+    ref = np.einsum("oc,nchw->nohw", Wt.astype(np.float64), x.astype(np.float64))
+    assert y.shape == ref.shape and np.abs(y - ref).max() <= 1e-5 * np.abs(ref).max()
+    # sizes that need no padding: the plain layer
+    x2 = rng.standard_normal((1, 3, 16, 8)).astype(np.float32)
+    W2 = rng.standard_normal((2, 3)).astype(np.float32)
+    assert np.array_equal(oracle.forward_padded(x2, W2, 3, 40, 8), oracle.forward(x2, W2, 3, 40, 8))
+
+
+def test_bitmap_is_the_index_list_in_another_form():
+    idx = np.array([[0, 5, 31, 32, 70], [1, 2, 3, 64, 95]], dtype=np.int32)
+    bm = oracle.bitmap_of(idx, 96)
+    assert bm.shape == (2, 3)
+    assert bm[0].tolist() == [(1 << 0) | (1 << 5) | (1 << 31), 1 << 0, 1 << 6]
+    assert bm[1].tolist() == [0b1110, 0, (1 << 0) | (1 << 31)]
+    back = [np.flatnonzero(np.unpackbits(bm[n].view(np.uint8), bitorder="little")) for n in range(2)]
+    assert all(np.array_equal(back[n], idx[n]) for n in range(2))
