@@ -224,6 +224,29 @@ def forward_padded(x: np.ndarray, Wt: np.ndarray, levels: int, k: int, bits: int
     return np.ascontiguousarray(forward(xp, Wt, levels, k, bits, out_bf16=out_bf16)[:, :, :H, :W])
 
 
+def dwconv3x3(x: np.ndarray, w: np.ndarray) -> np.ndarray:
+    """Depthwise 3x3 convolution, stride 1, zero padding 1, no bias: x [N][C][H][W], w [C][3][3] -> [N][C][H][W] (fp32)."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    N, Cc, H, W = x.shape
+    assert w.shape == (Cc, 3, 3)
+    y = np.empty_like(x)
+    _L().orc_dwconv3x3_f32(_p(x, C.c_float), _p(w, C.c_float), N, Cc, H, W, _p(y, C.c_float))
+    return y
+
+
+def block(x: np.ndarray, W1: np.ndarray, Wdw: np.ndarray, W3: np.ndarray, levels: int, k: int, bits: int = 8,
+          out_bf16: bool = False, taps: bool = False):
+    """The inverted residual block of Eq. 13 with both pointwise convolutions as WCC layers and no non-linearities:
+    y = x + WCC(W3, dw3x3(Wdw, WCC(W1, x))).  The expanded map u = WCC(W1, x) is rounded to the activation type like any
+    layer output; the depthwise convolution feeds the second layer's transform directly in fp32 (the two are one fused
+    step), and the skip connection is added after the second layer's inverse transform."""
+    u = forward(x, W1, levels, k, bits, out_bf16=out_bf16)
+    v = dwconv3x3(u, Wdw)
+    y = forward(v, W3, levels, k, bits, out_bf16=out_bf16, residual=np.ascontiguousarray(x, dtype=np.float32))
+    return (y, dict(u=u, v=v)) if taps else y
+
+
 def forward_f64(x: np.ndarray, Wt: np.ndarray, levels: int, k: int, idx_in: np.ndarray | None = None,
                 taps: bool = False):
     """The unquantized layer entirely in double (invariant tests)."""

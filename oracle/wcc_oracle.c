@@ -266,6 +266,31 @@ done:
     return rc;
 }
 
+/*
+ * Depthwise 3x3 convolution (the K_dw of the inverted residual block, Eq. 13): every channel on its own, stride 1,
+ * zero padding 1, no bias, cross-correlation.  w is [C][3][3].  fp32, one fused multiply-add per tap in row-major tap
+ * order starting from +0; taps that fall outside the map contribute nothing.
+ */
+void orc_dwconv3x3_f32(const float *x, const float *w, int N, int C, int H, int W, float *y)
+{
+#pragma omp parallel for schedule(static)
+    for (long pl = 0; pl < (long)N * C; ++pl) {
+        const float *xp = x + (size_t)pl * H * W;
+        const float *wp = w + (size_t)(pl % C) * 9;
+        float *yp = y + (size_t)pl * H * W;
+        for (int r = 0; r < H; ++r)
+            for (int c = 0; c < W; ++c) {
+                float acc = 0.0f;
+                for (int i = 0; i < 3; ++i)
+                    for (int j = 0; j < 3; ++j) {
+                        const int rr = r + i - 1, cc = c + j - 1;
+                        if (rr >= 0 && rr < H && cc >= 0 && cc < W) acc = fmaf(wp[i * 3 + j], xp[(size_t)rr * W + cc], acc);
+                    }
+                yp[(size_t)r * W + c] = acc;
+            }
+    }
+}
+
 int orc_num_threads(void)
 {
 #ifdef _OPENMP

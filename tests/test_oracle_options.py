@@ -134,3 +134,43 @@ def test_bitmap_is_the_index_list_in_another_form():
     assert bm[1].tolist() == [0b1110, 0, (1 << 0) | (1 << 31)]
     back = [np.flatnonzero(np.unpackbits(bm[n].view(np.uint8), bitorder="little")) for n in range(2)]
     assert all(np.array_equal(back[n], idx[n]) for n in range(2))
+
+
+def test_depthwise_conv_against_the_library_and_closed_forms():
+    import torch.nn.functional as F
+    rng = np.random.default_rng(14)
+    # small integers: every product and sum is exact, so any summation order gives the same bits
+    x = rng.integers(-8, 9, (2, 5, 7, 9)).astype(np.float32)
+    w = rng.integers(-4, 5, (5, 3, 3)).astype(np.float32)
+    ref = F.conv2d(torch.from_numpy(x).double(), torch.from_numpy(w).double()[:, None], padding=1, groups=5).numpy()
+    assert np.array_equal(oracle.dwconv3x3(x, w).astype(np.float64), ref)
+    # real values: within rounding of the double result
+    x = rng.standard_normal((1, 3, 16, 12)).astype(np.float32)
+    w = rng.standard_normal((3, 3, 3)).astype(np.float32)
+    ref = F.conv2d(torch.from_numpy(x).double(), torch.from_numpy(w).double()[:, None], padding=1, groups=3).numpy()
+    assert np.abs(oracle.dwconv3x3(x, w) - ref).max() <= 1e-5 * np.abs(ref).max()
+    # a kernel with a single 1 at tap (i, j) shifts the map by (1 - i, 1 - j) with zeros moving in: orientation of the taps
+    x = np.arange(20, dtype=np.float32).reshape(1, 1, 4, 5)
+    w = np.zeros((1, 3, 3), np.float32); w[0, 0, 2] = 1        # out[r][c] = x[r-1][c+1]
+    y = oracle.dwconv3x3(x, w)[0, 0]
+    assert y[0].tolist() == [0] * 5 and y[1].tolist() == [1, 2, 3, 4, 0] and y[3].tolist() == [11, 12, 13, 14, 0]
+    w = np.zeros((1, 3, 3), np.float32); w[0, 1, 1] = 1        # identity
+    assert np.array_equal(oracle.dwconv3x3(x, w), x)
+
+
+def test_block_with_identity_parts_returns_twice_the_input():
+    """Identity pointwise weights, identity depthwise kernel, everything kept, no quantization: every part is the
+    identity, so the block returns x + x (the skip connection of Eq. 13)."""
+    w = inputs.custom("blk", 15, 1, 4, 4, 8, 16, "f32", 3, 1.0, 0, n_sin=3, fmax=2.0)
+    eye = np.eye(4, dtype=np.float32)
+    dw = np.zeros((4, 3, 3), np.float32); dw[:, 1, 1] = 1
+    y = oracle.block(w.x, eye, dw, eye, 3, 128, 0)
+    assert np.abs(y - 2 * w.x).max() <= 1e-5 * np.abs(w.x).max()
+    # and with real parts it is the composition of its three steps plus the input
+    rng = np.random.default_rng(16)
+    W1, W3 = inputs.weights(1, 12, 4), inputs.weights(2, 4, 12)
+    dw = rng.standard_normal((12, 3, 3)).astype(np.float32)
+    y, t = oracle.block(w.x, W1, dw, W3, 3, 40, 8, taps=True)
+    assert np.array_equal(t["u"], oracle.forward(w.x, W1, 3, 40, 8))
+    assert np.array_equal(t["v"], oracle.dwconv3x3(t["u"], dw))
+    assert np.array_equal(y, oracle.forward(t["v"], W3, 3, 40, 8) + w.x)
