@@ -22,7 +22,9 @@
  *    along the width) top-right, y3 (difference along the height) bottom-left, y4 bottom-right.
  *    A "position" p = row * Wd + col indexes this layout; P = H * Wd.
  *  - levels is 1, 2 or 3 (the paper uses 3); H and Wd must be multiples of 2^levels.
- *  - Cin <= 256 and Cout <= 256 for wcc_forward (one tensor-core tile along each).
+ *  - Cin, Cout <= WCC_MAX_CHANNELS.  wcc_forward runs its fused two-pass kernels while the operands of one tile group
+ *    fit one SM's shared memory and tensor memory (up to 256 channels on the quantized path) and otherwise the
+ *    stage-by-stage pipeline of wcc_forward_staged, whose contraction tiles K and N; wcc_workspace_bytes accounts for it.
  *  - There is no CPU fallback: the library is built for sm_100a only.
  */
 #ifndef WCC_H_
@@ -50,6 +52,7 @@ typedef enum {
 } wcc_status;
 
 typedef enum { WCC_F32 = 0, WCC_BF16 = 1 } wcc_dtype;   /* element type of activations x and y */
+#define WCC_MAX_CHANNELS 8192
 
 /* Scratch bytes wcc_forward / wcc_forward_debug need for these arguments (0 on invalid arguments). */
 size_t wcc_workspace_bytes(int N, int Cin, int Cout, int H, int Wd, int levels, int k, int bits, wcc_dtype dt);
@@ -214,6 +217,29 @@ typedef struct wcc_options {
 wcc_status wcc_forward_ex(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int Wd,
                           int levels, int k, int bits, void* y, wcc_dtype dt,
                           void* ws, size_t ws_bytes, void* stream, const wcc_options* opt, const wcc_taps* taps);
+
+/*
+ * Depthwise 3x3 convolution fused with the forward transform (App. H, "a kernel for a fused depthwise convolution and
+ * Haar transform": both are separable per channel, so the convolution's output never goes to memory).
+ *   u    in : [N][C][H][Wd] of dt           Wdw in: fp32 [C][3][3], stride 1, zero padding 1, no bias, cross-correlation
+ *   coef out: fp32 [N][C][H][Wd] = forward transform of dw3x3(u), quadrant layout; nrm2 out: fp32 [N][P] or NULL
+ * Per pixel one fused multiply-add per tap in row-major tap order from +0; then exactly wcc_haar_fwd's arithmetic.
+ */
+wcc_status wcc_dwconv_haar_fwd(const void* u, const float* Wdw, int N, int C, int H, int Wd, int levels, wcc_dtype dt,
+                               float* coef, float* nrm2, void* stream);
+
+/*
+ * The inverted residual block of Eq. 13 with both pointwise convolutions as WCC layers and no non-linearities:
+ *     y = x + WCC(W3, dw3x3(Wdw, WCC(W1, x)))
+ *   x, y: [N][C][H][Wd] of dt      W1: fp32 [E][C]      Wdw: fp32 [E][3][3]      W3: fp32 [C][E]      (E: expanded channels)
+ * The expanded map u = WCC(W1, x) is stored in dt in the workspace; the depthwise convolution feeds the second layer's
+ * transform in fp32 without going to memory; the skip connection is added after the second layer's inverse transform.
+ * Same levels, k and bits for both layers.  ws: at least wcc_block_workspace_bytes(...) bytes.
+ */
+size_t wcc_block_workspace_bytes(int N, int C, int E, int H, int Wd, int levels, int k, int bits, wcc_dtype dt);
+wcc_status wcc_block_forward(const void* x, const float* W1, const float* Wdw, const float* W3, int N, int C, int E,
+                             int H, int Wd, int levels, int k, int bits, void* y, wcc_dtype dt,
+                             void* ws, size_t ws_bytes, void* stream);
 
 /*
  * A chain of pointwise WCC layers on one feature map (e.g. the 32 -> 192 -> 32 ... stacks of an inverted-residual

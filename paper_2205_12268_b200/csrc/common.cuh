@@ -85,7 +85,8 @@ wcc_status launch_haar_inv(const float* coef, int N, int C, int H, int W, int L,
 // Dequantize + scatter into a zero map + inverse Haar.  acc rows have pitch ldc (int32 or fp32 bits).
 wcc_status launch_scatter_inv(const int32_t* acc, int ldc, bool acc_is_float, const int32_t* rank,
                               const float* amax_kept, int bits, const float* scale_w,
-                              int N, int Cout, int H, int W, int L, int k, wcc_dtype dt, void* y, cudaStream_t st);
+                              int N, int Cout, int H, int W, int L, int k, wcc_dtype dt, void* y, cudaStream_t st,
+                              const void* residual = nullptr, int relu = 0);
 
 // Radix select + ordered compaction.  rank (int32 [N][P], -1 = dropped), amaxpos / amax_kept (max over the
 // kept positions of amaxpos, as float bits, must be zeroed by this call) are optional.

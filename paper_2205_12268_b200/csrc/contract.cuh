@@ -2,12 +2,12 @@
 // WCC workflow; Alg. 1 "Y_wt = Conv(K_1x1, X[I])"):
 //     acc[r][o] = sum_c Xq[r][c] * Wq[o][c],      r = kept position (row), o = output channel.
 // Positions are the long dimension, so they map to the MMA M (tiles of 128 rows = 128 TMEM lanes); the output
-// channels are the MMA N (one instruction covers all of them, N <= 256); the input channels are K.
+// channels are the MMA N (tiles of up to 256, one instruction each); the input channels are K, streamed in 128-byte atoms.
 //
 // Blackwell path: operands are staged by TMA (cp.async.bulk.tensor, 128-byte swizzle, no multicast) into shared
 // memory, one elected thread issues tcgen05.mma (kind::i8 with int32 accumulation, or kind::f16 on bf16 with
 // fp32 accumulation) into a double-buffered TMEM accumulator, and four epilogue warps read it back with
-// tcgen05.ld and store it.  Persistent CTAs walk the row tiles; the weights are loaded once per CTA.
+// tcgen05.ld and store it.  Persistent CTAs walk the (row tile, column tile) pairs; the weights come from L2 every time.
 // Every mbarrier wait is bounded: when one runs out the kernel raises WCC_ERR_TIMEOUT in the status word,
 // lets the copies in flight land, frees its TMEM and returns.
 #pragma once
@@ -18,11 +18,14 @@
 namespace wcc {
 namespace tc {
 
-constexpr int TILE_M = 128;
-constexpr int STAGES = 3;
+constexpr int TILE_M = 128;                     // rows (kept positions) per tile = TMEM lanes
+constexpr int TILE_N = 256;                     // output channels per tile (one instruction covers them)
+constexpr int STAGES = 4;
 constexpr int ATOM_BYTES = 128;                 // one swizzle row: 128 bytes of K
 constexpr int A_ATOM_BYTES = TILE_M * ATOM_BYTES;
-constexpr int MAX_KATOMS = 4;                   // K <= 512 bytes per row (Cin <= 512 int8, 256 bf16)
+constexpr int B_ATOM_BYTES = TILE_N * ATOM_BYTES;
+constexpr int STAGE_BYTES = A_ATOM_BYTES + B_ATOM_BYTES;      // 48 KB, a multiple of 1024 (swizzle alignment)
+constexpr int TMEM_COLS = 2 * TILE_N;           // two accumulator buffers
 
 // K-major operand tile, 128-byte swizzle: rows of 128 bytes, groups of 8 rows 1024 bytes apart.
 __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
@@ -59,7 +62,6 @@ __device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::aft
 struct SmemCtl {
     uint64_t full[STAGES];
     uint64_t empty[STAGES];
-    uint64_t bfull;
     uint64_t tfull[2];
     uint64_t tempty[2];
     uint32_t tmem_base;
@@ -67,35 +69,35 @@ struct SmemCtl {
 };
 
 // 192 threads: warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2-5 = epilogue.
+// Persistent CTAs walk the (row tile, column tile) pairs; every pair streams its K range through a ring of stages, each
+// holding one 128-byte K atom of the rows (128 x 128 B) and of the weights (TILE_N x 128 B), so any number of input
+// channels and of output channels is covered: K is a loop, N is tiled by TILE_N.
 template <bool I8>
 __global__ void __launch_bounds__(192, 1)
 contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                int M, int npad, int krow_bytes, int tmem_cols, int32_t* __restrict__ acc, int ldc, int* __restrict__ status)
+                int M, int npad, int krow_bytes, int32_t* __restrict__ acc, int ldc, int* __restrict__ status)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     const int katoms = (krow_bytes + ATOM_BYTES - 1) / ATOM_BYTES;
-    const uint32_t b_atom_bytes = (uint32_t)npad * ATOM_BYTES;
-    const uint32_t sB = base;
-    const uint32_t sA = sB + katoms * b_atom_bytes;                    // multiple of 2048: stays 1024-aligned
-    SmemCtl* ctl = reinterpret_cast<SmemCtl*>(smem_raw + (sA - raw) + (size_t)STAGES * katoms * A_ATOM_BYTES);
+    SmemCtl* ctl = reinterpret_cast<SmemCtl*>(smem_raw + (base - raw) + (size_t)STAGES * STAGE_BYTES);
     volatile int* abort_flag = &ctl->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tiles = (M + TILE_M - 1) / TILE_M;
+    const int m_tiles = (M + TILE_M - 1) / TILE_M, n_tiles = (npad + TILE_N - 1) / TILE_N;
+    const int items = m_tiles * n_tiles;                 // item = m_tile * n_tiles + n_tile: the column tiles of a row tile are neighbours
     const int elems_per_atom = I8 ? ATOM_BYTES : ATOM_BYTES / 2;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&ctl->full[s]), 1); mbar_init(smem_u32(&ctl->empty[s]), 1); }
-        mbar_init(smem_u32(&ctl->bfull), 1);
         for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&ctl->tfull[b]), 1); mbar_init(smem_u32(&ctl->tempty[b]), 4); }
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(&ctl->tmem_base)), "r"((uint32_t)tmem_cols) : "memory");
+                     ::"r"(smem_u32(&ctl->tmem_base)), "r"((uint32_t)TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     fence_before();
@@ -106,70 +108,76 @@ contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 
     if (warp == 0) {
         if (lane == 0) {
-            // weights: once
-            mbar_expect_tx(smem_u32(&ctl->bfull), katoms * b_atom_bytes);
-            for (int a = 0; a < katoms; ++a)
-                tma_load_2d(sB + a * b_atom_bytes, &tmB, a * elems_per_atom, 0, smem_u32(&ctl->bfull));
-            int it = 0;
-            for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++it) {
-                const int s = it % STAGES;
-                const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
-                if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1u, abort_flag)) { failed = true; break; }
-                mbar_expect_tx(smem_u32(&ctl->full[s]), (uint32_t)katoms * A_ATOM_BYTES);
-                for (int a = 0; a < katoms; ++a)
-                    tma_load_2d(sA + (uint32_t)(s * katoms + a) * A_ATOM_BYTES, &tmA, a * elems_per_atom, t * TILE_M,
-                                smem_u32(&ctl->full[s]));
+            int it = 0;                                  // stages filled so far
+            for (int w = blockIdx.x; w < items && !failed; w += gridDim.x) {
+                const int mt = w / n_tiles, nt = w - mt * n_tiles;
+                for (int a = 0; a < katoms; ++a, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                    if (!mbar_wait(smem_u32(&ctl->empty[s]), ph ^ 1u, abort_flag)) { failed = true; break; }
+                    const uint32_t sA = base + (uint32_t)s * STAGE_BYTES, sB = sA + A_ATOM_BYTES;
+                    mbar_expect_tx(smem_u32(&ctl->full[s]), (uint32_t)STAGE_BYTES);
+                    tma_load_2d(sA, &tmA, a * elems_per_atom, mt * TILE_M, smem_u32(&ctl->full[s]));
+                    tma_load_2d(sB, &tmB, a * elems_per_atom, nt * TILE_N, smem_u32(&ctl->full[s]));
+                }
             }
         }
         __syncwarp();
     } else if (warp == 1) {
         if (lane == 0) {
-            // instruction descriptor: D format, A/B formats, N >> 3 at bit 17, M >> 4 at bit 24; K-major A and B
-            const uint32_t idesc = (I8 ? (2u << 4) : (1u << 4)) | (1u << 7) | (1u << 10) |
-                                   ((uint32_t)(npad >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
-            if (!mbar_wait(smem_u32(&ctl->bfull), 0u, abort_flag)) failed = true;
-            int it = 0;
-            for (int t = blockIdx.x; t < tiles && !failed; t += gridDim.x, ++it) {
-                const int s = it % STAGES, buf = it & 1;
-                const uint32_t ph = (uint32_t)(it / STAGES) & 1u, bph = (uint32_t)(it >> 1) & 1u;
+            int it = 0, item = 0;
+            for (int w = blockIdx.x; w < items && !failed; w += gridDim.x, ++item) {
+                const int nt = w % n_tiles;
+                const int cur = min(TILE_N, npad - nt * TILE_N);
+                // instruction descriptor: D format, A/B formats, N >> 3 at bit 17, M >> 4 at bit 24; K-major A and B
+                const uint32_t idesc = (I8 ? (2u << 4) : (1u << 4)) | (1u << 7) | (1u << 10) |
+                                       ((uint32_t)(cur >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+                const int buf = item & 1;
+                const uint32_t bph = (uint32_t)(item >> 1) & 1u;
                 if (!mbar_wait(smem_u32(&ctl->tempty[buf]), bph ^ 1u, abort_flag)) { failed = true; break; }
-                if (!mbar_wait(smem_u32(&ctl->full[s]), ph, abort_flag)) { failed = true; break; }
                 fence_after();
-                const uint32_t d = tmem_base + (uint32_t)(buf * npad);
+                const uint32_t d = tmem_base + (uint32_t)(buf * TILE_N);
                 uint32_t accumulate = 0;
-                for (int a = 0; a < katoms; ++a) {
+                for (int a = 0; a < katoms; ++a, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+                    if (!mbar_wait(smem_u32(&ctl->full[s]), ph, abort_flag)) { failed = true; break; }
+                    fence_after();
+                    const uint32_t sA = base + (uint32_t)s * STAGE_BYTES, sB = sA + A_ATOM_BYTES;
                     const int ksteps = min(4, (krow_bytes - a * ATOM_BYTES) / 32);
-                    const uint64_t ad = smem_desc_sw128(sA + (uint32_t)(s * katoms + a) * A_ATOM_BYTES);
-                    const uint64_t bd = smem_desc_sw128(sB + a * b_atom_bytes);
+                    const uint64_t ad = smem_desc_sw128(sA), bd = smem_desc_sw128(sB);
                     for (int kk = 0; kk < ksteps; ++kk) {
                         mma_ss<I8>(d, ad + (uint64_t)(2 * kk), bd + (uint64_t)(2 * kk), idesc, accumulate);   // +32 bytes of K
                         accumulate = 1;
                     }
+                    mma_commit(smem_u32(&ctl->empty[s]));
                 }
-                mma_commit(smem_u32(&ctl->empty[s]));
+                if (failed) break;
                 mma_commit(smem_u32(&ctl->tfull[buf]));
             }
         }
         __syncwarp();
     } else {
         const int q = warp & 3;                       // TMEM lane quarter this warp may read
-        int it = 0;
-        for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++it) {
-            const int buf = it & 1;
-            const uint32_t bph = (uint32_t)(it >> 1) & 1u;
+        int item = 0;
+        for (int w = blockIdx.x; w < items; w += gridDim.x, ++item) {
+            const int mt = w / n_tiles, nt = w - mt * n_tiles;
+            const int n0 = nt * TILE_N, cur = min(TILE_N, npad - n0);
+            const int buf = item & 1;
+            const uint32_t bph = (uint32_t)(item >> 1) & 1u;
             int okw = mbar_wait(smem_u32(&ctl->tfull[buf]), bph, abort_flag) ? 1 : 0;
             okw = __all_sync(0xFFFFFFFFu, okw);
             if (!okw) { failed = true; break; }
             fence_after();
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * npad);
-            const long long grow = (long long)t * TILE_M + q * 32 + lane;
-            int32_t* dst = acc + grow * ldc;
-            for (int c0 = 0; c0 < ldc; c0 += 8) {
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * TILE_N);
+            const long long grow = (long long)mt * TILE_M + q * 32 + lane;
+            int32_t* dst = acc + grow * ldc + n0;
+            for (int c0 = 0; c0 < cur && n0 + c0 < ldc; c0 += 8) {
                 uint32_t r[8];
                 tmem_ld8(taddr + (uint32_t)c0, r);
                 if (grow < M) {
                     *reinterpret_cast<uint4*>(dst + c0) = make_uint4(r[0], r[1], r[2], r[3]);
-                    if (c0 + 4 < ldc) *reinterpret_cast<uint4*>(dst + c0 + 4) = make_uint4(r[4], r[5], r[6], r[7]);
+                    if (n0 + c0 + 4 < ldc) *reinterpret_cast<uint4*>(dst + c0 + 4) = make_uint4(r[4], r[5], r[6], r[7]);
                 }
             }
             fence_before();
@@ -191,7 +199,7 @@ contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     }
     if (warp == 1) {
         fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)tmem_cols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
     }
 }
 
@@ -218,17 +226,14 @@ wcc_status launch_contract(const void* Xq, const void* Wq, int M, int Cout, int 
     using namespace tc;
     const bool i8 = bits >= 2;
     const int krow_bytes = kpad * (i8 ? 1 : 2);
-    const int katoms = ceil_div(krow_bytes, ATOM_BYTES);
     const int npad = ceil_div(Cout, 16) * 16;
-    if (katoms > MAX_KATOMS || npad > 256 || (krow_bytes % 32) != 0) return WCC_ERR_SHAPE;
-    int tmem_cols = 32;
-    while (tmem_cols < 2 * npad) tmem_cols <<= 1;
+    if ((krow_bytes % 32) != 0) return WCC_ERR_SHAPE;
 
     CUtensorMap tmA, tmB;
     if (!make_map(&tmA, Xq, i8, (uint64_t)kpad, (uint64_t)M, TILE_M)) return WCC_ERR_CUDA;
-    if (!make_map(&tmB, Wq, i8, (uint64_t)kpad, (uint64_t)Cout, (uint32_t)npad)) return WCC_ERR_CUDA;
+    if (!make_map(&tmB, Wq, i8, (uint64_t)kpad, (uint64_t)Cout, TILE_N)) return WCC_ERR_CUDA;   // rows beyond Cout arrive as zeros
 
-    const size_t smem = 1024 + (size_t)katoms * npad * ATOM_BYTES + (size_t)STAGES * katoms * A_ATOM_BYTES + sizeof(SmemCtl) + 16;
+    const size_t smem = 1024 + (size_t)STAGES * STAGE_BYTES + sizeof(SmemCtl) + 16;
     static int sm_count[64] = {0};
     static bool attr_set[64][2] = {{false}};
     int dev = 0;
@@ -236,19 +241,18 @@ wcc_status launch_contract(const void* Xq, const void* Wq, int M, int Cout, int 
     if (dev < 0 || dev >= 64) return WCC_ERR_CUDA;
     if (!sm_count[dev]) WCC_CUDA_TRY(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
     if (!attr_set[dev][i8]) {
-        if (i8) WCC_CUDA_TRY(cudaFuncSetAttribute(contract_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-        else WCC_CUDA_TRY(cudaFuncSetAttribute(contract_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+        if (i8) WCC_CUDA_TRY(cudaFuncSetAttribute(contract_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        else WCC_CUDA_TRY(cudaFuncSetAttribute(contract_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         attr_set[dev][i8] = true;
     }
-    if (smem > 200 * 1024) return WCC_ERR_SHAPE;
     int* status = nullptr;
     WCC_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_status));
-    const int tiles = ceil_div(M, TILE_M);
-    const int grid = tiles < sm_count[dev] ? tiles : sm_count[dev];
+    const long long items = (long long)ceil_div(M, TILE_M) * ceil_div(npad, TILE_N);
+    const int grid = (int)(items < sm_count[dev] ? items : sm_count[dev]);
     if (i8)
-        contract_kernel<true><<<grid, 192, smem, st>>>(tmA, tmB, M, npad, krow_bytes, tmem_cols, acc, ldc, status);
+        contract_kernel<true><<<grid, 192, smem, st>>>(tmA, tmB, M, npad, krow_bytes, acc, ldc, status);
     else
-        contract_kernel<false><<<grid, 192, smem, st>>>(tmA, tmB, M, npad, krow_bytes, tmem_cols, acc, ldc, status);
+        contract_kernel<false><<<grid, 192, smem, st>>>(tmA, tmB, M, npad, krow_bytes, acc, ldc, status);
     WCC_LAUNCH_CHECK();
     return WCC_OK;
 }

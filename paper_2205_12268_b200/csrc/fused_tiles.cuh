@@ -39,9 +39,23 @@ struct Ctl {
     uint64_t empty_a[MAX_NA];
     uint64_t ready[2];
     uint64_t tfree[2];
+    uint64_t tok[TILES][2];      // NEXT: token of the norm chain has arrived for warp q of tile t
     uint32_t tmem_base;
     int abort_flag;
 };
+
+// With these pointers set (kernel variant NEXT) the kernel is also the first pass of the NEXT layer of a chain: the
+// output tile it has just computed (after the residual add / ReLU, rounded to the activation type as it is stored) is
+// transformed forward again while still in registers, and the channel norms, the per-position max |coefficient| and the
+// selection's histograms of the next layer's input come out of the same launch; the next layer never reads its input
+// for a first pass (App. H, "Memory bandwidth and traffic": consecutive separable steps done on a tile in one go).
+struct NextNorms {
+    float* nrm2;          // fp32 [N][P]
+    float* amaxpos;       // fp32 [N][P]
+    uint32_t* hist1;      // [N][3][2048], zero on entry (round 1 is filled)
+    uint32_t* fine;       // [N][65536], zero on entry
+};
+constexpr int TOKEN_BYTES = 32 * 16 * 4;     // per lane: 8 partial sums + 8 running maxima
 
 template <typename T, bool I8, int WPT>
 struct Cfg {
@@ -60,14 +74,16 @@ struct Params {
     float alpha;                 // > 0: given clipping parameter of the activation quantizer (codes are clamped)
     int relu;                    // non-zero: y = max(., 0)
     const void* residual;        // NULL, or [N][Cout][H][W] of the activation type, added before the ReLU
+    NextNorms nx;                // kernel variant NEXT only
     int N, Cin, Cout, H, W, k, kpad, npad, nchunk, nn, nbuf, tmem_cols, na, tiles_total;
     void* y; uint8_t* xq_tap; int32_t* acc_tap; int* status;
 };
 
-template <typename T, int L, bool I8, int WPT>
+template <typename T, int L, bool I8, int WPT, bool NEXT>
 __global__ void __launch_bounds__(Cfg<T, I8, WPT>::THREADS, 1)
 fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
 {
+    static_assert(!NEXT || WPT == 2, "the norm chain alternates between the two warps of a tile");
     using TT = HaarTile<L>;
     using C = Cfg<T, I8, WPT>;
     using Ring = TileRing<T, L, C::CB, C::S>;
@@ -82,6 +98,7 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
     uint64_t* ring_bars = reinterpret_cast<uint64_t*>(sB + (size_t)kchunks * pr.npad * 16);   // [CWARPS][S]
     Ctl* ctl = reinterpret_cast<Ctl*>(ring_bars + C::CWARPS * C::S);
     float* sscale = reinterpret_cast<float*>(ctl + 1);                        // [npad]
+    float4* stok = reinterpret_cast<float4*>((reinterpret_cast<uintptr_t>(sscale + pr.npad) + 15) & ~(uintptr_t)15);   // NEXT: [TILES][2][4][32]
     volatile int* abort_flag = &ctl->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -92,6 +109,7 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
     if (threadIdx.x == 0) {
         for (int i = 0; i < MAX_NA; ++i) { tc::mbar_init(tc::smem_u32(&ctl->full_a[i]), 2 * TILES); tc::mbar_init(tc::smem_u32(&ctl->empty_a[i]), 1); }
         for (int i = 0; i < 2; ++i) { tc::mbar_init(tc::smem_u32(&ctl->ready[i]), 1); tc::mbar_init(tc::smem_u32(&ctl->tfree[i]), C::CWARPS); }
+        for (int i = 0; i < TILES; ++i) { tc::mbar_init(tc::smem_u32(&ctl->tok[i][0]), 1); tc::mbar_init(tc::smem_u32(&ctl->tok[i][1]), 1); }
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -323,6 +341,17 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
         T* yout = static_cast<T*>(pr.y);
         const T* res = static_cast<const T*>(pr.residual);
         const bool coarse6 = L == 3 && ((lane / TT::CG) & 1) == 0;     // slot 6 holds a level-3 coefficient
+        // NEXT: the norm chain of the next layer's input.  Output channels leave in groups of eight that alternate between
+        // the two warps of a tile; the partial sums (one fused multiply-add per channel, ascending channel order, as the
+        // first pass builds them) and the running maxima travel with a token from the warp of group G to the warp of G + 1.
+        float2 nsum[4];
+        float nmax[8];
+        int tok_seen = 0;
+        const int last_group = (pr.Cout - 1) >> 3;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) nsum[i] = make_float2(0.0f, 0.0f);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) nmax[i] = 0.0f;
         for (int c = 0; c < pr.nn && ok; ++c) {
             const int tb = c % pr.nbuf;
             ok = tc::mbar_wait(tc::smem_u32(&ctl->ready[tb]), (uint32_t)(c / pr.nbuf) & 1u, abort_flag);
@@ -376,6 +405,73 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
                             store_patch<T, true>(yout + plane, pr.W, lp, p[d]);
                         }
                     }
+                    if (NEXT) {
+                        // what the next layer reads is the stored value: round to the activation type first.  Channels
+                        // beyond Cout have zero accumulators and get neither residual nor store: they add nothing.
+                        if (sizeof(T) == 2) {
+#pragma unroll
+                            for (int d = 0; d < 4; ++d)
+#pragma unroll
+                                for (int a = 0; a < 2; ++a)
+#pragma unroll
+                                    for (int b = 0; b < 4; ++b) p[d][a][b] = __bfloat162float(__float2bfloat16_rn(p[d][a][b]));
+                        }
+                        float o2[4][8];
+                        haar_fwd_lanes_raw<L, 4>(p, o2, lane);
+                        const int G = o0 >> 3;
+                        if (hh == 0 && G > 0) {            // partial sums and maxima of the channels before this group
+                            ok = ok && tc::mbar_wait(tc::smem_u32(&ctl->tok[t][q]), (uint32_t)tok_seen & 1u, abort_flag);
+                            ++tok_seen;
+                            const float4* tk = stok + ((size_t)(t * 2 + q) * 4) * 32;
+                            const float4 a0 = tk[lane], a1 = tk[32 + lane], m0 = tk[64 + lane], m1 = tk[96 + lane];
+                            nsum[0] = make_float2(a0.x, a0.y); nsum[1] = make_float2(a0.z, a0.w);
+                            nsum[2] = make_float2(a1.x, a1.y); nsum[3] = make_float2(a1.z, a1.w);
+                            nmax[0] = m0.x; nmax[1] = m0.y; nmax[2] = m0.z; nmax[3] = m0.w;
+                            nmax[4] = m1.x; nmax[5] = m1.y; nmax[6] = m1.z; nmax[7] = m1.w;
+                        }
+#pragma unroll
+                        for (int d = 0; d < 4; ++d) {
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const float2 v = make_float2(o2[d][2 * i], o2[d][2 * i + 1]);
+                                nsum[i] = __ffma2_rn(v, v, nsum[i]);
+                            }
+#pragma unroll
+                            for (int s = 0; s < 8; ++s) nmax[s] = fmaxf(nmax[s], fabsf(o2[d][s]));
+                        }
+                        if (hh == 1) {
+                            if (G < last_group) {          // hand over to the warp of the next group
+                                float4* tk = stok + ((size_t)(t * 2 + (q ^ 1)) * 4) * 32;
+                                tk[lane] = make_float4(nsum[0].x, nsum[0].y, nsum[1].x, nsum[1].y);
+                                tk[32 + lane] = make_float4(nsum[2].x, nsum[2].y, nsum[3].x, nsum[3].y);
+                                tk[64 + lane] = make_float4(nmax[0], nmax[1], nmax[2], nmax[3]);
+                                tk[96 + lane] = make_float4(nmax[4], nmax[5], nmax[6], nmax[7]);
+                                __syncwarp();
+                                if (lane == 0) tc::mbar_arrive(tc::smem_u32(&ctl->tok[t][q ^ 1]));
+                            } else if (ok) {               // last group: these are the next layer's norms of this tile
+                                float sc2[8], nacc[8], am[8];
+                                slot_scales<L>(lane, false, sc2);
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    nacc[2 * i] = __fmul_rn(nsum[i].x, __fmul_rn(sc2[2 * i], sc2[2 * i]));
+                                    nacc[2 * i + 1] = __fmul_rn(nsum[i].y, __fmul_rn(sc2[2 * i + 1], sc2[2 * i + 1]));
+                                }
+#pragma unroll
+                                for (int s = 0; s < 8; ++s) am[s] = __fmul_rn(nmax[s], fabsf(sc2[s]));
+                                store_slots<L, true>(pr.nx.nrm2 + (size_t)n * P, lp, nacc);
+                                store_slots<L, true>(pr.nx.amaxpos + (size_t)n * P, lp, am);
+                                uint32_t* h = pr.nx.hist1 + (size_t)n * 3 * 2048;      // zero norms are not counted
+#pragma unroll
+                                for (int s = 0; s < 8; ++s) hist_add(h, float_key(nacc[s]) >> 21, lp.ok0 && nacc[s] != 0.0f);
+                                if (lp.ok0) {
+                                    uint32_t* f = pr.nx.fine + (size_t)n * 65536;
+#pragma unroll
+                                    for (int s = 0; s < 8; ++s)
+                                        if (nacc[s] != 0.0f) atomicAdd(&f[float_key(nacc[s]) >> 16], 1u);
+                                }
+                            }
+                        }
+                    }
                 }
             }
             tc::fence_before();
@@ -408,7 +504,7 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
 // columns it takes, and whether the problem fits at all (ok).  Pure arithmetic: callers decide before anything is launched.
 struct FtPlan { int npad, nchunk, nn, nbuf, na, tmem_cols; size_t smem; bool ok; };
 
-static FtPlan ft_plan(const void* x, int esz, int W, int Cout, int kpad, int bits)
+static FtPlan ft_plan(const void* x, int esz, int W, int Cout, int kpad, int bits, bool next = false)
 {
     constexpr int WPT = 2, S = 4;                     // as instantiated below (Cfg<T, I8, 2>::S)
     FtPlan p = {};
@@ -426,6 +522,7 @@ static FtPlan ft_plan(const void* x, int esz, int W, int Cout, int kpad, int bit
     const size_t ring_bytes = (size_t)ft::TILES * WPT * S * 4096;
     p.smem = 128 + (size_t)p.na * ft::KSTEP_BYTES + ring_bytes + (size_t)kchunks * p.npad * 16 +
              (size_t)ft::TILES * WPT * 8 * 8 + sizeof(ft::Ctl) + (size_t)p.npad * 4 + 64;
+    if (next) p.smem += (size_t)ft::TILES * 2 * ft::TOKEN_BYTES + 16;
     p.ok = p.smem <= 227 * 1024;
     return p;
 }
@@ -435,15 +532,16 @@ template <typename T, int L>
 static wcc_status fused_tiles_dispatch(const void* x, const void* Wq, const int32_t* rank, const float* nrm2, const uint32_t* thr,
                                        const float* amax_kept, int bits, const float* scale_w, int N, int Cin, int Cout, int H,
                                        int W, int k, int kpad, void* y, void* xq_tap, int32_t* acc_tap, const FusedExtra& fx,
-                                       cudaStream_t st)
+                                       cudaStream_t st, const ft::NextNorms* nx = nullptr)
 {
     using TT = HaarTile<L>;
     constexpr int WPT = 2;
     static_assert(ft::Cfg<T, true, WPT>::S == 4 && ft::Cfg<T, false, WPT>::S == 4, "ft_plan assumes four boxes per ring");
     const bool i8 = bits >= 2;
-    const FtPlan plan = ft_plan(x, (int)sizeof(T), W, Cout, kpad, bits);
+    const FtPlan plan = ft_plan(x, (int)sizeof(T), W, Cout, kpad, bits, nx != nullptr);
     if (!plan.ok) return WCC_ERR_SHAPE;
     ft::Params pr = {};
+    if (nx) pr.nx = *nx;
     pr.npad = plan.npad; pr.nchunk = plan.nchunk; pr.nn = plan.nn; pr.nbuf = plan.nbuf; pr.na = plan.na; pr.tmem_cols = plan.tmem_cols;
     const size_t smem = plan.smem;
     const long long tiles = (long long)N * ceil_div(W, TT::TW) * (H / TT::TH);
@@ -463,17 +561,21 @@ static wcc_status fused_tiles_dispatch(const void* x, const void* Wq, const int3
         WCC_LAUNCH_CHECK();
         return WCC_OK;
     };
-    if (i8) return launch(ft::fused_tiles_kernel<T, L, true, WPT>, ft::Cfg<T, true, WPT>::THREADS);
-    return launch(ft::fused_tiles_kernel<T, L, false, WPT>, ft::Cfg<T, false, WPT>::THREADS);
+    if (nx) {
+        if (i8) return launch(ft::fused_tiles_kernel<T, L, true, WPT, true>, ft::Cfg<T, true, WPT>::THREADS);
+        return launch(ft::fused_tiles_kernel<T, L, false, WPT, true>, ft::Cfg<T, false, WPT>::THREADS);
+    }
+    if (i8) return launch(ft::fused_tiles_kernel<T, L, true, WPT, false>, ft::Cfg<T, true, WPT>::THREADS);
+    return launch(ft::fused_tiles_kernel<T, L, false, WPT, false>, ft::Cfg<T, false, WPT>::THREADS);
 }
 
 wcc_status launch_fused_tiles(const void* x, const void* Wq, const int32_t* rank, const float* nrm2, const uint32_t* thr,
                               const float* amax_kept, int bits, const float* scale_w, int N, int Cin, int Cout, int H, int W,
                               int L, int k, int kpad, wcc_dtype dt, void* y, void* xq_tap, int32_t* acc_tap, const FusedExtra& fx,
-                              cudaStream_t st)
+                              cudaStream_t st, const ft::NextNorms* nx = nullptr)
 {
     if ((W % 4) != 0) return WCC_ERR_SHAPE;
-#define WCC_FT(TY, LL) return fused_tiles_dispatch<TY, LL>(x, Wq, rank, nrm2, thr, amax_kept, bits, scale_w, N, Cin, Cout, H, W, k, kpad, y, xq_tap, acc_tap, fx, st)
+#define WCC_FT(TY, LL) return fused_tiles_dispatch<TY, LL>(x, Wq, rank, nrm2, thr, amax_kept, bits, scale_w, N, Cin, Cout, H, W, k, kpad, y, xq_tap, acc_tap, fx, st, nx)
     if (dt == WCC_F32) { if (L == 1) WCC_FT(float, 1); if (L == 2) WCC_FT(float, 2); WCC_FT(float, 3); }
     if (L == 1) WCC_FT(__nv_bfloat16, 1);
     if (L == 2) WCC_FT(__nv_bfloat16, 2);

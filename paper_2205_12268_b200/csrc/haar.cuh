@@ -609,6 +609,74 @@ haar_fwd_kernel(const T* __restrict__ x, int N, int C, int H, int W,
 }
 
 
+// ---- depthwise 3x3 convolution fused with the forward transform ------------------------------------------
+// The input of the block's second pointwise layer is a depthwise convolution of the expanded map (Eq. 13); both are
+// separable per channel, so the convolution's output never goes to memory: every lane computes the convolution at the
+// eight pixels of its patch (from a 4 x 6 neighbourhood of the input, zeros outside the map) and transforms them right
+// away.  Per output pixel: one fused multiply-add per tap, row-major tap order, starting from +0 (taps outside the map
+// contribute nothing).  Same work decomposition and outputs as haar_fwd_kernel; w is fp32 [C][3][3].
+template <typename T, int L, bool VEC>
+__global__ void __launch_bounds__(128)
+dwconv_haar_fwd_kernel(const T* __restrict__ u, const float* __restrict__ w, int N, int C, int H, int W,
+                       float* __restrict__ coef, float* __restrict__ nrm2, float* __restrict__ amaxpos)
+{
+    using TT = HaarTile<L>;
+    const int tiles_x = (W + TT::TW - 1) / TT::TW, tiles_y = H / TT::TH;
+    const int warp = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (warp >= N * tiles_x * tiles_y) return;
+    const int lane = threadIdx.x & 31;
+    int n, ty, tx;
+    tile_coords(warp, tiles_x, tiles_y, n, ty, tx);
+    const LanePos lp = lane_positions<L>(H, W, ty, tx, lane);
+    const size_t P = (size_t)H * W;
+    const T* uin = u + (size_t)n * C * P;
+    float* cout = coef ? coef + (size_t)n * C * P : nullptr;
+
+    float nacc[8], amax[8];
+#pragma unroll
+    for (int s = 0; s < 8; ++s) { nacc[s] = 0.0f; amax[s] = 0.0f; }
+    for (int c = 0; c < C; ++c) {
+        const T* plane = uin + (size_t)c * P;
+        float k9[9];
+#pragma unroll
+        for (int i = 0; i < 9; ++i) k9[i] = __ldg(w + (size_t)c * 9 + i);
+        float in[4][6];                                    // rows r0-1 .. r0+2, columns c0-1 .. c0+4
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int b = 0; b < 6; ++b) {
+                const int rr = lp.r0 + a - 1, cc = lp.c0 + b - 1;
+                float v = 0.0f;
+                if (rr >= 0 && rr < H && cc >= 0 && cc < W) {
+                    if (sizeof(T) == 4) v = __ldg(reinterpret_cast<const float*>(plane) + (size_t)rr * W + cc);
+                    else v = __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short*>(plane) + (size_t)rr * W + cc) << 16);
+                }
+                in[a][b] = v;
+            }
+        float p[2][4], o[8];
+#pragma unroll
+        for (int a = 0; a < 2; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                float acc = 0.0f;
+#pragma unroll
+                for (int i = 0; i < 3; ++i)
+#pragma unroll
+                    for (int j = 0; j < 3; ++j) acc = __fmaf_rn(k9[i * 3 + j], in[a + i][b + j], acc);
+                p[a][b] = acc;
+            }
+        haar_fwd_lane<L>(p, o, lane);
+        if (cout) store_slots<L, VEC>(cout + (size_t)c * P, lp, o);
+#pragma unroll
+        for (int s = 0; s < 8; ++s) {
+            nacc[s] = __fmaf_rn(o[s], o[s], nacc[s]);
+            amax[s] = fmaxf(amax[s], fabsf(o[s]));
+        }
+    }
+    if (nrm2) store_slots<L, VEC>(nrm2 + (size_t)n * P, lp, nacc);
+    if (amaxpos) store_slots<L, VEC>(amaxpos + (size_t)n * P, lp, amax);
+}
+
 // ---- per-warp asynchronous patch ring ------------------------------------------------------------
 // Each lane copies its own 2 x 4 patch of a few channels ahead of use with cp.async (global -> shared, no
 // registers held while the copy flies) and later reads back exactly the bytes it copied, so no barrier is needed:
@@ -1125,7 +1193,7 @@ template <typename T, int L, bool VEC, bool ACCF, int OCW>
 __global__ void __launch_bounds__(128)
 scatter_inv_kernel(const int32_t* __restrict__ acc, int ldc, const int32_t* __restrict__ rank,
                    const float* __restrict__ amax_kept, float qmax, const float* __restrict__ scale_w,
-                   int N, int Cout, int H, int W, int k, T* __restrict__ y)
+                   int N, int Cout, int H, int W, int k, T* __restrict__ y, const T* __restrict__ residual, int relu)
 {
     using TT = HaarTile<L>;
     const int tiles_x = (W + TT::TW - 1) / TT::TW, tiles_y = H / TT::TH;
@@ -1169,6 +1237,24 @@ scatter_inv_kernel(const int32_t* __restrict__ acc, int ldc, const int32_t* __re
                     sl[s] = ACCF ? __int_as_float(a) : __fmul_rn((float)a, sc);
                 }
                 haar_inv_lane<L>(sl, p, lane);
+                if (residual) {                        // the skip connection (Eq. 13): one fp32 addition per element
+                    RawPatch rr;
+                    float rp[2][4];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) rr.w[i] = 0u;
+                    load_patch<T, VEC>(residual + ((size_t)n * Cout + o) * P, W, lp, rr);
+                    unpack_patch<T>(rr, rp);
+#pragma unroll
+                    for (int a = 0; a < 2; ++a)
+#pragma unroll
+                        for (int b = 0; b < 4; ++b) p[a][b] = __fadd_rn(p[a][b], rp[a][b]);
+                }
+                if (relu) {
+#pragma unroll
+                    for (int a = 0; a < 2; ++a)
+#pragma unroll
+                        for (int b = 0; b < 4; ++b) p[a][b] = fmaxf(p[a][b], 0.0f);
+                }
                 store_patch<T, VEC>(y + ((size_t)n * Cout + o) * P, W, lp, p);
             }
         }
@@ -1250,6 +1336,26 @@ wcc_status launch_haar_norms(const void* x, int N, int C, int H, int W, int L, w
     WCC_DISPATCH_TLV(haar_norms_dispatch, dt, L, vec, x, N, C, H, W, nrm2, amaxpos, ex, st);
 }
 
+template <typename T, int L, bool VEC>
+static wcc_status dwconv_haar_dispatch(const void* u, const float* w, int N, int C, int H, int W, float* coef, float* nrm2,
+                                       float* amaxpos, cudaStream_t st)
+{
+    using TT = HaarTile<L>;
+    const long long warps = (long long)N * ceil_div(W, TT::TW) * (H / TT::TH);
+    const int blocks = (int)((warps + 3) / 4);
+    dwconv_haar_fwd_kernel<T, L, VEC><<<blocks, 128, 0, st>>>(static_cast<const T*>(u), w, N, C, H, W, coef, nrm2, amaxpos);
+    WCC_LAUNCH_CHECK();
+    return WCC_OK;
+}
+
+// Depthwise 3x3 convolution + forward Haar + norms (+ per-position max |coef|) in one pass over u.
+wcc_status launch_dwconv_haar_fwd(const void* u, const float* w, int N, int C, int H, int W, int L, wcc_dtype dt,
+                                  float* coef, float* nrm2, float* amaxpos, cudaStream_t st)
+{
+    const bool vec = (W % 4) == 0;
+    WCC_DISPATCH_TLV(dwconv_haar_dispatch, dt, L, vec, u, w, N, C, H, W, coef, nrm2, amaxpos, st);
+}
+
 wcc_status launch_haar_fwd(const void* x, int N, int C, int H, int W, int L, wcc_dtype dt,
                            float* coef, float* nrm2, float* amaxpos, cudaStream_t st)
 {
@@ -1278,7 +1384,8 @@ wcc_status launch_haar_inv(const float* coef, int N, int C, int H, int W, int L,
 template <typename T, int L, bool VEC>
 static wcc_status scatter_inv_dispatch(const int32_t* acc, int ldc, bool accf, const int32_t* rank,
                                        const float* amax_kept, float qmax, const float* scale_w,
-                                       int N, int Cout, int H, int W, int k, void* y, cudaStream_t st)
+                                       int N, int Cout, int H, int W, int k, void* y, const void* residual, int relu,
+                                       cudaStream_t st)
 {
     using TT = HaarTile<L>;
     constexpr int OCW = 8;
@@ -1286,22 +1393,25 @@ static wcc_status scatter_inv_dispatch(const int32_t* acc, int ldc, bool accf, c
     const int blocks = (int)((warps + 3) / 4);
     if (accf)
         scatter_inv_kernel<T, L, VEC, true, OCW><<<blocks, 128, 0, st>>>(acc, ldc, rank, amax_kept, qmax, scale_w,
-                                                                          N, Cout, H, W, k, static_cast<T*>(y));
+                                                                          N, Cout, H, W, k, static_cast<T*>(y),
+                                                                          static_cast<const T*>(residual), relu);
     else
         scatter_inv_kernel<T, L, VEC, false, OCW><<<blocks, 128, 0, st>>>(acc, ldc, rank, amax_kept, qmax, scale_w,
-                                                                           N, Cout, H, W, k, static_cast<T*>(y));
+                                                                           N, Cout, H, W, k, static_cast<T*>(y),
+                                                                           static_cast<const T*>(residual), relu);
     WCC_LAUNCH_CHECK();
     return WCC_OK;
 }
 
 wcc_status launch_scatter_inv(const int32_t* acc, int ldc, bool acc_is_float, const int32_t* rank,
                               const float* amax_kept, int bits, const float* scale_w,
-                              int N, int Cout, int H, int W, int L, int k, wcc_dtype dt, void* y, cudaStream_t st)
+                              int N, int Cout, int H, int W, int L, int k, wcc_dtype dt, void* y, cudaStream_t st,
+                              const void* residual, int relu)
 {
     const bool vec = (W % 4) == 0;
     const float qmax = (bits >= 2) ? (float)((1 << (bits - 1)) - 1) : 1.0f;
     WCC_DISPATCH_TLV(scatter_inv_dispatch, dt, L, vec, acc, ldc, acc_is_float, rank, amax_kept, qmax, scale_w,
-                     N, Cout, H, W, k, y, st);
+                     N, Cout, H, W, k, y, residual, relu, st);
 }
 
 }  // namespace wcc

@@ -26,7 +26,7 @@ static wcc_status check_forward_args(int N, int Cin, int Cout, int H, int W, int
 {
     wcc_status s = check_plane_args(N, Cin, H, W, L, dt);
     if (s != WCC_OK) return s;
-    if (Cout <= 0 || Cin > 256 || Cout > 256) return WCC_ERR_SHAPE;
+    if (Cout <= 0 || Cin > WCC_MAX_CHANNELS || Cout > WCC_MAX_CHANNELS) return WCC_ERR_SHAPE;
     if (k < 1 || (long long)k > (long long)H * W) return WCC_ERR_K;
     if (!(bits == 0 || (bits >= 2 && bits <= 8))) return WCC_ERR_BITS;
     if ((long long)N * k > (1LL << 30)) return WCC_ERR_SHAPE;
@@ -40,14 +40,12 @@ static bool fused_fits(const void* x, int Cout, int W, int bits, wcc_dtype dt, i
     return ft_plan(x, esz, W, Cout, kpad, bits).ok || fz_plan(esz, Cout, kpad, bits).ok;
 }
 
-// Can the staged contraction kernel run it?  (Mirrors launch_contract.)
+// Can the staged contraction kernel run it?  (Mirrors launch_contract: K is a loop and N is tiled, so only the
+// 32-byte granularity of a K step remains, which wcc_kpad guarantees.)
 static bool staged_fits(int Cin, int Cout, int bits)
 {
-    const int krow_bytes = wcc_kpad(Cin, bits) * (bits >= 2 ? 1 : 2);
-    const int katoms = ceil_div(krow_bytes, tc::ATOM_BYTES), npad = ceil_div(Cout, 16) * 16;
-    if (katoms > tc::MAX_KATOMS || npad > 256 || (krow_bytes % 32) != 0) return false;
-    const size_t smem = 1024 + (size_t)katoms * npad * tc::ATOM_BYTES + (size_t)tc::STAGES * katoms * tc::A_ATOM_BYTES + sizeof(tc::SmemCtl) + 16;
-    return smem <= 200 * 1024;
+    (void)Cout;
+    return (wcc_kpad(Cin, bits) * (bits >= 2 ? 1 : 2)) % 32 == 0;
 }
 
 struct FwdWs {
@@ -139,13 +137,20 @@ __global__ void scale_tap_kernel(const float* amax_kept, float alpha, float qmax
     *out = __fdiv_rn(alpha > 0.0f ? alpha : *amax_kept, qmax);
 }
 
+static wcc_status check_options(const wcc_options* o, int bits, const void* x, const void* y);
+__global__ void set_word_kernel(float* dst, float v) { *dst = v; }
+
+// dwk: NULL, or depthwise 3x3 kernels fp32 [Cin][3][3] applied to x before the transform (one fused pass).
 static wcc_status staged_impl(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int W,
                                int L, int k, int bits, void* y, wcc_dtype dt, void* ws, size_t ws_bytes,
-                               cudaStream_t st, const wcc_taps* taps)
+                               cudaStream_t st, const wcc_taps* taps, const wcc_options* opt = nullptr,
+                               const float* dwk = nullptr)
 {
     if (!x || !Wt || !y || !ws) return WCC_ERR_NULL;
     wcc_status s = check_forward_args(N, Cin, Cout, H, W, L, k, bits, dt);
     if (s != WCC_OK) return s;
+    if ((s = check_options(opt, bits, x, y)) != WCC_OK) return s;
+    if (opt && opt->Wq) return WCC_ERR_SHAPE;          // pre-quantized weights: fused path only
     if (!aligned16(x) || !aligned16(Wt) || !aligned16(y) || (reinterpret_cast<uintptr_t>(ws) & 255u)) return WCC_ERR_ALIGN;
     if (!staged_fits(Cin, Cout, bits)) return WCC_ERR_SHAPE;          // decided before anything is launched
     const FwdWs f = carve_forward_ws(ws, N, Cin, Cout, H, W, k, bits);
@@ -154,14 +159,19 @@ static wcc_status staged_impl(const void* x, const float* Wt, int N, int Cin, in
 
     if ((s = profile_mark(0, st)) != WCC_OK) return s;
     // A: Haar transform + channel norms (and the per-position max |coef| the activation scale is taken from)
-    s = launch_haar_fwd(x, N, Cin, H, W, L, dt, f.coef, f.nrm2, f.amaxpos, st);
+    s = dwk ? launch_dwconv_haar_fwd(x, dwk, N, Cin, H, W, L, dt, f.coef, f.nrm2, f.amaxpos, st)
+            : launch_haar_fwd(x, N, Cin, H, W, L, dt, f.coef, f.nrm2, f.amaxpos, st);
     if (s != WCC_OK) return s;
     if ((s = profile_mark(1, st)) != WCC_OK) return s;
     // B: joint shrinkage: kept index list, rank map, max |kept|
     s = launch_select(f.nrm2, N, P, k, f.idx, nullptr, f.rank, f.amaxpos, true, f.sel, f.sel_bytes, st);
     if (s != WCC_OK) return s;
+    if (opt && opt->alpha > 0.0f && bits >= 2) {        // a given clipping parameter replaces the largest kept magnitude
+        set_word_kernel<<<1, 1, 0, st>>>(f.amax_kept, opt->alpha);
+        WCC_LAUNCH_CHECK();
+    }
     if ((s = profile_mark(2, st)) != WCC_OK) return s;
-    s = launch_weight_prep(Wt, Cout, Cin, f.kpad, bits, f.Wq, f.scale_w, st);
+    s = launch_weight_prep(Wt, Cout, Cin, f.kpad, (opt && opt->weight_bits && bits) ? opt->weight_bits : bits, f.Wq, f.scale_w, st);
     if (s != WCC_OK) return s;
     if ((s = profile_mark(3, st)) != WCC_OK) return s;
     s = launch_gather_quant(f.coef, f.idx, f.amax_kept, N, Cin, P, k, f.kpad, bits, f.Xq, st);
@@ -172,7 +182,8 @@ static wcc_status staged_impl(const void* x, const float* Wt, int N, int Cin, in
     if (s != WCC_OK) return s;
     if ((s = profile_mark(5, st)) != WCC_OK) return s;
     // D + E: dequantize, zero-fill, inverse transform
-    s = launch_scatter_inv(f.acc, f.ldc, bits == 0, f.rank, f.amax_kept, bits, f.scale_w, N, Cout, H, W, L, k, dt, y, st);
+    s = launch_scatter_inv(f.acc, f.ldc, bits == 0, f.rank, f.amax_kept, bits, f.scale_w, N, Cout, H, W, L, k, dt, y, st,
+                           opt ? opt->residual : nullptr, opt ? opt->relu : 0);
     if (s != WCC_OK) return s;
     if ((s = profile_mark(6, st)) != WCC_OK) return s;
 
@@ -235,20 +246,34 @@ static FusedWs carve_fused_ws(void* ws, int N, int Cin, int Cout, int H, int W, 
 
 static wcc_status check_options(const wcc_options* o, int bits, const void* x, const void* y)
 {
+    (void)y;
     if (!o) return WCC_OK;
     if (o->weight_bits != 0 && (bits == 0 || o->weight_bits < 2 || o->weight_bits > 8)) return WCC_ERR_BITS;
     if (o->alpha != o->alpha || o->alpha > 3.0e38f) return WCC_ERR_SHAPE;      // NaN or infinite clipping parameter
     if ((o->Wq != nullptr) != (o->scale_w != nullptr)) return WCC_ERR_NULL;
     if (o->Wq && bits == 0) return WCC_ERR_BITS;                               // codes only exist on the quantized path
     if (!aligned16(o->residual) || !aligned16(o->Wq) || !aligned16(o->scale_w)) return WCC_ERR_ALIGN;
-    if (o->residual && o->residual == y) return WCC_OK;                        // in-place accumulation into y is allowed
     (void)x;
     return WCC_OK;
 }
 
+// Chain fusion hooks of forward_impl: norms_ready = the previous layer's second pass has already produced this layer's
+// norms, per-position maxima and histograms in this workspace (no first pass; the weights are quantized by a launch of
+// their own); next_ws = workspace of the next layer, whose first pass this layer's second pass performs.
+struct ChainHooks { bool norms_ready; void* next_ws; int next_cout; };
+
+// Can the second pass of layer (Cin -> Cout) also be the first pass of a next layer?  (The four-tile kernel with room
+// for the tokens, one cluster per image in the selection.)
+static bool chain_fusable(const void* x, int Cin, int Cout, int H, int W, int bits, wcc_dtype dt)
+{
+    const int esz = (dt == WCC_BF16) ? 2 : 4;
+    return select_in_cluster(H * W) && ft_plan(x, esz, W, Cout, wcc_kpad(Cin, bits), bits, true).ok;
+}
+
 static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int W,
                                int L, int k, int bits, void* y, wcc_dtype dt, void* ws, size_t ws_bytes,
-                               cudaStream_t st, const wcc_taps* taps, const wcc_options* opt = nullptr)
+                               cudaStream_t st, const wcc_taps* taps, const wcc_options* opt = nullptr,
+                               const ChainHooks* hooks = nullptr)
 {
     const bool own_codes = opt && opt->Wq;             // weights arrive quantized: Wt is not read
     if (!x || (!Wt && !own_codes) || !y || !ws) return WCC_ERR_NULL;
@@ -258,7 +283,10 @@ static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, i
     if (!aligned16(x) || !aligned16(Wt) || !aligned16(y) || (reinterpret_cast<uintptr_t>(ws) & 255u)) return WCC_ERR_ALIGN;
     if (taps && (!aligned16(taps->coef) || !aligned16(taps->Xq) || !aligned16(taps->Xb) || !aligned16(taps->acc)))
         return WCC_ERR_ALIGN;
-    if (!fused_fits(x, Cout, W, bits, dt, Cin)) return WCC_ERR_SHAPE;   // decided before anything is launched
+    if (!fused_fits(x, Cout, W, bits, dt, Cin)) {      // decided before anything is launched: channel counts beyond one
+        if (own_codes) return WCC_ERR_SHAPE;           // operand tile run stage by stage (the contraction there tiles K and N)
+        return staged_impl(x, Wt, N, Cin, Cout, H, W, L, k, bits, y, dt, ws, ws_bytes, st, taps, opt);
+    }
     const FusedWs f = carve_fused_ws(ws, N, Cin, Cout, H, W, k, bits);
     if (ws_bytes < f.total) return WCC_ERR_WORKSPACE;
     const int P = H * W, M = N * k;
@@ -268,7 +296,9 @@ static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, i
     // coefficient map is written only when a test asks for it).  The same launch fills round 1 of the select's
     // histogram and quantizes the weights in a few extra CTAs.
     const SelectWs sw = carve_select_ws(f.sel, N, P);
-    WCC_CUDA_TRY(cudaMemsetAsync(f.fine, 0, f.fine_bytes + sw.zero_bytes, st));   // histograms, max |kept|, barrier counters
+    const bool norms_ready = hooks && hooks->norms_ready;
+    if (!norms_ready)
+        WCC_CUDA_TRY(cudaMemsetAsync(f.fine, 0, f.fine_bytes + sw.zero_bytes, st));   // histograms, max |kept|, barrier counters
     if ((s = profile_mark(1, st)) != WCC_OK) return s;
     NormsExtra ex = {};
     ex.coef = taps ? taps->coef : nullptr;
@@ -279,8 +309,15 @@ static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, i
     const void* Wq_use = own_codes ? static_cast<const void*>(opt->Wq) : f.Wq;
     const float* scale_w_use = own_codes ? opt->scale_w : f.scale_w;
     const FusedExtra fx = {opt ? opt->alpha : 0.0f, opt ? opt->relu : 0, opt ? opt->residual : nullptr};
-    s = launch_haar_norms(x, N, Cin, H, W, L, dt, f.nrm2, f.amaxpos, ex, st);
-    if (s != WCC_OK) return s;
+    if (norms_ready) {
+        if (!own_codes) {
+            s = launch_weight_prep(Wt, Cout, Cin, f.kpad, wbits, f.Wq, f.scale_w, st);
+            if (s != WCC_OK) return s;
+        }
+    } else {
+        s = launch_haar_norms(x, N, Cin, H, W, L, dt, f.nrm2, f.amaxpos, ex, st);
+        if (s != WCC_OK) return s;
+    }
     if ((s = profile_mark(2, st)) != WCC_OK) return s;
     // joint shrinkage: index list, rank map, max |kept|
     s = launch_select(f.nrm2, N, P, k, f.idx, nullptr, f.rank, f.amaxpos, true, f.sel, f.sel_bytes, st, true,
@@ -289,8 +326,19 @@ static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, i
     if ((s = profile_mark(3, st)) != WCC_OK) return s;
     // second pass over x: transform, mask + quantize, tensor-core contraction, dequantize, inverse, store
     void* xq_tap = taps ? (bits >= 2 ? static_cast<void*>(taps->Xq) : taps->Xb) : nullptr;
+    ft::NextNorms nx = {};
+    const bool feeds_next = hooks && hooks->next_ws;
+    if (feeds_next) {
+        // the next layer's workspace (its input has Cout channels): clear its histograms, then let this layer's second
+        // pass fill its norms, maxima and histograms
+        const FusedWs g = carve_fused_ws(hooks->next_ws, N, Cout, hooks->next_cout, H, W, k, bits);
+        const SelectWs gs = carve_select_ws(g.sel, N, P);
+        WCC_CUDA_TRY(cudaMemsetAsync(g.fine, 0, g.fine_bytes + gs.zero_bytes, st));
+        nx.nrm2 = g.nrm2; nx.amaxpos = g.amaxpos; nx.hist1 = gs.hist; nx.fine = g.fine;
+    }
     s = launch_fused_tiles(x, Wq_use, f.rank, f.nrm2, f.thr, f.amax_kept, bits, scale_w_use, N, Cin, Cout, H, W, L, k, f.kpad, dt, y,
-                           xq_tap, taps ? taps->acc : nullptr, fx, st);
+                           xq_tap, taps ? taps->acc : nullptr, fx, st, feeds_next ? &nx : nullptr);
+    if (feeds_next && s != WCC_OK) return s == WCC_ERR_SHAPE ? WCC_ERR_CUDA : s;       // (chain_fusable said it fits)
     if (s == WCC_ERR_SHAPE)                            // shapes the four-tile kernel does not cover (nothing was launched)
         s = launch_fused_pass2(x, Wq_use, f.rank, f.nrm2, f.thr, f.amax_kept, bits, scale_w_use, N, Cin, Cout, H, W, L, k, f.kpad, dt, y,
                                xq_tap, taps ? taps->acc : nullptr, fx, st);
@@ -390,8 +438,28 @@ static PaddedWs carve_padded_ws(void* ws, int N, int Cin, int Cout, int H, int W
     return p;
 }
 
+// ---- inverted residual block -------------------------------------------------------------------------
+struct BlockWs { void* u; void* layer_ws; size_t layer_ws_bytes; size_t total; };
+
+static BlockWs carve_block_ws(void* ws, int N, int C, int E, int H, int W, int L, int k, int bits, wcc_dtype dt)
+{
+    BlockWs b = {};
+    const size_t es = (dt == WCC_BF16) ? 2 : 4;
+    const size_t w1 = wcc_workspace_bytes(N, C, E, H, W, L, k, bits, dt);
+    const size_t w3 = wcc_staged_workspace_bytes(N, E, C, H, W, L, k, bits, dt);
+    if (w1 == 0 || w3 == 0) return b;
+    char* base = static_cast<char*>(ws);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { char* p = base ? base + off : nullptr; off += align_up(bytes, 256); return p; };
+    b.u = take((size_t)N * E * H * W * es);
+    b.layer_ws_bytes = w1 > w3 ? w1 : w3;
+    b.layer_ws = take(b.layer_ws_bytes);
+    b.total = off;
+    return b;
+}
+
 // ---- chain of layers -------------------------------------------------------------------------------
-struct ChainWs { void* act[2]; void* layer_ws; size_t layer_ws_bytes; size_t total; };
+struct ChainWs { void* act[2]; void* layer_ws[2]; size_t layer_ws_bytes; size_t total; };
 
 static wcc_status chain_shapes_ok(const wcc_chain_layer* layers, int n_layers)
 {
@@ -420,7 +488,8 @@ static ChainWs carve_chain_ws(void* ws, const wcc_chain_layer* layers, int n_lay
     c.act[0] = take(act);
     c.act[1] = take(act);
     c.layer_ws_bytes = lw;
-    c.layer_ws = take(lw);
+    c.layer_ws[0] = take(lw);                          // consecutive layers alternate: a fused second pass writes the next
+    c.layer_ws[1] = take(lw);                          // layer's norms while it still reads its own
     c.total = off;
     return c;
 }
@@ -440,7 +509,8 @@ int wcc_kpad(int Cin, int bits)
 size_t wcc_workspace_bytes(int N, int Cin, int Cout, int H, int Wd, int levels, int k, int bits, wcc_dtype dt)
 {
     if (check_forward_args(N, Cin, Cout, H, Wd, levels, k, bits, dt) != WCC_OK) return 0;
-    if (!fused_fits(nullptr, Cout, Wd, bits, dt, Cin)) return 0;
+    if (!fused_fits(nullptr, Cout, Wd, bits, dt, Cin))                         // these shapes run stage by stage
+        return staged_fits(Cin, Cout, bits) ? carve_forward_ws(nullptr, N, Cin, Cout, H, Wd, k, bits).total : 0;
     return carve_fused_ws(nullptr, N, Cin, Cout, H, Wd, k, bits).total;
 }
 
@@ -517,6 +587,45 @@ wcc_status wcc_forward_ex(const void* x, const float* Wt, int N, int Cin, int Co
 {
     return forward_impl(x, Wt, N, Cin, Cout, H, Wd, levels, k, bits, y, dt, ws, ws_bytes,
                         static_cast<cudaStream_t>(stream), taps, opt);
+}
+
+wcc_status wcc_dwconv_haar_fwd(const void* u, const float* Wdw, int N, int C, int H, int Wd, int levels, wcc_dtype dt,
+                               float* coef, float* nrm2, void* stream)
+{
+    if (!u || !Wdw || !coef) return WCC_ERR_NULL;
+    wcc_status s = check_plane_args(N, C, H, Wd, levels, dt);
+    if (s != WCC_OK) return s;
+    if (!aligned16(u) || !aligned16(Wdw) || !aligned16(coef) || !aligned16(nrm2)) return WCC_ERR_ALIGN;
+    return launch_dwconv_haar_fwd(u, Wdw, N, C, H, Wd, levels, dt, coef, nrm2, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+size_t wcc_block_workspace_bytes(int N, int C, int E, int H, int Wd, int levels, int k, int bits, wcc_dtype dt)
+{
+    if (check_forward_args(N, C, E, H, Wd, levels, k, bits, dt) != WCC_OK) return 0;
+    return carve_block_ws(nullptr, N, C, E, H, Wd, levels, k, bits, dt).total;
+}
+
+wcc_status wcc_block_forward(const void* x, const float* W1, const float* Wdw, const float* W3, int N, int C, int E,
+                             int H, int Wd, int levels, int k, int bits, void* y, wcc_dtype dt,
+                             void* ws, size_t ws_bytes, void* stream)
+{
+    if (!x || !W1 || !Wdw || !W3 || !y || !ws) return WCC_ERR_NULL;
+    wcc_status s = check_forward_args(N, C, E, H, Wd, levels, k, bits, dt);
+    if (s != WCC_OK) return s;
+    if ((s = check_forward_args(N, E, C, H, Wd, levels, k, bits, dt)) != WCC_OK) return s;
+    if (!aligned16(x) || !aligned16(W1) || !aligned16(Wdw) || !aligned16(W3) || !aligned16(y) ||
+        (reinterpret_cast<uintptr_t>(ws) & 255u)) return WCC_ERR_ALIGN;
+    const BlockWs b = carve_block_ws(ws, N, C, E, H, Wd, levels, k, bits, dt);
+    if (b.total == 0) return WCC_ERR_SHAPE;
+    if (ws_bytes < b.total) return WCC_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // u = WCC(W1, x): C -> E channels
+    s = forward_impl(x, W1, N, C, E, H, Wd, levels, k, bits, b.u, dt, b.layer_ws, b.layer_ws_bytes, st, nullptr);
+    if (s != WCC_OK) return s;
+    // y = x + WCC(W3, dw3x3(u)): the depthwise convolution is fused with the second layer's transform
+    wcc_options o = {};
+    o.residual = x;
+    return staged_impl(b.u, W3, N, E, C, H, Wd, levels, k, bits, y, dt, b.layer_ws, b.layer_ws_bytes, st, nullptr, &o, Wdw);
 }
 
 size_t wcc_select_bitmap_workspace_bytes(int N, int P, int k)
@@ -607,15 +716,24 @@ wcc_status wcc_chain_forward(const void* x, const wcc_chain_layer* layers, int n
     const ChainWs c = carve_chain_ws(ws, layers, n_layers, N, H, Wd, levels, k, bits, dt);
     if (c.total == 0) return WCC_ERR_SHAPE;
     if (ws_bytes < c.total) return WCC_ERR_WORKSPACE;
+    // Layer i's second pass doubles as layer i+1's first pass (inverse transform, ReLU and the next forward transform
+    // on the same tile while it is in registers) wherever both layers run the four-tile kernel.
     const void* in = x;
+    bool norms_ready = false;
     for (int i = 0; i < n_layers; ++i) {
         void* out = (i + 1 == n_layers) ? y : c.act[i & 1];
         wcc_options o = {};
         o.alpha = layers[i].alpha;
         o.relu = layers[i].relu;
+        const bool this_fused = fused_fits(in, layers[i].Cout, Wd, bits, dt, layers[i].Cin);
+        const bool feed = this_fused && i + 1 < n_layers && chain_fusable(in, layers[i].Cin, layers[i].Cout, H, Wd, bits, dt) &&
+                          fused_fits(out, layers[i + 1].Cout, Wd, bits, dt, layers[i + 1].Cin) &&
+                          tc::tma_ok_x(out, dt == WCC_BF16 ? 2 : 4, Wd);
+        const ChainHooks hooks = {norms_ready, feed ? c.layer_ws[(i + 1) & 1] : nullptr, feed ? layers[i + 1].Cout : 0};
         s = forward_impl(in, layers[i].Wt, N, layers[i].Cin, layers[i].Cout, H, Wd, levels, k, bits, out, dt,
-                         c.layer_ws, c.layer_ws_bytes, static_cast<cudaStream_t>(stream), nullptr, &o);
+                         c.layer_ws[i & 1], c.layer_ws_bytes, static_cast<cudaStream_t>(stream), nullptr, &o, &hooks);
         if (s != WCC_OK) return s;
+        norms_ready = feed;
         in = out;
     }
     return WCC_OK;

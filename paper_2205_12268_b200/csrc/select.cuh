@@ -804,6 +804,9 @@ __global__ void thr_use_rank_kernel(uint32_t* thr, int N)
     if (n < N) { thr[n * 4 + 0] = 0u; thr[n * 4 + 1] = 0u; thr[n * 4 + 2] = 1u; }
 }
 
+// One cluster per image holds up to this many positions in registers (the path that uses a producer's histograms).
+inline bool select_in_cluster(int P) { return P <= 8 * CL_THREADS * CL_MAXKPT; }
+
 // hist1_ready: the caller has already cleared the zero region of the workspace (carve_select_ws(...).hist,
 // zero_bytes) and filled round 1 of the histogram (top 11 key bits of every norm) before this call.
 // fine / thr: see select_cluster_kernel; want_rank: idx (if non-NULL) and rank must be written even when the
@@ -837,7 +840,7 @@ wcc_status launch_select(const float* nrm2, int N, int P, int k, int32_t* idx, f
         (void)cudaGetLastError();
     }
     const int cs_cap = (devc >= 0 && devc < 64) ? max_cs[devc] : 8;
-    if (P <= 8 * CL_THREADS * CL_MAXKPT) {
+    if (select_in_cluster(P)) {
         // as many CTAs per image as useful, then as few threads as hold the keys (<= 16 each): the per-thread cost of
         // the scans and barriers is fixed, so fewer, busier threads finish sooner
         int cs = 1;

@@ -23,7 +23,8 @@ EXPORTS = ("wcc_staged_workspace_bytes", "wcc_forward_staged", "wcc_workspace_by
            "wcc_profile_enable", "wcc_profile_read", "wcc_kernel_launches", "wcc_select_topk_static",
            "wcc_debug_set_wait_limit", "wcc_debug_wait_selftest", "wcc_forward_ex", "wcc_chain_workspace_bytes",
            "wcc_chain_forward", "wcc_select_bitmap_workspace_bytes", "wcc_select_topk_bitmap",
-           "wcc_padded_workspace_bytes", "wcc_forward_padded")
+           "wcc_padded_workspace_bytes", "wcc_forward_padded", "wcc_dwconv_haar_fwd", "wcc_block_workspace_bytes",
+           "wcc_block_forward")
 STATIC_SCRATCH_BYTES = 512 * 1024
 STAGES = ("haar_fwd_norms", "select_topk", "weight_quant", "gather_quant", "contract", "scatter_inv")   # wcc_forward_staged
 FUSED_STAGES = ("clear", "haar_norms", "select_topk", "fused_pass2")                                      # wcc_forward
@@ -93,6 +94,12 @@ def lib() -> C.CDLL:
         L.wcc_padded_workspace_bytes.argtypes = [i] * 9
         L.wcc_forward_padded.restype = i
         L.wcc_forward_padded.argtypes = fwd
+        L.wcc_dwconv_haar_fwd.restype = i
+        L.wcc_dwconv_haar_fwd.argtypes = [vp, vp, i, i, i, i, i, i, vp, vp, vp]
+        L.wcc_block_workspace_bytes.restype = sz
+        L.wcc_block_workspace_bytes.argtypes = [i] * 9
+        L.wcc_block_forward.restype = i
+        L.wcc_block_forward.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, i, vp, i, vp, sz, vp]
         L.wcc_chain_workspace_bytes.restype = sz
         L.wcc_chain_workspace_bytes.argtypes = [C.POINTER(ChainLayer), i, i, i, i, i, i, i, i]
         L.wcc_chain_forward.restype = i
@@ -158,6 +165,50 @@ def haar_fwd(x: torch.Tensor, levels: int, want_norms: bool = True):
     _check(lib().wcc_haar_fwd(x.data_ptr(), N, Cc, H, W, levels, _dt(x), coef.data_ptr(), _ptr(nrm2), _stream()),
            "wcc_haar_fwd")
     return coef, nrm2
+
+
+def dwconv_haar_fwd(u: torch.Tensor, Wdw: torch.Tensor, levels: int):
+    """Depthwise 3x3 convolution (Wdw fp32 [C][3][3]) fused with the forward transform -> (coef, nrm2) as ``haar_fwd``."""
+    _dev(u, "u")
+    _dev(Wdw, "Wdw")
+    N, Cc, H, W = u.shape
+    if Wdw.dtype != torch.float32 or tuple(Wdw.shape) != (Cc, 3, 3):
+        raise ValueError("Wdw must be float32 [C][3][3]")
+    coef = torch.empty((N, Cc, H, W), dtype=torch.float32, device=u.device)
+    nrm2 = torch.empty((N, H * W), dtype=torch.float32, device=u.device)
+    _check(lib().wcc_dwconv_haar_fwd(u.data_ptr(), Wdw.data_ptr(), N, Cc, H, W, levels, _dt(u), coef.data_ptr(),
+                                     nrm2.data_ptr(), _stream()), "wcc_dwconv_haar_fwd")
+    return coef, nrm2
+
+
+class Block:
+    """The inverted residual block y = x + WCC(W3, dw3x3(Wdw, WCC(W1, x))) (wcc_block_forward); the workspace, which
+    also holds the expanded map, is allocated once, here."""
+
+    def __init__(self, x: torch.Tensor, W1: torch.Tensor, Wdw: torch.Tensor, W3: torch.Tensor, levels: int, k: int, bits: int = 8):
+        _dev(x, "x")
+        for t, name in ((W1, "W1"), (Wdw, "Wdw"), (W3, "W3")):
+            _dev(t, name)
+            if t.dtype != torch.float32:
+                raise TypeError("%s must be float32" % name)
+        self.N, self.C, self.H, self.W = x.shape
+        self.E = W1.shape[0]
+        if tuple(W1.shape) != (self.E, self.C) or tuple(Wdw.shape) != (self.E, 3, 3) or tuple(W3.shape) != (self.C, self.E):
+            raise ValueError("W1 [E][C], Wdw [E][3][3], W3 [C][E] expected")
+        self.W1, self.Wdw, self.W3, self.levels, self.k, self.bits, self.dt = W1, Wdw, W3, levels, k, bits, _dt(x)
+        n = int(lib().wcc_block_workspace_bytes(self.N, self.C, self.E, self.H, self.W, levels, k, bits, self.dt))
+        if n == 0:
+            raise WccError(2, "wcc_block_workspace_bytes")
+        self.ws = Workspace(n, x.device)
+
+    def __call__(self, x: torch.Tensor, y: torch.Tensor | None = None) -> torch.Tensor:
+        _dev(x, "x")
+        if y is None:
+            y = torch.empty_like(x)
+        _check(lib().wcc_block_forward(x.data_ptr(), self.W1.data_ptr(), self.Wdw.data_ptr(), self.W3.data_ptr(), self.N,
+                                       self.C, self.E, self.H, self.W, self.levels, self.k, self.bits, y.data_ptr(), self.dt,
+                                       self.ws.buf.data_ptr(), self.ws.nbytes, _stream()), "wcc_block_forward")
+        return y
 
 
 def haar_inv(coef: torch.Tensor, levels: int, dtype: torch.dtype = torch.float32) -> torch.Tensor:

@@ -1,0 +1,97 @@
+"""GPU parity of the fused depthwise-3x3 + Haar kernel, of the inverted residual block (Eq. 13) and of layers with
+channel counts beyond one operand tile (the contraction tiles K and N), against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2205_12268_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def wcc():
+    from paper_2205_12268_b200 import build, wcc as w
+    build.build()
+    assert torch.cuda.is_available()
+    w.lib()
+    return w
+
+
+def _dev(x, dtype):
+    if dtype == "bf16":
+        b = inputs.f32_to_bf16_bits(x)
+        return torch.from_numpy(b.view(np.int16)).cuda().view(torch.bfloat16), inputs.bf16_bits_to_f32(b)
+    return torch.from_numpy(x).cuda(), x
+
+
+def _bits(a):
+    return np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shape", [(1, 3, 8, 8, 3), (2, 5, 16, 24, 1), (2, 5, 16, 24, 2), (1, 2, 4, 6, 1), (2, 9, 40, 200, 3),
+                                   (1, 17, 96, 96, 3)])
+def test_dwconv_haar_fwd_bit_exact(wcc, shape, dtype):
+    N, Cc, H, W, L = shape
+    rng = np.random.default_rng(17)
+    u = inputs.feature_map(12, N, Cc, H, W, 4, 3.0).astype(np.float32)
+    k9 = rng.standard_normal((Cc, 3, 3)).astype(np.float32)
+    ud, uh = _dev(u, dtype)
+    coef, nrm2 = wcc.dwconv_haar_fwd(ud, torch.from_numpy(k9).cuda(), L)
+    assert wcc.last_status() == 0
+    want = oracle.haar_fwd(oracle.dwconv3x3(uh, k9), L)
+    assert np.array_equal(_bits(coef.cpu().numpy()), _bits(want))
+    assert np.array_equal(_bits(nrm2.cpu().numpy()), _bits(oracle.norms(want)))
+
+
+LARGE = [  # N, Cin, Cout, H, W, dtype, levels, gamma, bits
+    (1, 512, 1024, 96, 96, "bf16", 3, 0.25, 8),     # the paper's GPU benchmark has layers of this size
+    (1, 1024, 512, 32, 32, "f32", 3, 0.25, 8),
+    (2, 300, 520, 16, 32, "f32", 2, 0.5, 8),        # ragged K atom and a ragged column tile
+    (1, 256, 256, 16, 32, "f32", 3, 0.6, 0),        # unquantized at the channel counts the fused kernels do not hold
+    (1, 256, 128, 16, 32, "f32", 3, 0.6, 0),
+    (1, 640, 264, 16, 32, "bf16", 3, 0.5, 0),
+]
+
+
+@pytest.mark.parametrize("cfg", LARGE, ids=lambda c: "N%d_%dto%d_%dx%d_%s_L%d_g%s_b%d" % c)
+def test_layer_with_many_channels(wcc, cfg):
+    N, Cin, Cout, H, W, dtype, L, gamma, bits = cfg
+    w = inputs.custom("wide", 41, N, Cin, Cout, H, W, dtype, L, gamma, bits, n_sin=4, fmax=3.0)
+    x = torch.from_numpy(w.x.view(np.int16)).cuda().view(torch.bfloat16) if dtype == "bf16" else torch.from_numpy(w.x).cuda()
+    y, t = wcc.forward(x, torch.from_numpy(w.Wt).cuda(), L, w.k, bits, taps=True)
+    assert wcc.last_status() == 0
+    want, o = oracle.forward(w.x_f32(), w.Wt, L, w.k, bits, out_bf16=(dtype == "bf16"), taps=True)
+    assert np.array_equal(t["idx"].cpu().numpy(), o["idx"])
+    if bits:
+        assert np.array_equal(t["acc"].cpu().numpy(), o["acc"].reshape(-1, Cout))
+        assert np.array_equal(_bits(y.float().cpu().numpy()), _bits(want))
+    else:
+        assert np.abs(y.float().cpu().numpy() - want).max() <= 2e-2 * np.abs(want).max()
+
+
+BLOCKS = [  # N, C, E, H, W, dtype, levels, gamma
+    (2, 8, 32, 16, 32, "f32", 2, 0.5),
+    (1, 16, 96, 32, 64, "bf16", 3, 0.25),
+    (2, 128, 512, 32, 32, "bf16", 3, 0.25),         # expansion 4 at 128 channels, as in the paper's timing table
+    (1, 256, 1024, 24, 24, "f32", 3, 0.125),
+]
+
+
+@pytest.mark.parametrize("cfg", BLOCKS, ids=lambda c: "N%d_c%d_e%d_%dx%d_%s_L%d_g%s" % c)
+def test_inverted_residual_block(wcc, cfg):
+    N, Cc, E, H, W, dtype, L, gamma = cfg
+    rng = np.random.default_rng(E)
+    x0 = inputs.feature_map(13, N, Cc, H, W, 4, 3.0).astype(np.float32)
+    xd, xh = _dev(x0, dtype)
+    W1, W3 = inputs.weights(51, E, Cc), inputs.weights(52, Cc, E)
+    dw = (rng.standard_normal((E, 3, 3)) / 3).astype(np.float32)
+    k = inputs.keep_count(gamma, H * W)
+    blk = wcc.Block(xd, torch.from_numpy(W1).cuda(), torch.from_numpy(dw).cuda(), torch.from_numpy(W3).cuda(), L, k, 8)
+    y = blk(xd)
+    assert wcc.last_status() == 0
+    want = oracle.block(xh, W1, dw, W3, L, k, 8, out_bf16=(dtype == "bf16"))
+    assert np.array_equal(_bits(y.float().cpu().numpy()), _bits(want))
+    assert torch.equal(y, blk(xd))

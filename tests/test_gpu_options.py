@@ -151,6 +151,26 @@ def test_chain_small(wcc):
     _chain_case(wcc, 2, 32, 64, 3, 0.25, "bf16", alphas=[2.0, 3.0, 2.5, 3.0, 2.5, 3.0])
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("L", [1, 2, 3])
+def test_chain_with_odd_channel_counts(wcc, dtype, L):
+    """Channel counts that are no multiples of eight, a single group of output channels, several chunks of 32, ragged
+    tile groups: every layer's second pass also produces the next layer's norms, and the end result must still equal
+    the oracle's loop of single layers (which it can only do if every intermediate norm, threshold and scale did)."""
+    chans = [12, 20, 7, 40, 100, 9, 33]
+    N, H, W = 3, 24, 72
+    w0 = inputs.custom("oddchain", 60 + L, N, chans[0], chans[1], H, W, dtype, L, 0.3, 8, n_sin=4, fmax=3.0)
+    Ws = [inputs.weights(200 + i, chans[i + 1], chans[i]) for i in range(len(chans) - 1)]
+    x = _x_dev(w0)
+    for alphas in (None, [1.5, 0.0, 2.0, 0.0, 1.0, 0.0]):
+        ch = wcc.Chain(x, [torch.from_numpy(a).cuda() for a in Ws], L, w0.k, 8, alphas=alphas)
+        y = ch(x)
+        assert wcc.last_status() == 0
+        outs = oracle.chain(w0.x_f32(), Ws, L, w0.k, 8, out_bf16=(dtype == "bf16"), alphas=alphas)
+        assert np.array_equal(_bits(y.float().cpu().numpy()), _bits(outs[-1]))
+        assert torch.equal(y, ch(x))
+
+
 def test_chain_full_size(wcc):
     """The six-layer chain workload as the benchmark runs it: 2 x 256 x 512 bf16, three levels, a quarter kept."""
     outs = _chain_case(wcc, 2, 256, 512, 3, 0.25, "bf16")
