@@ -347,6 +347,54 @@ def chain_context(wcc, torch, np, inputs, dev, flush, peak, use_graph, steps=100
     return out
 
 
+def block_context(wcc, torch, np, inputs, dev, flush, steps=30):
+    """The inverted residual block of the paper's own GPU benchmark, y = x + K3(Kdw(K1 x)) with both pointwise
+    convolutions as WCC layers (three levels, 8 bits) at a few of its shapes, beside the same block with dense bf16
+    library kernels (matmul, grouped conv2d).  Batches are smaller than the paper's (its batches filled an 11 GB card)."""
+    import torch.nn.functional as F
+    shapes = [(8, 512, 2, 96, 96, 0.25), (4, 256, 4, 128, 128, 0.25), (2, 256, 4, 256, 256, 0.125), (2, 128, 4, 128, 128, 0.25)]
+    out = []
+    for (N, Cc, e, H, W, gamma) in shapes:
+        E = Cc * e
+        g = torch.Generator(device=dev).manual_seed(Cc + H)
+        x = torch.relu(torch.randn((N, Cc, H, W), device=dev, generator=g)).to(torch.bfloat16)
+        W1 = torch.randn((E, Cc), device=dev, generator=g) / Cc ** 0.5
+        W3 = torch.randn((Cc, E), device=dev, generator=g) / E ** 0.5
+        Wdw = torch.randn((E, 3, 3), device=dev, generator=g) / 3
+        k = inputs.keep_count(gamma, H * W)
+        blk = wcc.Block(x, W1, Wdw, W3, 3, k, 8)
+        y = torch.empty_like(x)
+
+        def timed(fn):
+            fn()
+            torch.cuda.synchronize()
+            ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+            for a, b in ev:
+                flush.fill_(1)
+                a.record()
+                fn()
+                b.record()
+            torch.cuda.synchronize()
+            t = [a.elapsed_time(b) for a, b in ev]
+            return sum(t) / len(t)
+
+        W1b, W3b, Wdwb = W1.to(torch.bfloat16), W3.to(torch.bfloat16), Wdw.to(torch.bfloat16)[:, None]
+
+        def dense():
+            u = torch.matmul(W1b, x.reshape(N, Cc, H * W)).reshape(N, E, H, W)
+            v = F.conv2d(u, Wdwb, padding=1, groups=E)
+            return x + torch.matmul(W3b, v.reshape(N, E, H * W)).reshape(N, Cc, H, W)
+
+        t_wcc = timed(lambda: blk(x, y))
+        t_dense = timed(dense)
+        out.append({"N": N, "c": Cc, "expansion": e, "H": H, "W": W, "keep": gamma, "wcc_block_ms": t_wcc,
+                    "dense_bf16_block_ms": t_dense, "dense_over_wcc": t_dense / t_wcc})
+        del blk, x, y
+        torch.cuda.empty_cache()
+    assert wcc.last_status() == 0
+    return out
+
+
 def run_ours(args):
     import numpy as np
     import torch
@@ -500,9 +548,10 @@ def run_ours(args):
                 del c
                 torch.cuda.empty_cache()
         assert wcc.last_status() == 0
-    chain = None
+    chain = blocks = None
     if not args.batch and not args.no_context:
         chain = chain_context(wcc, torch, np, inputs, dev, flush, peak, not args.no_graph)
+        blocks = block_context(wcc, torch, np, inputs, dev, flush)
     clocks_all = sampler.stop()
     timed = sampler.samples[:max(1, n_timed_samples)]
     clocks = {"sm_mhz": (statistics.median(timed) if timed else None), "sm_max_mhz": clocks_all["sm_max_mhz"],
@@ -538,7 +587,7 @@ def run_ours(args):
            "gpu_launches": int(case.launches_per_step * args.steps),
            "roofline": roofline, "cpu_baseline": cpu,
            "context": {"dense_1x1_matmul_ms": dense_ms, "ms_per_step_median": statistics.median(ms),
-                       "ms_per_step_min": min(ms), "workloads": workloads, "chain": chain}}
+                       "ms_per_step_min": min(ms), "workloads": workloads, "chain": chain, "inverted_residual_blocks": blocks}}
     print(json.dumps(out))
     if dist:
         dist.destroy_process_group()

@@ -79,10 +79,14 @@ struct Params {
     void* y; uint8_t* xq_tap; int32_t* acc_tap; int* status;
 };
 
-template <typename T, int L, bool I8, int WPT, bool NEXT>
+// MODE 0: the plain layer; 1: with the options (given clipping parameter, residual, ReLU); 2: residual / ReLU + next
+// layer's norms; 3: all options + next layer's norms.  The plain layer is a variant of its own so that it carries none
+// of the options' instructions and registers, and the chain's kernel clamps only when a clipping parameter is given.
+template <typename T, int L, bool I8, int WPT, int MODE>
 __global__ void __launch_bounds__(Cfg<T, I8, WPT>::THREADS, 1)
 fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
 {
+    constexpr bool OPTS = MODE >= 1, NEXT = MODE >= 2, CLAMP = MODE == 1 || MODE == 3;
     static_assert(!NEXT || WPT == 2, "the norm chain alternates between the two warps of a tile");
     using TT = HaarTile<L>;
     using C = Cfg<T, I8, WPT>;
@@ -171,7 +175,7 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
     for (int s = 0; s < 8; ++s) { mul[s] = 0.0f; rk[s] = -1; }
     // all independent loads first (threshold, norms, max |kept|), so that their latencies overlap
     float amax = 0.0f;
-    if (I8) amax = (pr.alpha > 0.0f) ? pr.alpha : *pr.amax_kept;
+    if (I8) amax = (CLAMP && pr.alpha > 0.0f) ? pr.alpha : *pr.amax_kept;
     if (live) {
         const uint4 th = *reinterpret_cast<const uint4*>(pr.thr + n * 4);      // {threshold key, ties kept, use-rank flag, -}
         float nv[8];
@@ -249,7 +253,7 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
         __syncwarp();
     } else {
         // ---- phase 1: transform + quantize into the A operand ---------------------------------------------
-        const bool clamp = I8 && pr.alpha > 0.0f;      // a given clipping parameter can be exceeded
+        const bool clamp = CLAMP && I8 && pr.alpha > 0.0f;     // a given clipping parameter can be exceeded
         const float qmax = pr.qmax;
         int m = 0;                                     // boxes consumed so far
         for (int ci = 0; ci < my_chunks && ok; ++ci) {
@@ -292,7 +296,7 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
                                 // written as fma(v, 1, 1.5*2^23): the product above keeps its own rounding (a packed add right
                                 // after the packed product gets contracted into one fused operation, which changes half-way codes).
                                 // clamping before the rounding is the same as after it: the bounds are integers
-                                if (clamp) { v.x = fminf(fmaxf(v.x, -qmax), qmax); v.y = fminf(fmaxf(v.y, -qmax), qmax); }
+                                if (CLAMP && clamp) { v.x = fminf(fmaxf(v.x, -qmax), qmax); v.y = fminf(fmaxf(v.y, -qmax), qmax); }
                                 if (I8) v = __ffma2_rn(v, make_float2(1.0f, 1.0f), make_float2(fz::MAGIC, fz::MAGIC));
                                 code[d][s] = __float_as_uint(v.x);
                                 code[d][s + 1] = __float_as_uint(v.y);
@@ -400,8 +404,8 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
                         const int o = o0 + hh * 4 + d;
                         if (o < pr.Cout) {
                             const size_t plane = ((size_t)n * pr.Cout + o) * P;
-                            if (res) fz::add_residual<T, true>(res + plane, pr.W, lp, p[d]);
-                            if (pr.relu) fz::relu_patch(p[d]);
+                            if (OPTS && res) fz::add_residual<T, true>(res + plane, pr.W, lp, p[d]);
+                            if (OPTS && pr.relu) fz::relu_patch(p[d]);
                             store_patch<T, true>(yout + plane, pr.W, lp, p[d]);
                         }
                     }
@@ -561,12 +565,17 @@ static wcc_status fused_tiles_dispatch(const void* x, const void* Wq, const int3
         WCC_LAUNCH_CHECK();
         return WCC_OK;
     };
+    if (nx && fx.alpha > 0.0f && i8) return launch(ft::fused_tiles_kernel<T, L, true, WPT, 3>, ft::Cfg<T, true, WPT>::THREADS);
     if (nx) {
-        if (i8) return launch(ft::fused_tiles_kernel<T, L, true, WPT, true>, ft::Cfg<T, true, WPT>::THREADS);
-        return launch(ft::fused_tiles_kernel<T, L, false, WPT, true>, ft::Cfg<T, false, WPT>::THREADS);
+        if (i8) return launch(ft::fused_tiles_kernel<T, L, true, WPT, 2>, ft::Cfg<T, true, WPT>::THREADS);
+        return launch(ft::fused_tiles_kernel<T, L, false, WPT, 2>, ft::Cfg<T, false, WPT>::THREADS);
     }
-    if (i8) return launch(ft::fused_tiles_kernel<T, L, true, WPT, false>, ft::Cfg<T, true, WPT>::THREADS);
-    return launch(ft::fused_tiles_kernel<T, L, false, WPT, false>, ft::Cfg<T, false, WPT>::THREADS);
+    if (fx.alpha > 0.0f || fx.relu || fx.residual) {
+        if (i8) return launch(ft::fused_tiles_kernel<T, L, true, WPT, 1>, ft::Cfg<T, true, WPT>::THREADS);
+        return launch(ft::fused_tiles_kernel<T, L, false, WPT, 1>, ft::Cfg<T, false, WPT>::THREADS);
+    }
+    if (i8) return launch(ft::fused_tiles_kernel<T, L, true, WPT, 0>, ft::Cfg<T, true, WPT>::THREADS);
+    return launch(ft::fused_tiles_kernel<T, L, false, WPT, 0>, ft::Cfg<T, false, WPT>::THREADS);
 }
 
 wcc_status launch_fused_tiles(const void* x, const void* Wq, const int32_t* rank, const float* nrm2, const uint32_t* thr,

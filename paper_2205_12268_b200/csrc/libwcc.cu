@@ -264,10 +264,16 @@ struct ChainHooks { bool norms_ready; void* next_ws; int next_cout; };
 
 // Can the second pass of layer (Cin -> Cout) also be the first pass of a next layer?  (The four-tile kernel with room
 // for the tokens, one cluster per image in the selection.)
+// It pays while the next layer's input is narrow: the extra transform and norm chain cost the second pass about 0.2 us
+// per output channel on a 2 x 256 x 512 map (192 channels: +41 us against a 31 us first pass of its own; 32 channels:
+// +12 us against 18 us), because the pass is bound by instruction issue, not by the bytes the fusion saves.
+constexpr int CHAIN_FUSE_MAX_CHANNELS = 64;
+
 static bool chain_fusable(const void* x, int Cin, int Cout, int H, int W, int bits, wcc_dtype dt)
 {
     const int esz = (dt == WCC_BF16) ? 2 : 4;
-    return select_in_cluster(H * W) && ft_plan(x, esz, W, Cout, wcc_kpad(Cin, bits), bits, true).ok;
+    return Cout <= CHAIN_FUSE_MAX_CHANNELS && select_in_cluster(H * W) &&
+           ft_plan(x, esz, W, Cout, wcc_kpad(Cin, bits), bits, true).ok;
 }
 
 static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int W,
