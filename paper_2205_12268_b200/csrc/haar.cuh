@@ -981,22 +981,24 @@ __device__ __noinline__ void tma_timeout(int* status)
 // of box r to the warp of box r + 1 through shared memory (a "token", signalled on an mbarrier).  So the sums are the
 // same sequential chains a single thread would build, while loads, unpacking, transforms and maxima of different boxes
 // overlap.  The transform runs without its halvings (haar_fwd_lanes_raw); one exact multiplication per slot at the end.
-template <typename T, int L>
+// NW warps share a tile (one CTA = one tile at a time): 4 when tiles are few and deep in channels, so that enough warps
+// are in flight; 1 when there are many tiles, which needs no hand-over at all (C4-like maps: 20.5 us instead of 24.5).
+template <typename T, int L, int NW_>
 struct NormsTokCfg {
-    static constexpr int W = 4;                                   // warps per tile
+    static constexpr int W = NW_;                                 // warps per tile
     static constexpr int CB = (sizeof(T) == 2) ? 8 : 4;           // channels per box: 4 KB
     static constexpr int S = 3;                                   // boxes in flight per warp
     using Ring = TileRing<T, L, CB, S>;
     static constexpr size_t SMEM = 128 + (size_t)W * Ring::BYTES + 8 * 32 * 4 + (size_t)W * 8 * 32 * 4 + (size_t)W * S * 8 + W * 8;
 };
 
-template <typename T, int L>
-__global__ void __launch_bounds__(NormsTokCfg<T, L>::W * 32, 4)
+template <typename T, int L, int NW_>
+__global__ void __launch_bounds__(NW_ * 32, 16 / NW_)
 haar_norms_token_kernel(const __grid_constant__ CUtensorMap tmx, int N, int C, int H, int W, int tiles_total, int tile_ctas,
                         float* __restrict__ nrm2, float* __restrict__ amaxpos, const NormsExtra ex, int* __restrict__ status)
 {
     using TT = HaarTile<L>;
-    using Cfg = NormsTokCfg<T, L>;
+    using Cfg = NormsTokCfg<T, L, NW_>;
     using Ring = typename Cfg::Ring;
     constexpr int CB = Cfg::CB, S = Cfg::S, NW = Cfg::W;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -1300,26 +1302,32 @@ static wcc_status haar_norms_dispatch(const void* x, int N, int C, int H, int W,
     using TT = HaarTile<L>;
     const long long tiles = (long long)N * ceil_div(W, TT::TW) * (H / TT::TH);
     if (VEC && tc::tma_ok_x(x, (int)sizeof(T), W)) {
-        using Cfg = NormsTokCfg<T, L>;
-        CUtensorMap tmx;
-        if (!tc::make_map_x(&tmx, x, (int)sizeof(T), N, C, H, W, TT::TW, TT::TH, Cfg::CB)) return WCC_ERR_CUDA;
-        int* status = nullptr;
-        WCC_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_status));
-        WCC_CUDA_TRY(cudaFuncSetAttribute(haar_norms_token_kernel<T, L>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM));
         if (tiles > 0x7FFFFFFFLL) return WCC_ERR_SHAPE;
         static int sm_count[64] = {0};
         int dev = 0;
         WCC_CUDA_TRY(cudaGetDevice(&dev));
         if (dev < 0 || dev >= 64) return WCC_ERR_CUDA;
         if (!sm_count[dev]) WCC_CUDA_TRY(cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev));
-        const long long resident = 4LL * sm_count[dev];                 // four CTAs per SM: every tile CTA is resident at once
-        const int tile_ctas = (int)(tiles < resident ? tiles : resident);
-        const long long grid = tile_ctas + (ex.Wt ? ceil_div(ex.Cout, Cfg::W) : 0);
+        int* status = nullptr;
+        WCC_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_status));
         ex.tiles = (int)tiles;
-        haar_norms_token_kernel<T, L><<<(unsigned)grid, Cfg::W * 32, Cfg::SMEM, st>>>(tmx, N, C, H, W, (int)tiles, tile_ctas, nrm2,
-                                                                                         amaxpos, ex, status);
-        WCC_LAUNCH_CHECK();
-        return WCC_OK;
+        // sixteen warps per SM are resident whatever the split: as many warps per tile as keeps them all busy
+        const long long warps = 16LL * sm_count[dev];
+        auto launch = [&](auto kern, auto cfg) -> wcc_status {
+            using Cfg = decltype(cfg);
+            CUtensorMap tmx;
+            if (!tc::make_map_x(&tmx, x, (int)sizeof(T), N, C, H, W, TT::TW, TT::TH, Cfg::CB)) return WCC_ERR_CUDA;
+            WCC_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM));
+            const long long resident = warps / Cfg::W;                  // every tile CTA is resident at once
+            const int tile_ctas = (int)(tiles < resident ? tiles : resident);
+            const long long grid = tile_ctas + (ex.Wt ? ceil_div(ex.Cout, Cfg::W) : 0);
+            kern<<<(unsigned)grid, Cfg::W * 32, Cfg::SMEM, st>>>(tmx, N, C, H, W, (int)tiles, tile_ctas, nrm2, amaxpos, ex, status);
+            WCC_LAUNCH_CHECK();
+            return WCC_OK;
+        };
+        if (tiles * 2 > warps) return launch(haar_norms_token_kernel<T, L, 1>, NormsTokCfg<T, L, 1>{});
+        if (tiles * 4 > warps) return launch(haar_norms_token_kernel<T, L, 2>, NormsTokCfg<T, L, 2>{});
+        return launch(haar_norms_token_kernel<T, L, 4>, NormsTokCfg<T, L, 4>{});
     }
     ex.tiles = (int)tiles;
     const long long grid = tiles + (ex.Wt ? ceil_div(ex.Cout, NORMS_WARPS) : 0);
