@@ -247,6 +247,53 @@ def block(x: np.ndarray, W1: np.ndarray, Wdw: np.ndarray, W3: np.ndarray, levels
     return (y, dict(u=u, v=v)) if taps else y
 
 
+def dwt(x: np.ndarray, levels: int, lo, hi, inverse: bool = False) -> np.ndarray:
+    """Multi-level 2-D wavelet transform of every plane with a two-channel filter bank (periodic extension, quadrant
+    layout): forward with the decomposition filters ``lo, hi``, or (``inverse``) the synthesis with the reconstruction
+    filters.  x float32 or float64 [N][C][H][W]; the taps are taken in x's precision."""
+    x = np.ascontiguousarray(x)
+    suf, ty = _real(x.dtype)
+    lo = np.ascontiguousarray(lo, dtype=x.dtype)
+    hi = np.ascontiguousarray(hi, dtype=x.dtype)
+    assert lo.shape == hi.shape and lo.ndim == 1
+    N, Cc, H, W = x.shape
+    out = np.empty_like(x)
+    rc = getattr(_L(), "orc_dwt_" + suf)(_p(x, ty), N, Cc, H, W, levels, _p(lo, ty), _p(hi, ty), lo.size, int(inverse), _p(out, ty))
+    if rc:
+        raise ValueError("orc_dwt rc=%d" % rc)
+    return out
+
+
+def forward_wavelet(x: np.ndarray, Wt: np.ndarray, levels: int, k: int, bits: int, dec_lo, dec_hi, rec_lo, rec_hi,
+                    out_bf16: bool = False, taps: bool = False):
+    """The WCC layer (Alg. 1) with another wavelet in place of Haar: the same steps, the transform and its inverse
+    swapped for the given filter bank.  The steps are composed here from the oracle's own parts."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    Wt = np.ascontiguousarray(Wt, dtype=np.float32)
+    N, Cin, H, W = x.shape
+    Cout, P = Wt.shape[0], H * W
+    coef = dwt(x, levels, dec_lo, dec_hi)
+    nrm2 = norms(coef)
+    idx, _ = select_topk(nrm2, k)
+    cols = np.stack([coef[n].reshape(Cin, P)[:, idx[n]].T for n in range(N)])            # [N][k][Cin]
+    t = dict(coef=coef.reshape(N, Cin, P), nrm2=nrm2, idx=idx)
+    if bits > 0:
+        Xq, scale_a = quantize(cols, bits)
+        Wq, scale_w = quantize_weights(Wt, bits)
+        acc = np.einsum("oc,nkc->nko", Wq.astype(np.int64), Xq.astype(np.int64)).astype(np.int32)
+        Yc = acc.astype(np.float32) * (np.float32(scale_a) * scale_w)[None, None, :]
+        t.update(Xq=Xq, scale_a=np.array([scale_a], np.float32), Wq=Wq, scale_w=scale_w, acc=acc)
+    else:
+        Yc = np.einsum("oc,nkc->nko", Wt.astype(np.float64), cols.astype(np.float64)).astype(np.float32)
+    Ywt = np.zeros((N, Cout, P), dtype=np.float32)
+    for n in range(N):
+        Ywt[n][:, idx[n]] = Yc[n].T
+    y = dwt(Ywt.reshape(N, Cout, H, W), levels, rec_lo, rec_hi, inverse=True)
+    if out_bf16:
+        y = round_bf16(y)
+    return (y, t) if taps else y
+
+
 def forward_f64(x: np.ndarray, Wt: np.ndarray, levels: int, k: int, idx_in: np.ndarray | None = None,
                 taps: bool = False):
     """The unquantized layer entirely in double (invariant tests)."""

@@ -126,6 +126,105 @@ int SUF(orc_haar_inv)(const REAL *coef, int N, int C, int H, int W, int levels, 
     return bad ? -2 : 0;
 }
 
+/* ---------------------------------------------------------------------------
+ * Other wavelets (App. F compares Haar with db2, db3, coif1, bior1.3, bior2.2, sym4: filters of 4 to 8 taps).
+ * A two-channel filter bank with T taps per filter (T even), periodic extension, so that an n-sample signal gives
+ * n/2 + n/2 coefficients and the transformed map has the size of the input (what the in-place compression needs;
+ * the paper does not name the extension).  One 2-D level on the hc x wc corner, as a stride-2 cross-correlation with
+ * the outer products of the 1-D decomposition filters, origin c0 = T/2 - 1:
+ *     band[i][j] = sum_{tr, tc} f_row[tr] * f_col[tc] * x[(2i + tr - c0) mod hc][(2j + tc - c0) mod wc]
+ * y1 = (lo, lo), y2 = (lo along the height, hi along the width), y3 = (hi, lo), y4 = (hi, hi); same quadrant
+ * placement as the Haar level above.  w2 holds the four T x T tap products, rounded once to REAL; one fused
+ * multiply-add per tap, row-major tap order, from +0.  With lo = [1, 1]/sqrt 2, hi = [1, -1]/sqrt 2 this is Eq. 3.
+ * ------------------------------------------------------------------------- */
+static void SUF(dwt_level_fwd)(const REAL *src, REAL *dst, int W, int hc, int wc, const REAL *w2, int T)
+{
+    const int h = hc / 2, w = wc / 2, c0 = T / 2 - 1;
+    for (int i = 0; i < h; ++i)
+        for (int j = 0; j < w; ++j)
+            for (int b = 0; b < 4; ++b) {
+                REAL acc = (REAL)0;
+                for (int tr = 0; tr < T; ++tr) {
+                    const int rr = ((2 * i + tr - c0) % hc + hc) % hc;
+                    for (int tc = 0; tc < T; ++tc) {
+                        const int cc = ((2 * j + tc - c0) % wc + wc) % wc;
+                        acc = FMA(w2[(b * T + tr) * T + tc], src[(size_t)rr * W + cc], acc);
+                    }
+                }
+                dst[(size_t)(i + (b >> 1) * h) * W + j + (b & 1) * w] = acc;
+            }
+}
+
+/* The synthesis step: the adjoint structure with the reconstruction filters (for an orthogonal wavelet they are the
+ * decomposition filters and this is the transpose, Eq. 4):
+ *     x[r][c] = sum over bands b, taps (tr, tc) with (r - tr + c0) mod hc and (c - tc + c0) mod wc both even
+ *               of g_row[tr] * g_col[tc] * band_b[((r - tr + c0) mod hc) / 2][((c - tc + c0) mod wc) / 2]
+ * summed in the order tr, tc, b, one fused multiply-add each, from +0. */
+static void SUF(dwt_level_inv)(const REAL *src, REAL *dst, int W, int hc, int wc, const REAL *v2, int T)
+{
+    const int h = hc / 2, w = wc / 2, c0 = T / 2 - 1;
+    for (int r = 0; r < hc; ++r)
+        for (int c = 0; c < wc; ++c) {
+            REAL acc = (REAL)0;
+            for (int tr = 0; tr < T; ++tr) {
+                const int mr = ((r - tr + c0) % hc + hc) % hc;
+                if (mr & 1) continue;
+                for (int tc = 0; tc < T; ++tc) {
+                    const int mc = ((c - tc + c0) % wc + wc) % wc;
+                    if (mc & 1) continue;
+                    const int i = mr / 2, j = mc / 2;
+                    for (int b = 0; b < 4; ++b)
+                        acc = FMA(v2[(b * T + tr) * T + tc], src[(size_t)(i + (b >> 1) * h) * W + j + (b & 1) * w], acc);
+                }
+            }
+            dst[(size_t)r * W + c] = acc;
+        }
+}
+
+/* The four T x T tap products of a filter pair: [0] lo x lo, [1] lo (rows) x hi (columns), [2] hi x lo, [3] hi x hi. */
+static void SUF(tap_products)(const REAL *lo, const REAL *hi, int T, REAL *out)
+{
+    for (int b = 0; b < 4; ++b)
+        for (int tr = 0; tr < T; ++tr)
+            for (int tc = 0; tc < T; ++tc)
+                out[(b * T + tr) * T + tc] = ((b >> 1) ? hi[tr] : lo[tr]) * ((b & 1) ? hi[tc] : lo[tc]);
+}
+
+/* Multi-level transform of every plane with a given filter pair (taps T <= 16, even); dir = 0 forward (decomposition
+ * filters), 1 inverse (reconstruction filters).  Returns 0, -1 on a bad shape. */
+int SUF(orc_dwt)(const REAL *in, int N, int C, int H, int W, int levels, const REAL *lo, const REAL *hi, int T, int dir, REAL *out)
+{
+    if (levels < 1 || T < 2 || T > 16 || (T & 1) || H <= 0 || W <= 0 || (H % (1 << levels)) || (W % (1 << levels))) return -1;
+    const long planes = (long)N * C;
+    const size_t P = (size_t)H * W;
+    REAL w2[4 * 16 * 16];
+    SUF(tap_products)(lo, hi, T, w2);
+    int bad = 0;
+#pragma omp parallel
+    {
+        REAL *scratch = (REAL *)malloc(sizeof(REAL) * P);
+        if (!scratch) {
+#pragma omp atomic write
+            bad = 1;
+        }
+#pragma omp for schedule(static)
+        for (long p = 0; p < planes; ++p) {
+            if (!scratch) continue;
+            REAL *o = out + (size_t)p * P;
+            memcpy(o, in + (size_t)p * P, sizeof(REAL) * P);
+            for (int step = 0; step < levels; ++step) {
+                const int l = dir ? levels - step : step + 1;
+                const int hc = H >> (l - 1), wc = W >> (l - 1);
+                for (int r = 0; r < hc; ++r) memcpy(scratch + (size_t)r * W, o + (size_t)r * W, sizeof(REAL) * (size_t)wc);
+                if (dir) SUF(dwt_level_inv)(scratch, o, W, hc, wc, w2, T);
+                else SUF(dwt_level_fwd)(scratch, o, W, hc, wc, w2, T);
+            }
+        }
+        free(scratch);
+    }
+    return bad ? -2 : 0;
+}
+
 /*
  * Re-read one transformed plane (quadrant layout) as the concatenated vector of Eq. 6:
  * [y1^L, y2^L, y3^L, y4^L, y2^(L-1), y3^(L-1), y4^(L-1), ..., y2^1, y3^1, y4^1],
