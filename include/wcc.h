@@ -219,6 +219,35 @@ wcc_status wcc_forward_ex(const void* x, const float* Wt, int N, int Cin, int Co
                           void* ws, size_t ws_bytes, void* stream, const wcc_options* opt, const wcc_taps* taps);
 
 /*
+ * Other wavelets than Haar (App. F compares db2, db3, coif1, bior1.3, bior2.2, sym4 under the same layer): a generic
+ * two-channel filter bank.  Filters are HOST arrays of `taps` floats (taps even, 2..8; shorter filters are zero padded
+ * by the caller), in this indexing: one 2-D level on the low-pass corner (hc x wc) is the stride-2 cross-correlation
+ *     band[i][j] = sum_{tr, tc} f_row[tr] * f_col[tc] * x[(2i + tr - c0) mod hc][(2j + tc - c0) mod wc],  c0 = taps/2 - 1
+ * with periodic extension (the transformed map keeps the size of the input; the paper does not name the extension),
+ * bands placed like Haar's: (lo, lo) top-left, (lo along the height, hi along the width) top-right, (hi, lo)
+ * bottom-left, (hi, hi) bottom-right.  The inverse is the adjoint structure with the reconstruction filters (equal to
+ * the decomposition filters for an orthogonal wavelet).  fp32, one fused multiply-add per tap in row-major tap order.
+ * [1, 1]/sqrt 2 and [1, -1]/sqrt 2 give Eq. 3 up to rounding.  Plain kernels: this is the ablation, not the hot path.
+ *   wcc_dwt_fwd        x [N][C][H][Wd] of dt -> coef fp32 (quadrant layout), nrm2 fp32 [N][P] or NULL;
+ *                      ws: at least N*C*H*Wd*4 bytes
+ *   wcc_dwt_inv        coef -> x_out of dt; ws: at least 2 * align256(N*C*H*Wd*4) bytes
+ *   wcc_forward_wavelet  the layer of Alg. 1 stage by stage with these transforms (selection, quantization and the
+ *                      tensor-core contraction as in wcc_forward_staged); taps may be NULL (coef, nrm2, idx, Xq, acc are
+ *                      served); ws: at least wcc_wavelet_workspace_bytes(...) bytes, 256-byte aligned
+ */
+wcc_status wcc_dwt_fwd(const void* x, int N, int C, int H, int Wd, int levels, wcc_dtype dt,
+                       const float* dec_lo, const float* dec_hi, int taps, float* coef, float* nrm2,
+                       void* ws, size_t ws_bytes, void* stream);
+wcc_status wcc_dwt_inv(const float* coef, int N, int C, int H, int Wd, int levels, wcc_dtype dt,
+                       const float* rec_lo, const float* rec_hi, int taps, void* x_out,
+                       void* ws, size_t ws_bytes, void* stream);
+size_t wcc_wavelet_workspace_bytes(int N, int Cin, int Cout, int H, int Wd, int levels, int k, int bits, wcc_dtype dt);
+wcc_status wcc_forward_wavelet(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int Wd,
+                               int levels, int k, int bits, const float* dec_lo, const float* dec_hi,
+                               const float* rec_lo, const float* rec_hi, int taps, void* y, wcc_dtype dt,
+                               void* ws, size_t ws_bytes, void* stream, const wcc_taps* tp_out);
+
+/*
  * Depthwise 3x3 convolution fused with the forward transform (App. H, "a kernel for a fused depthwise convolution and
  * Haar transform": both are separable per channel, so the convolution's output never goes to memory).
  *   u    in : [N][C][H][Wd] of dt           Wdw in: fp32 [C][3][3], stride 1, zero padding 1, no bias, cross-correlation

@@ -6,6 +6,7 @@
 #include "contract.cuh"
 #include "fused.cuh"
 #include "fused_tiles.cuh"
+#include "wavelet.cuh"
 
 namespace wcc {
 
@@ -444,6 +445,31 @@ static PaddedWs carve_padded_ws(void* ws, int N, int Cin, int Cout, int H, int W
     return p;
 }
 
+// ---- other wavelets -----------------------------------------------------------------------------------
+static wcc_status check_filters(const float* lo, const float* hi, int taps)
+{
+    if (!lo || !hi) return WCC_ERR_NULL;
+    if (taps < 2 || taps > wv::MAX_TAPS || (taps & 1)) return WCC_ERR_SHAPE;
+    return WCC_OK;
+}
+
+struct WaveletWs { FwdWs f; float* scratch_in; float* ywt; float* scratch_out; size_t total; };
+
+static WaveletWs carve_wavelet_ws(void* ws, int N, int Cin, int Cout, int H, int W, int k, int bits)
+{
+    WaveletWs w = {};
+    w.f = carve_forward_ws(ws, N, Cin, Cout, H, W, k, bits);
+    const size_t P = (size_t)H * W;
+    char* base = static_cast<char*>(ws);
+    size_t off = w.f.total;
+    auto take = [&](size_t bytes) { char* p = base ? base + off : nullptr; off += align_up(bytes, 256); return p; };
+    w.scratch_in = reinterpret_cast<float*>(take((size_t)N * Cin * P * 4));
+    w.ywt = reinterpret_cast<float*>(take((size_t)N * Cout * P * 4));
+    w.scratch_out = reinterpret_cast<float*>(take((size_t)N * Cout * P * 4));
+    w.total = off;
+    return w;
+}
+
 // ---- inverted residual block -------------------------------------------------------------------------
 struct BlockWs { void* u; void* layer_ws; size_t layer_ws_bytes; size_t total; };
 
@@ -632,6 +658,106 @@ wcc_status wcc_block_forward(const void* x, const float* W1, const float* Wdw, c
     wcc_options o = {};
     o.residual = x;
     return staged_impl(b.u, W3, N, E, C, H, Wd, levels, k, bits, y, dt, b.layer_ws, b.layer_ws_bytes, st, nullptr, &o, Wdw);
+}
+
+wcc_status wcc_dwt_fwd(const void* x, int N, int C, int H, int Wd, int levels, wcc_dtype dt,
+                       const float* dec_lo, const float* dec_hi, int taps, float* coef, float* nrm2,
+                       void* ws, size_t ws_bytes, void* stream)
+{
+    if (!x || !coef || !ws) return WCC_ERR_NULL;
+    wcc_status s = check_plane_args(N, C, H, Wd, levels, dt);
+    if (s != WCC_OK) return s;
+    if ((s = check_filters(dec_lo, dec_hi, taps)) != WCC_OK) return s;
+    if (!aligned16(x) || !aligned16(coef) || !aligned16(nrm2) || !aligned16(ws)) return WCC_ERR_ALIGN;
+    const size_t need = (size_t)N * C * H * Wd * 4;
+    if (ws_bytes < need) return WCC_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const wv::TapProducts tp = wv::tap_products(dec_lo, dec_hi, taps);
+    s = launch_dwt_fwd(x, (long long)N * C, H, Wd, levels, dt, tp, coef, static_cast<float*>(ws), st);
+    if (s != WCC_OK) return s;
+    if (nrm2) {
+        const long long P = (long long)H * Wd;
+        wv::norms_of_coef_kernel<<<(unsigned)((N * P + 255) / 256), 256, 0, st>>>(coef, N, C, P, nrm2, nullptr);
+        WCC_LAUNCH_CHECK();
+    }
+    return WCC_OK;
+}
+
+wcc_status wcc_dwt_inv(const float* coef, int N, int C, int H, int Wd, int levels, wcc_dtype dt,
+                       const float* rec_lo, const float* rec_hi, int taps, void* x_out,
+                       void* ws, size_t ws_bytes, void* stream)
+{
+    if (!coef || !x_out || !ws) return WCC_ERR_NULL;
+    wcc_status s = check_plane_args(N, C, H, Wd, levels, dt);
+    if (s != WCC_OK) return s;
+    if ((s = check_filters(rec_lo, rec_hi, taps)) != WCC_OK) return s;
+    if (!aligned16(coef) || !aligned16(x_out) || (reinterpret_cast<uintptr_t>(ws) & 255u)) return WCC_ERR_ALIGN;
+    const size_t plane_bytes = align_up((size_t)N * C * H * Wd * 4, 256);
+    if (ws_bytes < 2 * plane_bytes) return WCC_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    float* work = static_cast<float*>(ws);
+    float* scratch = reinterpret_cast<float*>(static_cast<char*>(ws) + plane_bytes);
+    WCC_CUDA_TRY(cudaMemcpyAsync(work, coef, (size_t)N * C * H * Wd * 4, cudaMemcpyDeviceToDevice, st));
+    const wv::TapProducts tp = wv::tap_products(rec_lo, rec_hi, taps);
+    return launch_dwt_inv(work, (long long)N * C, H, Wd, levels, dt, tp, x_out, scratch, st);
+}
+
+size_t wcc_wavelet_workspace_bytes(int N, int Cin, int Cout, int H, int Wd, int levels, int k, int bits, wcc_dtype dt)
+{
+    if (check_forward_args(N, Cin, Cout, H, Wd, levels, k, bits, dt) != WCC_OK || !staged_fits(Cin, Cout, bits)) return 0;
+    return carve_wavelet_ws(nullptr, N, Cin, Cout, H, Wd, k, bits).total;
+}
+
+wcc_status wcc_forward_wavelet(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int Wd,
+                               int levels, int k, int bits, const float* dec_lo, const float* dec_hi,
+                               const float* rec_lo, const float* rec_hi, int taps, void* y, wcc_dtype dt,
+                               void* ws, size_t ws_bytes, void* stream, const wcc_taps* tp_out)
+{
+    if (!x || !Wt || !y || !ws) return WCC_ERR_NULL;
+    wcc_status s = check_forward_args(N, Cin, Cout, H, Wd, levels, k, bits, dt);
+    if (s != WCC_OK) return s;
+    if ((s = check_filters(dec_lo, dec_hi, taps)) != WCC_OK) return s;
+    if ((s = check_filters(rec_lo, rec_hi, taps)) != WCC_OK) return s;
+    if (!aligned16(x) || !aligned16(Wt) || !aligned16(y) || (reinterpret_cast<uintptr_t>(ws) & 255u)) return WCC_ERR_ALIGN;
+    if (!staged_fits(Cin, Cout, bits)) return WCC_ERR_SHAPE;
+    const WaveletWs w = carve_wavelet_ws(ws, N, Cin, Cout, H, Wd, k, bits);
+    if (ws_bytes < w.total) return WCC_ERR_WORKSPACE;
+    const FwdWs& f = w.f;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const long long P = (long long)H * Wd;
+    const int M = N * k;
+    // A: the transform with the given decomposition filters, then norms and per-position maxima
+    s = launch_dwt_fwd(x, (long long)N * Cin, H, Wd, levels, dt, wv::tap_products(dec_lo, dec_hi, taps), f.coef, w.scratch_in, st);
+    if (s != WCC_OK) return s;
+    wv::norms_of_coef_kernel<<<(unsigned)((N * P + 255) / 256), 256, 0, st>>>(f.coef, N, Cin, P, f.nrm2, f.amaxpos);
+    WCC_LAUNCH_CHECK();
+    // B, C: as for Haar
+    s = launch_select(f.nrm2, N, (int)P, k, f.idx, nullptr, f.rank, f.amaxpos, true, f.sel, f.sel_bytes, st);
+    if (s != WCC_OK) return s;
+    if ((s = launch_weight_prep(Wt, Cout, Cin, f.kpad, bits, f.Wq, f.scale_w, st)) != WCC_OK) return s;
+    if ((s = launch_gather_quant(f.coef, f.idx, f.amax_kept, N, Cin, (int)P, k, f.kpad, bits, f.Xq, st)) != WCC_OK) return s;
+    if ((s = launch_contract(f.Xq, f.Wq, M, Cout, f.kpad, bits, f.acc, f.ldc, st)) != WCC_OK) return s;
+    // D: dequantize into the zero map; E: the synthesis with the reconstruction filters
+    WCC_CUDA_TRY(cudaMemsetAsync(w.ywt, 0, (size_t)N * Cout * P * 4, st));
+    const long long items = (long long)M * Cout;
+    const float qmax = (bits >= 2) ? (float)((1 << (bits - 1)) - 1) : 1.0f;
+    if (bits == 0)
+        wv::scatter_coef_kernel<true><<<(unsigned)((items + 255) / 256), 256, 0, st>>>(f.acc, f.ldc, f.idx, f.amax_kept, qmax, f.scale_w, N, Cout, P, k, w.ywt);
+    else
+        wv::scatter_coef_kernel<false><<<(unsigned)((items + 255) / 256), 256, 0, st>>>(f.acc, f.ldc, f.idx, f.amax_kept, qmax, f.scale_w, N, Cout, P, k, w.ywt);
+    WCC_LAUNCH_CHECK();
+    s = launch_dwt_inv(w.ywt, (long long)N * Cout, H, Wd, levels, dt, wv::tap_products(rec_lo, rec_hi, taps), y, w.scratch_out, st);
+    if (s != WCC_OK) return s;
+    if (tp_out) {
+        const cudaMemcpyKind dd = cudaMemcpyDeviceToDevice;
+        if (tp_out->coef) WCC_CUDA_TRY(cudaMemcpyAsync(tp_out->coef, f.coef, (size_t)N * Cin * P * 4, dd, st));
+        if (tp_out->nrm2) WCC_CUDA_TRY(cudaMemcpyAsync(tp_out->nrm2, f.nrm2, (size_t)N * P * 4, dd, st));
+        if (tp_out->idx) WCC_CUDA_TRY(cudaMemcpyAsync(tp_out->idx, f.idx, (size_t)M * 4, dd, st));
+        if (bits >= 2 && tp_out->Xq) WCC_CUDA_TRY(cudaMemcpyAsync(tp_out->Xq, f.Xq, (size_t)M * f.kpad, dd, st));
+        if (tp_out->acc)
+            WCC_CUDA_TRY(cudaMemcpy2DAsync(tp_out->acc, (size_t)Cout * 4, f.acc, (size_t)f.ldc * 4, (size_t)Cout * 4, M, dd, st));
+    }
+    return WCC_OK;
 }
 
 size_t wcc_select_bitmap_workspace_bytes(int N, int P, int k)

@@ -24,7 +24,7 @@ EXPORTS = ("wcc_staged_workspace_bytes", "wcc_forward_staged", "wcc_workspace_by
            "wcc_debug_set_wait_limit", "wcc_debug_wait_selftest", "wcc_forward_ex", "wcc_chain_workspace_bytes",
            "wcc_chain_forward", "wcc_select_bitmap_workspace_bytes", "wcc_select_topk_bitmap",
            "wcc_padded_workspace_bytes", "wcc_forward_padded", "wcc_dwconv_haar_fwd", "wcc_block_workspace_bytes",
-           "wcc_block_forward")
+           "wcc_block_forward", "wcc_dwt_fwd", "wcc_dwt_inv", "wcc_wavelet_workspace_bytes", "wcc_forward_wavelet")
 STATIC_SCRATCH_BYTES = 512 * 1024
 STAGES = ("haar_fwd_norms", "select_topk", "weight_quant", "gather_quant", "contract", "scatter_inv")   # wcc_forward_staged
 FUSED_STAGES = ("clear", "haar_norms", "select_topk", "fused_pass2")                                      # wcc_forward
@@ -100,6 +100,15 @@ def lib() -> C.CDLL:
         L.wcc_block_workspace_bytes.argtypes = [i] * 9
         L.wcc_block_forward.restype = i
         L.wcc_block_forward.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, i, i, vp, i, vp, sz, vp]
+        fp = C.POINTER(C.c_float)
+        L.wcc_dwt_fwd.restype = i
+        L.wcc_dwt_fwd.argtypes = [vp, i, i, i, i, i, i, fp, fp, i, vp, vp, vp, sz, vp]
+        L.wcc_dwt_inv.restype = i
+        L.wcc_dwt_inv.argtypes = [vp, i, i, i, i, i, i, fp, fp, i, vp, vp, sz, vp]
+        L.wcc_wavelet_workspace_bytes.restype = sz
+        L.wcc_wavelet_workspace_bytes.argtypes = [i] * 9
+        L.wcc_forward_wavelet.restype = i
+        L.wcc_forward_wavelet.argtypes = [vp, vp, i, i, i, i, i, i, i, i, fp, fp, fp, fp, i, vp, i, vp, sz, vp, C.POINTER(Taps)]
         L.wcc_chain_workspace_bytes.restype = sz
         L.wcc_chain_workspace_bytes.argtypes = [C.POINTER(ChainLayer), i, i, i, i, i, i, i, i]
         L.wcc_chain_forward.restype = i
@@ -179,6 +188,66 @@ def dwconv_haar_fwd(u: torch.Tensor, Wdw: torch.Tensor, levels: int):
     _check(lib().wcc_dwconv_haar_fwd(u.data_ptr(), Wdw.data_ptr(), N, Cc, H, W, levels, _dt(u), coef.data_ptr(),
                                      nrm2.data_ptr(), _stream()), "wcc_dwconv_haar_fwd")
     return coef, nrm2
+
+
+def _taps(f):
+    import numpy as np
+    a = np.ascontiguousarray(f, dtype=np.float32)
+    return a, a.ctypes.data_as(C.POINTER(C.c_float))
+
+
+def dwt_fwd(x: torch.Tensor, levels: int, dec_lo, dec_hi):
+    """Generic wavelet transform (host filter arrays, see wcc.h) -> (coef fp32, nrm2 fp32 [N][P])."""
+    _dev(x, "x")
+    N, Cc, H, W = x.shape
+    lo, plo = _taps(dec_lo)
+    hi, phi = _taps(dec_hi)
+    coef = torch.empty((N, Cc, H, W), dtype=torch.float32, device=x.device)
+    nrm2 = torch.empty((N, H * W), dtype=torch.float32, device=x.device)
+    ws = torch.empty((N * Cc * H * W * 4,), dtype=torch.uint8, device=x.device)
+    _check(lib().wcc_dwt_fwd(x.data_ptr(), N, Cc, H, W, levels, _dt(x), plo, phi, lo.size, coef.data_ptr(), nrm2.data_ptr(),
+                             ws.data_ptr(), ws.numel(), _stream()), "wcc_dwt_fwd")
+    return coef, nrm2
+
+
+def dwt_inv(coef: torch.Tensor, levels: int, rec_lo, rec_hi, dtype: torch.dtype = torch.float32) -> torch.Tensor:
+    _dev(coef, "coef")
+    N, Cc, H, W = coef.shape
+    lo, plo = _taps(rec_lo)
+    hi, phi = _taps(rec_hi)
+    out = torch.empty((N, Cc, H, W), dtype=dtype, device=coef.device)
+    ws = torch.empty((2 * (N * Cc * H * W * 4 + 256),), dtype=torch.uint8, device=coef.device)
+    _check(lib().wcc_dwt_inv(coef.data_ptr(), N, Cc, H, W, levels, _dt(out), plo, phi, lo.size, out.data_ptr(),
+                             ws.data_ptr(), ws.numel(), _stream()), "wcc_dwt_inv")
+    return out
+
+
+def forward_wavelet(x: torch.Tensor, Wt: torch.Tensor, levels: int, k: int, bits: int, bank, taps: bool = False):
+    """The layer with another wavelet: ``bank`` = (dec_lo, dec_hi, rec_lo, rec_hi) host arrays of equal even length."""
+    _dev(x, "x")
+    _dev(Wt, "Wt")
+    N, Cin, H, W = x.shape
+    Cout = Wt.shape[0]
+    f = [_taps(b) for b in bank]
+    nbytes = int(lib().wcc_wavelet_workspace_bytes(N, Cin, Cout, H, W, levels, k, bits, _dt(x)))
+    if nbytes == 0:
+        raise WccError(2, "wcc_wavelet_workspace_bytes")
+    ws = torch.empty((nbytes,), dtype=torch.uint8, device=x.device)
+    y = torch.empty((N, Cout, H, W), dtype=x.dtype, device=x.device)
+    t, s = {}, None
+    if taps:
+        P, M, kp = H * W, N * k, kpad(Cin, bits)
+        t = dict(coef=torch.empty((N, Cin, P), dtype=torch.float32, device=x.device),
+                 nrm2=torch.empty((N, P), dtype=torch.float32, device=x.device),
+                 idx=torch.empty((N, k), dtype=torch.int32, device=x.device),
+                 acc=torch.empty((M, Cout), dtype=torch.int32, device=x.device))
+        if bits >= 2:
+            t["Xq"] = torch.empty((M, kp), dtype=torch.int8, device=x.device)
+        s = Taps(**{name: _ptr(t.get(name)) for name, _ in Taps._fields_})
+    _check(lib().wcc_forward_wavelet(x.data_ptr(), Wt.data_ptr(), N, Cin, Cout, H, W, levels, k, bits, f[0][1], f[1][1], f[2][1],
+                                     f[3][1], f[0][0].size, y.data_ptr(), _dt(x), ws.data_ptr(), nbytes, _stream(),
+                                     C.byref(s) if s is not None else None), "wcc_forward_wavelet")
+    return (y, t) if taps else y
 
 
 class Block:
