@@ -420,6 +420,30 @@ def run_ours(args):
         dist.barrier()
     wcc.lib()
 
+    if args.workload == "C5chain":                      # profiling aid: the six-layer chain alone (three levels, keep 1/4)
+        flush = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device=dev)
+        peak, _ = _peaks()
+        N, H, W = (args.batch or 2), 256, 512
+        chans = [32, 192, 32, 192, 32, 192, 32]
+        first = inputs.custom("C5", 0, N, 32, 192, H, W, "bf16", 3, 0.25, 8, n_sin=16, fmax=8.0)
+        x = torch.from_numpy(first.x.view(np.int16)).view(torch.bfloat16).to(dev)
+        Ws = [torch.from_numpy(inputs.weights(100 + i, chans[i + 1], chans[i])).to(dev) for i in range(6)]
+        ch = wcc.Chain(x, Ws, 3, first.k, 8)
+        y = torch.empty((N, 32, H, W), dtype=torch.bfloat16, device=dev)
+        for _ in range(max(3, args.warmup)):
+            flush.fill_(1)
+            ch(x, y)
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        for a, b in ev:
+            flush.fill_(1)
+            a.record()
+            ch(x, y)
+            b.record()
+        torch.cuda.synchronize()
+        assert wcc.last_status() == 0
+        t = sum(a.elapsed_time(b) for a, b in ev) / len(ev)
+        print(json.dumps({"workload": "C5chain N=%d L=3 keep=0.25 (eager launches)" % N, "ms_per_chain": t, "lean": True}))
+        return 0
     over = {"N": args.batch} if args.batch else {}
     w = inputs.make(args.workload, seed=rank_seed(rank), **over)
     case = Case(wcc, torch, np, w, dev, staged=args.staged, graph=not args.no_graph)
