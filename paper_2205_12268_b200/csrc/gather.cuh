@@ -44,13 +44,14 @@ weight_prep_kernel(const float* __restrict__ Wt, int Cout, int Cin, int kpad, in
     if (o < Cout) weight_prep_row(Wt, o, Cin, kpad, bits, Wq, scale_w);
 }
 
-// One thread per kept position (row r = n*k + j of the compressed matrix): reads coef[n][c][idx[n][j]] for every
-// channel and writes one K-major row.  Consecutive rows are consecutive kept positions, so a warp's reads of one
-// channel are contiguous wherever the kept set is dense (the low-pass corner) and sector-sparse elsewhere.
+// One thread per kept position (row r = n*k + j of the compressed matrix) and chunk of `cpc` channels (blockIdx.y; a
+// multiple of 64): reads coef[n][c][idx[n][j]] for its channels and writes that part of one K-major row.  Consecutive
+// rows are consecutive kept positions, so a warp's reads of one channel are contiguous wherever the kept set is dense
+// (the low-pass corner) and sector-sparse elsewhere.
 template <bool QUANT>
 __global__ void __launch_bounds__(128)
 gather_quant_kernel(const float* __restrict__ coef, const int32_t* __restrict__ idx, const float* __restrict__ amax_kept,
-                    int M, int Cin, int P, int k, int kpad, float qmax, void* __restrict__ Xq)
+                    int M, int Cin, int P, int k, int kpad, int cpc, float qmax, void* __restrict__ Xq)
 {
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= M) return;
@@ -64,7 +65,8 @@ gather_quant_kernel(const float* __restrict__ coef, const int32_t* __restrict__ 
     }
     constexpr int CH = QUANT ? 16 : 8;      // channels per 16-byte store
     uint4* dst = reinterpret_cast<uint4*>(static_cast<char*>(Xq) + (size_t)r * kpad * (QUANT ? 1 : 2));
-    for (int c0 = 0; c0 < kpad; c0 += CH) {
+    const int c_lo = (int)blockIdx.y * cpc, c_hi = min(kpad, c_lo + cpc);
+    for (int c0 = c_lo; c0 < c_hi; c0 += CH) {
         float v[CH];
 #pragma unroll
         for (int i = 0; i < CH; ++i) v[i] = (c0 + i < Cin) ? src[(size_t)(c0 + i) * P] : 0.0f;
@@ -99,10 +101,13 @@ wcc_status launch_gather_quant(const float* coef, const int32_t* idx, const floa
 {
     const int M = N * k;
     const float qmax = (bits >= 2) ? (float)((1 << (bits - 1)) - 1) : 1.0f;
+    // rows alone fill the GPU from about 150 K kept positions on; below that the channels are split as well
+    const int cpc = (M >= 148 * 1024) ? kpad : 64;
+    const dim3 grid(ceil_div(M, 128), ceil_div(kpad, cpc));
     if (bits >= 2)
-        gather_quant_kernel<true><<<ceil_div(M, 128), 128, 0, st>>>(coef, idx, amax_kept, M, Cin, P, k, kpad, qmax, Xq);
+        gather_quant_kernel<true><<<grid, 128, 0, st>>>(coef, idx, amax_kept, M, Cin, P, k, kpad, cpc, qmax, Xq);
     else
-        gather_quant_kernel<false><<<ceil_div(M, 128), 128, 0, st>>>(coef, idx, amax_kept, M, Cin, P, k, kpad, qmax, Xq);
+        gather_quant_kernel<false><<<grid, 128, 0, st>>>(coef, idx, amax_kept, M, Cin, P, k, kpad, cpc, qmax, Xq);
     WCC_LAUNCH_CHECK();
     return WCC_OK;
 }

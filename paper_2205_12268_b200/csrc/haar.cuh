@@ -560,11 +560,13 @@ __device__ __forceinline__ void tile_coords(int warp, int tiles_x, int tiles_y, 
 }
 
 // ---- forward: Haar + norms ---------------------------------------------------------------------
-// One warp per (image, tile); the warp walks the channels in ascending order, D channels of loads in
-// flight at a time.  Writes coef (optional), nrm2 (optional) and amaxpos = max_c |coef| (optional).
+// One warp per (image, tile, chunk of cpc channels; blockIdx.y = chunk); the warp walks its channels in ascending
+// order, D channels of loads in flight at a time.  Writes coef (optional) and, when one chunk holds all channels,
+// nrm2 (optional) and amaxpos = max_c |coef| (optional): the norm is one chain of fused multiply-adds over all
+// channels, so with several chunks it is taken from the stored coefficients afterwards (coef_norms_kernel).
 template <typename T, int L, bool VEC, int D>
 __global__ void __launch_bounds__(128)
-haar_fwd_kernel(const T* __restrict__ x, int N, int C, int H, int W,
+haar_fwd_kernel(const T* __restrict__ x, int N, int C, int H, int W, int cpc,
                 float* __restrict__ coef, float* __restrict__ nrm2, float* __restrict__ amaxpos)
 {
     using TT = HaarTile<L>;
@@ -578,20 +580,22 @@ haar_fwd_kernel(const T* __restrict__ x, int N, int C, int H, int W,
     const size_t P = (size_t)H * W;
     const T* xin = x + (size_t)n * C * P;
     float* cout = coef ? coef + (size_t)n * C * P : nullptr;
+    const int c_lo = (int)blockIdx.y * cpc, c_hi = min(C, c_lo + cpc);
+    if (gridDim.y > 1) { nrm2 = nullptr; amaxpos = nullptr; }
 
     float nacc[8], amax[8];
 #pragma unroll
     for (int s = 0; s < 8; ++s) { nacc[s] = 0.0f; amax[s] = 0.0f; }
 
-    for (int c0 = 0; c0 < C; c0 += D) {
+    for (int c0 = c_lo; c0 < c_hi; c0 += D) {
         RawPatch raw[D];
 #pragma unroll
         for (int d = 0; d < D; ++d) {
-            if (c0 + d < C) load_patch<T, VEC>(xin + (size_t)(c0 + d) * P, W, lp, raw[d]);
+            if (c0 + d < c_hi) load_patch<T, VEC>(xin + (size_t)(c0 + d) * P, W, lp, raw[d]);
         }
 #pragma unroll
         for (int d = 0; d < D; ++d) {
-            if (c0 + d < C) {
+            if (c0 + d < c_hi) {
                 float p[2][4], o[8];
                 unpack_patch<T>(raw[d], p);
                 haar_fwd_lane<L>(p, o, lane);
@@ -614,10 +618,91 @@ haar_fwd_kernel(const T* __restrict__ x, int N, int C, int H, int W,
 // separable per channel, so the convolution's output never goes to memory: every lane computes the convolution at the
 // eight pixels of its patch (from a 4 x 6 neighbourhood of the input, zeros outside the map) and transforms them right
 // away.  Per output pixel: one fused multiply-add per tap, row-major tap order, starting from +0 (taps outside the map
-// contribute nothing).  Same work decomposition and outputs as haar_fwd_kernel; w is fp32 [C][3][3].
-template <typename T, int L, bool VEC>
+// contribute nothing).  Same work decomposition (channel chunks included) and outputs as haar_fwd_kernel; w is fp32
+// [C][3][3].
+
+// One channel's input of the convolution as loaded: rows r0-1 .. r0+2, columns c0-1 .. c0+4 of the lane's patch (zeros
+// outside the map), and the channel's nine taps.  With W % 4 == 0 the four middle columns are one aligned vector; bf16
+// rows then stay packed (two words of middle columns, one word holding the left and the right neighbour).
+template <typename T, bool VEC>
+struct DwRaw {
+    static constexpr bool PACKED = VEC && sizeof(T) == 2;
+    static constexpr int RW = PACKED ? 3 : 6;
+    uint32_t v[4][RW];
+    float k[9];
+};
+
+template <typename T, bool VEC>
+__device__ __forceinline__ void dwconv_load(const T* __restrict__ plane, const float* __restrict__ w9, const LanePos& lp,
+                                            int H, int W, DwRaw<T, VEC>& r)
+{
+#pragma unroll
+    for (int i = 0; i < 9; ++i) r.k[i] = __ldg(w9 + i);
+    auto load1 = [&](int rr, int cc) -> uint32_t {         // one element as fp32 bits (bf16: the upper half)
+        if (sizeof(T) == 4) return __ldg(reinterpret_cast<const uint32_t*>(plane) + (size_t)rr * W + cc);
+        return (uint32_t)__ldg(reinterpret_cast<const unsigned short*>(plane) + (size_t)rr * W + cc) << 16;
+    };
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+        const int rr = lp.r0 + a - 1;
+        const bool row_in = rr >= 0 && rr < H;
+        if constexpr (VEC) {
+            const uint32_t left = (row_in && lp.c0 > 0 && lp.c0 - 1 < W) ? load1(rr, lp.c0 - 1) : 0u;
+            const uint32_t right = (row_in && lp.c0 + 4 < W) ? load1(rr, lp.c0 + 4) : 0u;
+            if constexpr (sizeof(T) == 4) {
+                uint4 m = make_uint4(0u, 0u, 0u, 0u);
+                if (row_in && lp.ok0) m = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint32_t*>(plane) + (size_t)rr * W + lp.c0));
+                r.v[a][0] = left; r.v[a][1] = m.x; r.v[a][2] = m.y; r.v[a][3] = m.z; r.v[a][4] = m.w; r.v[a][5] = right;
+            } else {
+                uint2 m = make_uint2(0u, 0u);
+                if (row_in && lp.ok0) m = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const unsigned short*>(plane) + (size_t)rr * W + lp.c0));
+                r.v[a][0] = m.x; r.v[a][1] = m.y; r.v[a][2] = (left >> 16) | right;
+            }
+        } else {
+#pragma unroll
+            for (int b = 0; b < 6; ++b) {
+                const int cc = lp.c0 + b - 1;
+                r.v[a][b] = (row_in && cc >= 0 && cc < W) ? load1(rr, cc) : 0u;
+            }
+        }
+    }
+}
+
+// The convolution at the eight pixels of the lane's patch: one fused multiply-add per tap, row-major tap order, from +0.
+template <typename T, bool VEC>
+__device__ __forceinline__ void dwconv_compute(const DwRaw<T, VEC>& r, float (&p)[2][4])
+{
+    float in[4][6];
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+        if constexpr (DwRaw<T, VEC>::PACKED) {
+            in[a][0] = bf16lo(r.v[a][2]);
+            in[a][1] = bf16lo(r.v[a][0]); in[a][2] = bf16hi(r.v[a][0]);
+            in[a][3] = bf16lo(r.v[a][1]); in[a][4] = bf16hi(r.v[a][1]);
+            in[a][5] = bf16hi(r.v[a][2]);
+        } else {
+#pragma unroll
+            for (int b = 0; b < 6; ++b) in[a][b] = __uint_as_float(r.v[a][b]);
+        }
+    }
+#pragma unroll
+    for (int a = 0; a < 2; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            float acc = 0.0f;
+#pragma unroll
+            for (int i = 0; i < 3; ++i)
+#pragma unroll
+                for (int j = 0; j < 3; ++j) acc = __fmaf_rn(r.k[i * 3 + j], in[a + i][b + j], acc);
+            p[a][b] = acc;
+        }
+}
+
+// NORMS = false: a chunk of the channels (blockIdx.y), coefficients only.  The next channel's input is loaded while
+// the current one is convolved and transformed.
+template <typename T, int L, bool VEC, bool NORMS>
 __global__ void __launch_bounds__(128)
-dwconv_haar_fwd_kernel(const T* __restrict__ u, const float* __restrict__ w, int N, int C, int H, int W,
+dwconv_haar_fwd_kernel(const T* __restrict__ u, const float* __restrict__ w, int N, int C, int H, int W, int cpc,
                        float* __restrict__ coef, float* __restrict__ nrm2, float* __restrict__ amaxpos)
 {
     using TT = HaarTile<L>;
@@ -631,50 +716,84 @@ dwconv_haar_fwd_kernel(const T* __restrict__ u, const float* __restrict__ w, int
     const size_t P = (size_t)H * W;
     const T* uin = u + (size_t)n * C * P;
     float* cout = coef ? coef + (size_t)n * C * P : nullptr;
+    const int c_lo = (int)blockIdx.y * cpc, c_hi = min(C, c_lo + cpc);
 
     float nacc[8], amax[8];
 #pragma unroll
     for (int s = 0; s < 8; ++s) { nacc[s] = 0.0f; amax[s] = 0.0f; }
-    for (int c = 0; c < C; ++c) {
-        const T* plane = uin + (size_t)c * P;
-        float k9[9];
-#pragma unroll
-        for (int i = 0; i < 9; ++i) k9[i] = __ldg(w + (size_t)c * 9 + i);
-        float in[4][6];                                    // rows r0-1 .. r0+2, columns c0-1 .. c0+4
-#pragma unroll
-        for (int a = 0; a < 4; ++a)
-#pragma unroll
-            for (int b = 0; b < 6; ++b) {
-                const int rr = lp.r0 + a - 1, cc = lp.c0 + b - 1;
-                float v = 0.0f;
-                if (rr >= 0 && rr < H && cc >= 0 && cc < W) {
-                    if (sizeof(T) == 4) v = __ldg(reinterpret_cast<const float*>(plane) + (size_t)rr * W + cc);
-                    else v = __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short*>(plane) + (size_t)rr * W + cc) << 16);
-                }
-                in[a][b] = v;
-            }
+    DwRaw<T, VEC> cur, nxt;
+    dwconv_load<T, VEC>(uin + (size_t)c_lo * P, w + (size_t)c_lo * 9, lp, H, W, cur);
+    nxt = cur;
+    for (int c = c_lo; c < c_hi; ++c) {
+        if (c + 1 < c_hi) dwconv_load<T, VEC>(uin + (size_t)(c + 1) * P, w + (size_t)(c + 1) * 9, lp, H, W, nxt);
         float p[2][4], o[8];
-#pragma unroll
-        for (int a = 0; a < 2; ++a)
-#pragma unroll
-            for (int b = 0; b < 4; ++b) {
-                float acc = 0.0f;
-#pragma unroll
-                for (int i = 0; i < 3; ++i)
-#pragma unroll
-                    for (int j = 0; j < 3; ++j) acc = __fmaf_rn(k9[i * 3 + j], in[a + i][b + j], acc);
-                p[a][b] = acc;
-            }
+        dwconv_compute<T, VEC>(cur, p);
         haar_fwd_lane<L>(p, o, lane);
         if (cout) store_slots<L, VEC>(cout + (size_t)c * P, lp, o);
+        if (NORMS) {
 #pragma unroll
-        for (int s = 0; s < 8; ++s) {
-            nacc[s] = __fmaf_rn(o[s], o[s], nacc[s]);
-            amax[s] = fmaxf(amax[s], fabsf(o[s]));
+            for (int s = 0; s < 8; ++s) {
+                nacc[s] = __fmaf_rn(o[s], o[s], nacc[s]);
+                amax[s] = fmaxf(amax[s], fabsf(o[s]));
+            }
+        }
+        cur = nxt;
+    }
+    if (NORMS) {
+        if (nrm2) store_slots<L, VEC>(nrm2 + (size_t)n * P, lp, nacc);
+        if (amaxpos) store_slots<L, VEC>(amaxpos + (size_t)n * P, lp, amax);
+    }
+}
+
+// Channel norms of a stored coefficient map: one thread per position builds the chain of fused multiply-adds over the
+// channels in ascending order, from +0, and max |coef|.  Thirty-two channels of loads in flight per thread.
+__global__ void __launch_bounds__(256)
+coef_norms_kernel(const float* __restrict__ coef, int N, int C, long long P, float* __restrict__ nrm2, float* __restrict__ amaxpos)
+{
+    const long long id = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (id >= (long long)N * P) return;
+    const long long n = id / P, p = id - n * P;
+    const float* src = coef + (size_t)n * C * P + p;
+    constexpr int UN = 32;
+    float acc = 0.0f, am = 0.0f;
+    int c = 0;
+    for (; c + UN <= C; c += UN) {
+        float v[UN];
+#pragma unroll
+        for (int i = 0; i < UN; ++i) v[i] = __ldcs(src + (size_t)(c + i) * P);
+#pragma unroll
+        for (int i = 0; i < UN; ++i) {
+            acc = __fmaf_rn(v[i], v[i], acc);
+            am = fmaxf(am, fabsf(v[i]));
         }
     }
-    if (nrm2) store_slots<L, VEC>(nrm2 + (size_t)n * P, lp, nacc);
-    if (amaxpos) store_slots<L, VEC>(amaxpos + (size_t)n * P, lp, amax);
+    for (; c < C; ++c) {
+        const float v = __ldcs(src + (size_t)c * P);
+        acc = __fmaf_rn(v, v, acc);
+        am = fmaxf(am, fabsf(v));
+    }
+    if (nrm2) nrm2[id] = acc;
+    if (amaxpos) amaxpos[id] = am;
+}
+
+// Channels per chunk of the forward kernels: one chunk (norms in the same pass) when the tiles alone fill the GPU or no
+// coefficient map is stored; otherwise chunks of a multiple of `unit` channels, about 32 warps for each of the 148 SMs.
+static int forward_chunk_channels(long long tile_warps, int C, int unit, bool has_coef)
+{
+    constexpr long long want = 148 * 32;
+    if (!has_coef || tile_warps >= want || C <= 2 * unit) return C;
+    const long long chunks = std::min<long long>((C + unit - 1) / unit, (want + tile_warps - 1) / tile_warps);
+    int cpc = (int)((C + chunks - 1) / chunks);
+    cpc = (cpc + unit - 1) / unit * unit;
+    return std::min(cpc, C);
+}
+
+static wcc_status launch_coef_norms(const float* coef, int N, int C, long long P, float* nrm2, float* amaxpos, cudaStream_t st)
+{
+    if (!nrm2 && !amaxpos) return WCC_OK;
+    coef_norms_kernel<<<(unsigned)(((long long)N * P + 255) / 256), 256, 0, st>>>(coef, N, C, P, nrm2, amaxpos);
+    WCC_LAUNCH_CHECK();
+    return WCC_OK;
 }
 
 // ---- per-warp asynchronous patch ring ------------------------------------------------------------
@@ -1277,8 +1396,11 @@ static wcc_status haar_fwd_dispatch(const void* x, int N, int C, int H, int W, f
     const long long warps = (long long)N * ceil_div(W, TT::TW) * (H / TT::TH);
     if (!coef && nrm2) return haar_norms_dispatch<T, L, VEC>(x, N, C, H, W, nrm2, amaxpos, NormsExtra{}, st);   // norms only
     const int blocks = (int)((warps + 3) / 4);
-    haar_fwd_kernel<T, L, VEC, D><<<blocks, 128, 0, st>>>(static_cast<const T*>(x), N, C, H, W, coef, nrm2, amaxpos);
+    const int cpc = forward_chunk_channels(warps, C, D, coef != nullptr);
+    const dim3 grid(blocks, ceil_div(C, cpc));
+    haar_fwd_kernel<T, L, VEC, D><<<grid, 128, 0, st>>>(static_cast<const T*>(x), N, C, H, W, cpc, coef, nrm2, amaxpos);
     WCC_LAUNCH_CHECK();
+    if (grid.y > 1) return launch_coef_norms(coef, N, C, (long long)H * W, nrm2, amaxpos, st);
     return WCC_OK;
 }
 
@@ -1351,8 +1473,14 @@ static wcc_status dwconv_haar_dispatch(const void* u, const float* w, int N, int
     using TT = HaarTile<L>;
     const long long warps = (long long)N * ceil_div(W, TT::TW) * (H / TT::TH);
     const int blocks = (int)((warps + 3) / 4);
-    dwconv_haar_fwd_kernel<T, L, VEC><<<blocks, 128, 0, st>>>(static_cast<const T*>(u), w, N, C, H, W, coef, nrm2, amaxpos);
+    const int cpc = forward_chunk_channels(warps, C, 8, coef != nullptr);
+    const dim3 grid(blocks, ceil_div(C, cpc));
+    if (grid.y > 1)
+        dwconv_haar_fwd_kernel<T, L, VEC, false><<<grid, 128, 0, st>>>(static_cast<const T*>(u), w, N, C, H, W, cpc, coef, nullptr, nullptr);
+    else
+        dwconv_haar_fwd_kernel<T, L, VEC, true><<<grid, 128, 0, st>>>(static_cast<const T*>(u), w, N, C, H, W, cpc, coef, nrm2, amaxpos);
     WCC_LAUNCH_CHECK();
+    if (grid.y > 1) return launch_coef_norms(coef, N, C, (long long)H * W, nrm2, amaxpos, st);
     return WCC_OK;
 }
 

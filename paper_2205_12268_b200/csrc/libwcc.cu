@@ -677,8 +677,7 @@ wcc_status wcc_dwt_fwd(const void* x, int N, int C, int H, int Wd, int levels, w
     if (s != WCC_OK) return s;
     if (nrm2) {
         const long long P = (long long)H * Wd;
-        wv::norms_of_coef_kernel<<<(unsigned)((N * P + 255) / 256), 256, 0, st>>>(coef, N, C, P, nrm2, nullptr);
-        WCC_LAUNCH_CHECK();
+        if ((s = launch_coef_norms(coef, N, C, P, nrm2, nullptr, st)) != WCC_OK) return s;
     }
     return WCC_OK;
 }
@@ -729,8 +728,7 @@ wcc_status wcc_forward_wavelet(const void* x, const float* Wt, int N, int Cin, i
     // A: the transform with the given decomposition filters, then norms and per-position maxima
     s = launch_dwt_fwd(x, (long long)N * Cin, H, Wd, levels, dt, wv::tap_products(dec_lo, dec_hi, taps), f.coef, w.scratch_in, st);
     if (s != WCC_OK) return s;
-    wv::norms_of_coef_kernel<<<(unsigned)((N * P + 255) / 256), 256, 0, st>>>(f.coef, N, Cin, P, f.nrm2, f.amaxpos);
-    WCC_LAUNCH_CHECK();
+    if ((s = launch_coef_norms(f.coef, N, Cin, P, f.nrm2, f.amaxpos, st)) != WCC_OK) return s;
     // B, C: as for Haar
     s = launch_select(f.nrm2, N, (int)P, k, f.idx, nullptr, f.rank, f.amaxpos, true, f.sel, f.sel_bytes, st);
     if (s != WCC_OK) return s;

@@ -100,24 +100,6 @@ dwt_level_inv_kernel(const float* __restrict__ src, TO* __restrict__ dst, long l
     store_from_float(dst + (size_t)pl * H * W + (size_t)r * W + c, acc);
 }
 
-// Channel norms (one fused multiply-add per channel, ascending, from +0) and per-position max |coef| of a coefficient map.
-__global__ void __launch_bounds__(256)
-norms_of_coef_kernel(const float* __restrict__ coef, int N, int C, long long P, float* __restrict__ nrm2, float* __restrict__ amaxpos)
-{
-    const long long id = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (id >= (long long)N * P) return;
-    const long long n = id / P, p = id - n * P;
-    const float* src = coef + (size_t)n * C * P + p;
-    float acc = 0.0f, am = 0.0f;
-    for (int c = 0; c < C; ++c) {
-        const float v = src[(size_t)c * P];
-        acc = __fmaf_rn(v, v, acc);
-        am = fmaxf(am, fabsf(v));
-    }
-    nrm2[id] = acc;
-    if (amaxpos) amaxpos[id] = am;
-}
-
 // Dequantize the accumulators of the kept positions into the (zeroed) wavelet-domain output map:
 // Ywt[n][o][idx[n][j]] = float(acc[n*k + j][o]) * (scale_a * scale_w[o])   (or the fp32 products when ACCF).
 template <bool ACCF>
