@@ -1307,18 +1307,19 @@ haar_inv_kernel(const float* __restrict__ coef, int planes, int H, int W, T* __r
 }
 
 // ---- fused dequantize + scatter + inverse ----------------------------------------------------
-// One warp per (image, tile, group of OCW output channels).  rank[n][p] is the row of position p in the
-// compressed matrix (or -1 when p was dropped: the zero map).  acc row r = n*k + rank holds the int32
-// accumulators (or fp32 products when ACCF) of all output channels, pitch ldc (multiple of 4).
-template <typename T, int L, bool VEC, bool ACCF, int OCW>
-__global__ void __launch_bounds__(128)
+// One warp per (image, tile, group of ocw output channels; ocw a multiple of 4).  rank[n][p] is the row of position p
+// in the compressed matrix (or -1 when p was dropped: the zero map).  acc row r = n*k + rank holds the int32
+// accumulators (or fp32 products when ACCF) of all output channels, pitch ldc (multiple of 4).  The accumulators of
+// the next four channels are gathered while the current four are transformed.
+template <typename T, int L, bool VEC, bool ACCF>
+__global__ void __launch_bounds__(128, 5)
 scatter_inv_kernel(const int32_t* __restrict__ acc, int ldc, const int32_t* __restrict__ rank,
                    const float* __restrict__ amax_kept, float qmax, const float* __restrict__ scale_w,
-                   int N, int Cout, int H, int W, int k, T* __restrict__ y, const T* __restrict__ residual, int relu)
+                   int N, int Cout, int ocw, int H, int W, int k, T* __restrict__ y, const T* __restrict__ residual, int relu)
 {
     using TT = HaarTile<L>;
     const int tiles_x = (W + TT::TW - 1) / TT::TW, tiles_y = H / TT::TH;
-    const int groups = (Cout + OCW - 1) / OCW;
+    const int groups = (Cout + ocw - 1) / ocw;
     const long long gw = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (gw >= (long long)N * tiles_x * tiles_y * groups) return;
     const int lane = threadIdx.x & 31;
@@ -1339,25 +1340,42 @@ scatter_inv_kernel(const int32_t* __restrict__ acc, int ldc, const int32_t* __re
     float scale_a = 1.0f;
     if (!ACCF) scale_a = __fdiv_rn(*amax_kept, qmax);
 
-    const int o_end = min(Cout, (g + 1) * OCW);
-    for (int o0 = g * OCW; o0 < o_end; o0 += 4) {
-        int4 v[8];
+    // Four channels at a time: dequantize straight into the pre-scaled slots of haar_inv_lanes_raw, acc * (scale * 2^-level)
+    // (the halvings of the inverse transform are exact powers of two and commute with every rounding).
+    const bool coarse6 = L == 3 && ((lane / TT::CG) & 1) == 0;         // slot 6 holds a level-3 coefficient
+    const int o_end = min(Cout, (g + 1) * ocw);
+    int4 v[8], vn[8];
 #pragma unroll
-        for (int s = 0; s < 8; ++s)
-            v[s] = rowp[s] ? *reinterpret_cast<const int4*>(rowp[s] + o0) : make_int4(0, 0, 0, 0);
+    for (int s = 0; s < 8; ++s) {
+        v[s] = rowp[s] ? __ldg(reinterpret_cast<const int4*>(rowp[s] + g * ocw)) : make_int4(0, 0, 0, 0);
+        vn[s] = v[s];
+    }
+    for (int o0 = g * ocw; o0 < o_end; o0 += 4) {
+        if (o0 + 4 < o_end) {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int o = o0 + j;
+            for (int s = 0; s < 8; ++s)
+                vn[s] = rowp[s] ? __ldg(reinterpret_cast<const int4*>(rowp[s] + o0 + 4)) : make_int4(0, 0, 0, 0);
+        }
+        float sl[4][8], p[4][2][4];
+#pragma unroll
+        for (int d = 0; d < 4; ++d) {
+            const int o = o0 + d;
+            float sc = 1.0f;
+            if (!ACCF) sc = (o < o_end) ? __fmul_rn(scale_a, scale_w[o]) : 0.0f;
+            const float s1 = __fmul_rn(sc, 0.5f), s2 = __fmul_rn(sc, 0.25f);
+            const float s6 = (L == 1) ? s1 : (coarse6 ? __fmul_rn(sc, 0.125f) : s2), s7 = (L == 1) ? s1 : s2;
+#pragma unroll
+            for (int s = 0; s < 8; ++s) {
+                const int a = (d == 0) ? v[s].x : (d == 1) ? v[s].y : (d == 2) ? v[s].z : v[s].w;
+                const float f = ACCF ? __int_as_float(a) : __int2float_rn(a);
+                sl[d][s] = __fmul_rn(f, s < 6 ? s1 : (s == 6 ? s6 : s7));
+            }
+        }
+        haar_inv_lanes_raw<L, 4>(sl, p, lane);
+#pragma unroll
+        for (int d = 0; d < 4; ++d) {
+            const int o = o0 + d;
             if (o < o_end) {      // warp-uniform
-                float sc = 1.0f;
-                if (!ACCF) sc = __fmul_rn(scale_a, scale_w[o]);
-                float sl[8], p[2][4];
-#pragma unroll
-                for (int s = 0; s < 8; ++s) {
-                    const int a = (j == 0) ? v[s].x : (j == 1) ? v[s].y : (j == 2) ? v[s].z : v[s].w;
-                    sl[s] = ACCF ? __int_as_float(a) : __fmul_rn((float)a, sc);
-                }
-                haar_inv_lane<L>(sl, p, lane);
                 if (residual) {                        // the skip connection (Eq. 13): one fp32 addition per element
                     RawPatch rr;
                     float rp[2][4];
@@ -1368,17 +1386,19 @@ scatter_inv_kernel(const int32_t* __restrict__ acc, int ldc, const int32_t* __re
 #pragma unroll
                     for (int a = 0; a < 2; ++a)
 #pragma unroll
-                        for (int b = 0; b < 4; ++b) p[a][b] = __fadd_rn(p[a][b], rp[a][b]);
+                        for (int b = 0; b < 4; ++b) p[d][a][b] = __fadd_rn(p[d][a][b], rp[a][b]);
                 }
                 if (relu) {
 #pragma unroll
                     for (int a = 0; a < 2; ++a)
 #pragma unroll
-                        for (int b = 0; b < 4; ++b) p[a][b] = fmaxf(p[a][b], 0.0f);
+                        for (int b = 0; b < 4; ++b) p[d][a][b] = fmaxf(p[d][a][b], 0.0f);
                 }
-                store_patch<T, VEC>(y + ((size_t)n * Cout + o) * P, W, lp, p);
+                store_patch<T, VEC>(y + ((size_t)n * Cout + o) * P, W, lp, p[d]);
             }
         }
+#pragma unroll
+        for (int s = 0; s < 8; ++s) v[s] = vn[s];
     }
 }
 
@@ -1524,17 +1544,20 @@ static wcc_status scatter_inv_dispatch(const int32_t* acc, int ldc, bool accf, c
                                        cudaStream_t st)
 {
     using TT = HaarTile<L>;
-    constexpr int OCW = 8;
-    const long long warps = (long long)N * ceil_div(W, TT::TW) * (H / TT::TH) * ceil_div(Cout, OCW);
+    // channels per warp: as many as still leave about 32 warps for each of the 148 SMs (8 to 64)
+    const long long tiles = (long long)N * ceil_div(W, TT::TW) * (H / TT::TH);
+    int ocw = 64;
+    while (ocw > 8 && tiles * ceil_div(Cout, ocw) < 148 * 32) ocw >>= 1;
+    const long long warps = tiles * ceil_div(Cout, ocw);
     const int blocks = (int)((warps + 3) / 4);
     if (accf)
-        scatter_inv_kernel<T, L, VEC, true, OCW><<<blocks, 128, 0, st>>>(acc, ldc, rank, amax_kept, qmax, scale_w,
-                                                                          N, Cout, H, W, k, static_cast<T*>(y),
-                                                                          static_cast<const T*>(residual), relu);
+        scatter_inv_kernel<T, L, VEC, true><<<blocks, 128, 0, st>>>(acc, ldc, rank, amax_kept, qmax, scale_w,
+                                                                     N, Cout, ocw, H, W, k, static_cast<T*>(y),
+                                                                     static_cast<const T*>(residual), relu);
     else
-        scatter_inv_kernel<T, L, VEC, false, OCW><<<blocks, 128, 0, st>>>(acc, ldc, rank, amax_kept, qmax, scale_w,
-                                                                           N, Cout, H, W, k, static_cast<T*>(y),
-                                                                           static_cast<const T*>(residual), relu);
+        scatter_inv_kernel<T, L, VEC, false><<<blocks, 128, 0, st>>>(acc, ldc, rank, amax_kept, qmax, scale_w,
+                                                                      N, Cout, ocw, H, W, k, static_cast<T*>(y),
+                                                                      static_cast<const T*>(residual), relu);
     WCC_LAUNCH_CHECK();
     return WCC_OK;
 }
