@@ -366,16 +366,26 @@ def block_context(wcc, torch, np, inputs, dev, flush, steps=30):
         y = torch.empty_like(x)
 
         def timed(fn):
+            # both arms are captured once and replayed, as the headline layer is: neither pays for its launches
             fn()
             torch.cuda.synchronize()
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                fn()
+            torch.cuda.current_stream().wait_stream(side)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                fn()
             ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
             for a, b in ev:
                 flush.fill_(1)
                 a.record()
-                fn()
+                g.replay()
                 b.record()
             torch.cuda.synchronize()
             t = [a.elapsed_time(b) for a, b in ev]
+            del g
             return sum(t) / len(t)
 
         W1b, W3b, Wdwb = W1.to(torch.bfloat16), W3.to(torch.bfloat16), Wdw.to(torch.bfloat16)[:, None]

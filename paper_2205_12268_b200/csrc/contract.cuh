@@ -56,6 +56,12 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8])
                  : "r"(taddr));
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void tmem_ld8_nowait(uint32_t taddr, uint32_t (&r)[8])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr));
+}
 __device__ __forceinline__ void fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -172,12 +178,27 @@ contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * TILE_N);
             const long long grow = (long long)mt * TILE_M + q * 32 + lane;
             int32_t* dst = acc + grow * ldc + n0;
-            for (int c0 = 0; c0 < cur && n0 + c0 < ldc; c0 += 8) {
-                uint32_t r[8];
-                tmem_ld8(taddr + (uint32_t)c0, r);
+            for (int c0 = 0; c0 < cur && n0 + c0 < ldc; c0 += 32) {       // 32 columns per wait: a 128-byte line per lane
+                uint32_t r[4][8];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (c0 + 8 * j < cur) {             // warp-uniform
+                        tmem_ld8_nowait(taddr + (uint32_t)(c0 + 8 * j), r[j]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) r[j][i] = 0u;
+                    }
+                }
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 if (grow < M) {
-                    *reinterpret_cast<uint4*>(dst + c0) = make_uint4(r[0], r[1], r[2], r[3]);
-                    if (n0 + c0 + 4 < ldc) *reinterpret_cast<uint4*>(dst + c0 + 4) = make_uint4(r[4], r[5], r[6], r[7]);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int c = c0 + 8 * j;
+                        if (c < cur && n0 + c < ldc) {
+                            *reinterpret_cast<uint4*>(dst + c) = make_uint4(r[j][0], r[j][1], r[j][2], r[j][3]);
+                            if (n0 + c + 4 < ldc) *reinterpret_cast<uint4*>(dst + c + 4) = make_uint4(r[j][4], r[j][5], r[j][6], r[j][7]);
+                        }
+                    }
                 }
             }
             fence_before();

@@ -76,6 +76,7 @@ struct Params {
     const void* residual;        // NULL, or [N][Cout][H][W] of the activation type, added before the ReLU
     NextNorms nx;                // kernel variant NEXT only
     int N, Cin, Cout, H, W, k, kpad, npad, nchunk, nn, nbuf, tmem_cols, na, tiles_total;
+    int split_from, parts;       // CTAs from split_from on share a tile group `parts` ways by output channels
     void* y; uint8_t* xq_tap; int32_t* acc_tap; int* status;
 };
 
@@ -110,6 +111,16 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool is_mma = warp == C::CWARPS;
     const int t = warp & 3, q = warp >> 2;
+    // The last, partial wave of tile groups is spread over the SMs that would idle: `parts` CTAs take one group each,
+    // all of them build the whole operand (the transform and quantization are repeated) and each runs the contraction and
+    // the way out for its own share of the output channels.
+    int grp = (int)blockIdx.x, o_lo = 0, o_cnt = pr.npad;
+    if ((int)blockIdx.x >= pr.split_from) {
+        const int r = (int)blockIdx.x - pr.split_from;
+        grp = pr.split_from + r / pr.parts;
+        o_cnt = pr.npad / pr.parts;
+        o_lo = (r % pr.parts) * o_cnt;
+    }
 
     // ---- set-up -------------------------------------------------------------------------------------
     if (threadIdx.x == 0) {
@@ -127,7 +138,7 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
         // Lane w of this warp starts the input ring of compute warp w (barriers and the first S boxes), so that the
         // compute warps spend the set-up on their own global loads instead of waiting for the first TMA issue.
         if (lane < C::CWARPS) {
-            const int t2 = lane & 3, q2 = lane >> 2, tile2 = (int)blockIdx.x * TILES + t2;
+            const int t2 = lane & 3, q2 = lane >> 2, tile2 = grp * TILES + t2;
             const uint32_t bar2 = tc::smem_u32(ring_bars + lane * C::S);
             const uint32_t ring2 = tc::smem_u32(sRing + (size_t)lane * Ring::BYTES);
 #pragma unroll
@@ -149,7 +160,7 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
         }
         __syncwarp();
     }
-    const int tile = (int)blockIdx.x * TILES + t;
+    const int tile = grp * TILES + t;
     const bool live = !is_mma && tile < pr.tiles_total;
     int n = 0, ty = 0, tx = 0;
     if (live) tile_coords(tile, tiles_x, tiles_y, n, ty, tx);
@@ -164,10 +175,10 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
     Ring ring;
     if (!is_mma) ring.attach(sRing + (size_t)warp * Ring::BYTES, ring_bars + warp * C::S, lane);
     // weights -> B operand (core-matrix layout), all threads
-    for (int i = threadIdx.x; i < pr.npad * kchunks; i += C::THREADS) {
+    for (int i = threadIdx.x; i < o_cnt * kchunks; i += C::THREADS) {      // rows o_lo .. o_lo + o_cnt of the weights
         const int row = i / kchunks, j = i - row * kchunks;
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (row < pr.Cout) v = *reinterpret_cast<const uint4*>(pr.Wq + (size_t)row * krow + j * 16);
+        if (o_lo + row < pr.Cout) v = *reinterpret_cast<const uint4*>(pr.Wq + (size_t)(o_lo + row) * krow + j * 16);
         *reinterpret_cast<uint4*>(sB + ((size_t)j * pr.npad + row) * 16) = v;
     }
     // kept or dropped: from the rank map when the select wrote one (thr[n][2] != 0), else by the threshold key
@@ -232,7 +243,7 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
                     ok = tc::mbar_wait(tc::smem_u32(&ctl->full_a[buf]), (uint32_t)(ks / pr.na) & 1u, abort_flag);
                     if (!ok) break;
                     tc::fence_after();
-                    mma_kstep(ks, buf, 0, pr.npad, tmem, ks == 0);
+                    mma_kstep(ks, buf, 0, o_cnt, tmem, ks == 0);
                     tc::mma_commit(tc::smem_u32(&ctl->empty_a[buf]));
                 }
                 if (ok) tc::mma_commit(tc::smem_u32(&ctl->ready[0]));
@@ -364,9 +375,9 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
             ok = __all_sync(0xFFFFFFFFu, ok ? 1 : 0) != 0;
             if (!ok) break;
             tc::fence_after();
-            const int n0 = c * pr.nchunk, cur = min(pr.nchunk, pr.npad - n0);
+            const int n0 = c * pr.nchunk, cur = min(min(pr.nchunk, pr.npad - n0), o_cnt);
             for (int g = q; g * 8 < cur; g += WPT) {
-                const int o0 = n0 + g * 8;
+                const int o0 = o_lo + n0 + g * 8;      // first output channel of the group
                 if (!live || o0 >= pr.Cout) continue;
                 uint32_t r[8][8];                      // [slot][channel]
                 const uint32_t taddr = tmem + ((uint32_t)(t * 32) << 16) + (uint32_t)(tb * 8 * pr.nchunk + g * 8);
@@ -560,7 +571,21 @@ static wcc_status fused_tiles_dispatch(const void* x, const void* Wq, const int3
     pr.y = y; pr.xq_tap = static_cast<uint8_t*>(xq_tap); pr.acc_tap = acc_tap;
     pr.alpha = fx.alpha; pr.relu = fx.relu; pr.residual = fx.residual;
     WCC_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&pr.status), g_status));
-    const unsigned ctas = (unsigned)((tiles + ft::TILES - 1) / ft::TILES);
+    const unsigned groups = (unsigned)((tiles + ft::TILES - 1) / ft::TILES);
+    // One CTA per SM at a time: the groups run in waves.  The groups of a last, partial wave are shared 4 or 2 ways by
+    // output channels when that still fits one wave (the SMs would idle otherwise); the chain variant keeps whole
+    // groups, its norm chain runs over all output channels of a tile.
+    int dev = 0, sms = 0;
+    WCC_CUDA_TRY(cudaGetDevice(&dev));
+    WCC_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const unsigned rem = sms > 0 ? groups % (unsigned)sms : 0u;
+    pr.parts = 1;
+    if (plan.nn == 1 && !nx && rem > 0) {
+        for (int parts = 4; parts >= 2; parts >>= 1)
+            if (rem * (unsigned)parts <= (unsigned)sms && plan.npad % (16 * parts) == 0) { pr.parts = parts; break; }
+    }
+    pr.split_from = (pr.parts > 1) ? (int)(groups - rem) : (int)groups;
+    const unsigned ctas = (unsigned)pr.split_from + (groups - (unsigned)pr.split_from) * (unsigned)pr.parts;
     auto launch = [&](auto kern, int threads) -> wcc_status {
         WCC_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         kern<<<ctas, threads, smem, st>>>(tmx, pr);
