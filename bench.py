@@ -33,9 +33,13 @@ STAGE_FILES = ("haar.cuh", "select.cuh", "gather.cuh", "contract.cuh", "fused.cu
 # DRAM bytes per launch of the dominant kernel from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum),
 # keyed by (workload, stage); valid only while the kernel sources still hash to `src`.
 NCU_TRAFFIC = {
-    # captured with N=16 images of C2 (x = 151 MB > L2) and divided by 4: every stage is per image
-    ("C2", "fused_pass2"): {"bytes": (153168896 + 13174272) / 4, "src": "858dc5d135d2"},
-    ("C2", "haar_norms"): {"bytes": (151201536 + 4285184) / 4, "src": "858dc5d135d2"},
+    # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu captures summarised under profiles/.
+    # C4 was captured with N=24 images (x = 189 MB > L2) and is divided by 2, C2 with N=16 and divided by 4: every stage
+    # is per image, so traffic grows in proportion to the batch.
+    ("C4", "fused_pass2"): {"bytes": (191774208 + 135275264) / 2, "src": "29cee81a216b"},
+    ("C4", "haar_norms"): {"bytes": (189054208 + 4007424) / 2, "src": "29cee81a216b"},
+    ("C2", "fused_pass2"): {"bytes": (153169920 + 13190656) / 4, "src": "29cee81a216b"},
+    ("C2", "haar_norms"): {"bytes": (151204608 + 4880128) / 4, "src": "29cee81a216b"},
 }
 
 
@@ -347,22 +351,32 @@ def chain_context(wcc, torch, np, inputs, dev, flush, peak, use_graph, steps=100
     return out
 
 
+# (N, c_in, expansion, H, W, keep ratio): a few of the shapes of the paper's own GPU benchmark of the block (App. H, Table 8)
+BLOCK_SHAPES = [(8, 512, 2, 96, 96, 0.25), (4, 256, 4, 128, 128, 0.25), (2, 256, 4, 256, 256, 0.125), (2, 128, 4, 128, 128, 0.25)]
+
+
+def make_block(wcc, torch, inputs, dev, shape):
+    N, Cc, e, H, W, gamma = shape
+    E = Cc * e
+    g = torch.Generator(device=dev).manual_seed(Cc + H)
+    x = torch.relu(torch.randn((N, Cc, H, W), device=dev, generator=g)).to(torch.bfloat16)
+    W1 = torch.randn((E, Cc), device=dev, generator=g) / Cc ** 0.5
+    W3 = torch.randn((Cc, E), device=dev, generator=g) / E ** 0.5
+    Wdw = torch.randn((E, 3, 3), device=dev, generator=g) / 3
+    blk = wcc.Block(x, W1, Wdw, W3, 3, inputs.keep_count(gamma, H * W), 8)
+    return x, W1, Wdw, W3, blk
+
+
 def block_context(wcc, torch, np, inputs, dev, flush, steps=30):
     """The inverted residual block of the paper's own GPU benchmark, y = x + K3(Kdw(K1 x)) with both pointwise
     convolutions as WCC layers (three levels, 8 bits) at a few of its shapes, beside the same block with dense bf16
     library kernels (matmul, grouped conv2d).  Batches are smaller than the paper's (its batches filled an 11 GB card)."""
     import torch.nn.functional as F
-    shapes = [(8, 512, 2, 96, 96, 0.25), (4, 256, 4, 128, 128, 0.25), (2, 256, 4, 256, 256, 0.125), (2, 128, 4, 128, 128, 0.25)]
     out = []
-    for (N, Cc, e, H, W, gamma) in shapes:
+    for shape in BLOCK_SHAPES:
+        N, Cc, e, H, W, gamma = shape
         E = Cc * e
-        g = torch.Generator(device=dev).manual_seed(Cc + H)
-        x = torch.relu(torch.randn((N, Cc, H, W), device=dev, generator=g)).to(torch.bfloat16)
-        W1 = torch.randn((E, Cc), device=dev, generator=g) / Cc ** 0.5
-        W3 = torch.randn((Cc, E), device=dev, generator=g) / E ** 0.5
-        Wdw = torch.randn((E, 3, 3), device=dev, generator=g) / 3
-        k = inputs.keep_count(gamma, H * W)
-        blk = wcc.Block(x, W1, Wdw, W3, 3, k, 8)
+        x, W1, Wdw, W3, blk = make_block(wcc, torch, inputs, dev, shape)
         y = torch.empty_like(x)
 
         def timed(fn):
@@ -430,6 +444,16 @@ def run_ours(args):
         dist.barrier()
     wcc.lib()
 
+    if args.workload.startswith("block"):               # profiling aid: one inverted residual block alone (eager launches)
+        shape = BLOCK_SHAPES[int(args.workload[5:] or 0)]
+        x, _, _, _, blk = make_block(wcc, torch, inputs, dev, shape)
+        y = torch.empty_like(x)
+        for _ in range(max(3, args.warmup) + args.steps):
+            blk(x, y)
+        torch.cuda.synchronize()
+        assert wcc.last_status() == 0
+        print(json.dumps({"workload": "inverted residual block N=%d c=%d e=%d %dx%d keep=%g" % shape, "lean": True}))
+        return 0
     if args.workload == "C5chain":                      # profiling aid: the six-layer chain alone (three levels, keep 1/4)
         flush = torch.empty(FLUSH_BYTES, dtype=torch.uint8, device=dev)
         peak, _ = _peaks()
