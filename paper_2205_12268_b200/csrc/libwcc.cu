@@ -2,6 +2,7 @@
 #include "common.cuh"
 #include "gather.cuh"
 #include "haar.cuh"
+#include "regather.cuh"
 #include "select.cuh"
 #include "contract.cuh"
 #include "fused.cuh"
@@ -258,6 +259,111 @@ static wcc_status check_options(const wcc_options* o, int bits, const void* x, c
     return WCC_OK;
 }
 
+// ---- many channels: two passes over x, the kept columns gathered from the second ---------------------------------
+// Layers beyond one operand tile of the fused kernels.  Like the fused path, the first pass keeps only norms, maxima and
+// histograms; the select writes index list and rank map; the kept columns are then transformed again and quantized
+// straight into the compressed matrix (no coefficient map in memory), and the contraction over the kept columns, the
+// scatter and the inverse transform follow as in the stage-by-stage pipeline.
+struct WideWs {
+    float* nrm2; float* amaxpos; int32_t* rank; int32_t* idx; uint32_t* thr; uint32_t* fine; size_t fine_bytes;
+    void* sel; size_t sel_bytes; float* amax_kept; void* Xq; void* Wq; float* scale_w; int32_t* acc;
+    int kpad, ldc, es;
+    size_t total;
+};
+
+static WideWs carve_wide_ws(void* ws, int N, int Cin, int Cout, int H, int W, int k, int bits)
+{
+    WideWs f;
+    const size_t P = (size_t)H * W, M = (size_t)N * k;
+    f.kpad = wcc_kpad(Cin, bits);
+    f.es = (bits == 0) ? 2 : 1;
+    f.ldc = ceil_div(Cout, 4) * 4;
+    size_t off = 0;
+    char* b = static_cast<char*>(ws);
+    auto take = [&](size_t bytes) { char* p = b ? b + off : nullptr; off += align_up(bytes, 256); return p; };
+    f.nrm2 = reinterpret_cast<float*>(take((size_t)N * P * 4));
+    f.amaxpos = reinterpret_cast<float*>(take((size_t)N * P * 4));
+    f.rank = reinterpret_cast<int32_t*>(take((size_t)N * P * 4));
+    f.idx = reinterpret_cast<int32_t*>(take(M * 4));
+    f.thr = reinterpret_cast<uint32_t*>(take((size_t)N * 16));
+    f.fine_bytes = align_up((size_t)N * FINE_BINS * 4, 256);       // right before the select scratch: one memset clears both
+    f.fine = reinterpret_cast<uint32_t*>(take(f.fine_bytes));
+    f.sel_bytes = select_ws_bytes(N, (int)P);
+    f.sel = take(f.sel_bytes);
+    f.amax_kept = b ? carve_select_ws(f.sel, N, (int)P).amax : nullptr;
+    f.Xq = take(M * f.kpad * f.es);
+    f.Wq = take((size_t)Cout * f.kpad * f.es);
+    f.scale_w = reinterpret_cast<float*>(take((size_t)Cout * 4));
+    f.acc = reinterpret_cast<int32_t*>(take(M * f.ldc * 4));
+    f.total = off;
+    return f;
+}
+
+// One cluster per image in the selection (it reads the first pass's histograms), vector loads of whole patches.
+static bool wide_fits(const void* x, int Cin, int Cout, int H, int W, int bits, wcc_dtype dt)
+{
+    (void)x; (void)dt;
+    return staged_fits(Cin, Cout, bits) && select_in_cluster(H * W) && (W % 4) == 0;
+}
+
+static wcc_status wide_impl(const void* x, const float* Wt, int N, int Cin, int Cout, int H, int W,
+                            int L, int k, int bits, void* y, wcc_dtype dt, void* ws, size_t ws_bytes,
+                            cudaStream_t st, const wcc_taps* taps, const wcc_options* opt)
+{
+    const WideWs f = carve_wide_ws(ws, N, Cin, Cout, H, W, k, bits);
+    if (ws_bytes < f.total) return WCC_ERR_WORKSPACE;
+    const int P = H * W, M = N * k;
+    wcc_status s;
+    if ((s = profile_mark(0, st)) != WCC_OK) return s;
+    const SelectWs sw = carve_select_ws(f.sel, N, P);
+    WCC_CUDA_TRY(cudaMemsetAsync(f.fine, 0, f.fine_bytes + sw.zero_bytes, st));       // histograms, max |kept|, barrier counters
+    NormsExtra ex = {};
+    ex.hist1 = sw.hist;
+    ex.fine = f.fine;
+    const int wbits = (opt && opt->weight_bits && bits) ? opt->weight_bits : bits;
+    ex.Wt = Wt; ex.Wq = f.Wq; ex.scale_w = f.scale_w; ex.Cout = Cout; ex.kpad = f.kpad; ex.bits = wbits;
+    s = launch_haar_norms(x, N, Cin, H, W, L, dt, f.nrm2, f.amaxpos, ex, st);
+    if (s != WCC_OK) return s;
+    if ((s = profile_mark(1, st)) != WCC_OK) return s;
+    s = launch_select(f.nrm2, N, P, k, f.idx, nullptr, f.rank, f.amaxpos, true, f.sel, f.sel_bytes, st, true, f.fine, f.thr, true);
+    if (s != WCC_OK) return s;
+    if (opt && opt->alpha > 0.0f && bits >= 2) {        // a given clipping parameter replaces the largest kept magnitude
+        set_word_kernel<<<1, 1, 0, st>>>(f.amax_kept, opt->alpha);
+        WCC_LAUNCH_CHECK();
+    }
+    for (int i = 2; i <= 3; ++i)
+        if ((s = profile_mark(i, st)) != WCC_OK) return s;
+    s = launch_regather_quant(x, f.rank, f.amax_kept, N, Cin, H, W, L, k, f.kpad, bits, dt, f.Xq, st);
+    if (s != WCC_OK) return s;
+    if ((s = profile_mark(4, st)) != WCC_OK) return s;
+    s = launch_contract(f.Xq, f.Wq, M, Cout, f.kpad, bits, f.acc, f.ldc, st);
+    if (s != WCC_OK) return s;
+    if ((s = profile_mark(5, st)) != WCC_OK) return s;
+    s = launch_scatter_inv(f.acc, f.ldc, bits == 0, f.rank, f.amax_kept, bits, f.scale_w, N, Cout, H, W, L, k, dt, y, st,
+                           opt ? opt->residual : nullptr, opt ? opt->relu : 0);
+    if (s != WCC_OK) return s;
+    if ((s = profile_mark(6, st)) != WCC_OK) return s;
+    if (taps) {
+        const cudaMemcpyKind dd = cudaMemcpyDeviceToDevice;
+        if (taps->nrm2) WCC_CUDA_TRY(cudaMemcpyAsync(taps->nrm2, f.nrm2, (size_t)N * P * 4, dd, st));
+        if (taps->idx) WCC_CUDA_TRY(cudaMemcpyAsync(taps->idx, f.idx, (size_t)M * 4, dd, st));
+        if (bits >= 2) {
+            if (taps->Xq) WCC_CUDA_TRY(cudaMemcpyAsync(taps->Xq, f.Xq, (size_t)M * f.kpad, dd, st));
+            if (taps->Wq) WCC_CUDA_TRY(cudaMemcpyAsync(taps->Wq, f.Wq, (size_t)Cout * f.kpad, dd, st));
+            if (taps->scale_w) WCC_CUDA_TRY(cudaMemcpyAsync(taps->scale_w, f.scale_w, (size_t)Cout * 4, dd, st));
+            if (taps->scale_a) {
+                scale_tap_kernel<<<1, 1, 0, st>>>(f.amax_kept, 0.0f, (float)((1 << (bits - 1)) - 1), taps->scale_a);
+                WCC_LAUNCH_CHECK();
+            }
+        } else if (taps->Xb) {
+            WCC_CUDA_TRY(cudaMemcpyAsync(taps->Xb, f.Xq, (size_t)M * f.kpad * 2, dd, st));
+        }
+        if (taps->acc)
+            WCC_CUDA_TRY(cudaMemcpy2DAsync(taps->acc, (size_t)Cout * 4, f.acc, (size_t)f.ldc * 4, (size_t)Cout * 4, M, dd, st));
+    }
+    return WCC_OK;
+}
+
 // Chain fusion hooks of forward_impl: norms_ready = the previous layer's second pass has already produced this layer's
 // norms, per-position maxima and histograms in this workspace (no first pass; the weights are quantized by a launch of
 // their own); next_ws = workspace of the next layer, whose first pass this layer's second pass performs.
@@ -292,6 +398,8 @@ static wcc_status forward_impl(const void* x, const float* Wt, int N, int Cin, i
         return WCC_ERR_ALIGN;
     if (!fused_fits(x, Cout, W, bits, dt, Cin)) {      // decided before anything is launched: channel counts beyond one
         if (own_codes) return WCC_ERR_SHAPE;           // operand tile run stage by stage (the contraction there tiles K and N)
+        if (wide_fits(x, Cin, Cout, H, W, bits, dt) && !(taps && taps->coef))
+            return wide_impl(x, Wt, N, Cin, Cout, H, W, L, k, bits, y, dt, ws, ws_bytes, st, taps, opt);
         return staged_impl(x, Wt, N, Cin, Cout, H, W, L, k, bits, y, dt, ws, ws_bytes, st, taps, opt);
     }
     const FusedWs f = carve_fused_ws(ws, N, Cin, Cout, H, W, k, bits);
@@ -541,8 +649,12 @@ int wcc_kpad(int Cin, int bits)
 size_t wcc_workspace_bytes(int N, int Cin, int Cout, int H, int Wd, int levels, int k, int bits, wcc_dtype dt)
 {
     if (check_forward_args(N, Cin, Cout, H, Wd, levels, k, bits, dt) != WCC_OK) return 0;
-    if (!fused_fits(nullptr, Cout, Wd, bits, dt, Cin))                         // these shapes run stage by stage
-        return staged_fits(Cin, Cout, bits) ? carve_forward_ws(nullptr, N, Cin, Cout, H, Wd, k, bits).total : 0;
+    if (!fused_fits(nullptr, Cout, Wd, bits, dt, Cin)) {                       // these shapes run around the tiled contraction
+        if (!staged_fits(Cin, Cout, bits)) return 0;
+        const size_t a = carve_forward_ws(nullptr, N, Cin, Cout, H, Wd, k, bits).total;
+        const size_t b = carve_wide_ws(nullptr, N, Cin, Cout, H, Wd, k, bits).total;
+        return a > b ? a : b;
+    }
     return carve_fused_ws(nullptr, N, Cin, Cout, H, Wd, k, bits).total;
 }
 
