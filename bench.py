@@ -27,8 +27,8 @@ if ROOT not in sys.path:
 METRIC = "WCC layer output Gpix/s"
 UNIT = "Gpix/s"
 FLUSH_BYTES = 256 << 20          # > 126 MB of L2
-STAGE_FILES = ("haar.cuh", "select.cuh", "gather.cuh", "contract.cuh", "fused.cuh", "fused_tiles.cuh", "tma.cuh", "libwcc.cu",
-               "common.cuh")
+STAGE_FILES = ("haar.cuh", "select.cuh", "gather.cuh", "regather.cuh", "contract.cuh", "fused.cuh", "fused_tiles.cuh", "tma.cuh",
+               "libwcc.cu", "common.cuh")
 
 # DRAM bytes per launch of the dominant kernel from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum),
 # keyed by (workload, stage); valid only while the kernel sources still hash to `src`.
@@ -36,10 +36,10 @@ NCU_TRAFFIC = {
     # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu captures summarised under profiles/.
     # C4 was captured with N=24 images (x = 189 MB > L2) and is divided by 2, C2 with N=16 and divided by 4: every stage
     # is per image, so traffic grows in proportion to the batch.
-    ("C4", "fused_pass2"): {"bytes": (191774208 + 135275264) / 2, "src": "29cee81a216b"},
-    ("C4", "haar_norms"): {"bytes": (189054208 + 4007424) / 2, "src": "29cee81a216b"},
-    ("C2", "fused_pass2"): {"bytes": (153169920 + 13190656) / 4, "src": "29cee81a216b"},
-    ("C2", "haar_norms"): {"bytes": (151204608 + 4880128) / 4, "src": "29cee81a216b"},
+    ("C4", "fused_pass2"): {"bytes": (191774208 + 135275264) / 2, "src": "2fcf053994b2"},
+    ("C4", "haar_norms"): {"bytes": (189054208 + 4007424) / 2, "src": "2fcf053994b2"},
+    ("C2", "fused_pass2"): {"bytes": (153169920 + 13190656) / 4, "src": "2fcf053994b2"},
+    ("C2", "haar_norms"): {"bytes": (151204608 + 4880128) / 4, "src": "2fcf053994b2"},
 }
 
 
