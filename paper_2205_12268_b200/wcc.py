@@ -368,7 +368,8 @@ def forward(x: torch.Tensor, Wt: torch.Tensor | None, levels: int, k: int, bits:
             ws: Workspace | None = None, taps: bool = False, staged: bool = False, alpha: float = 0.0, wbits: int = 0,
             relu: bool = False, residual: torch.Tensor | None = None, Wq: torch.Tensor | None = None,
             scale_w: torch.Tensor | None = None):
-    """The WCC layer.  Returns y, or (y, dict of intermediate tensors) when ``taps`` is set.
+    """The WCC layer.  Returns y, or (y, dict of intermediate tensors) when ``taps`` is set (True: all of them; or an
+    iterable of names out of coef, nrm2, idx, acc, Xq / Xb, scale_a, Wq, scale_w).
     ``staged`` selects wcc_forward_staged (every intermediate in memory) instead of the fused wcc_forward.
     ``alpha``, ``wbits``, ``relu``, ``residual``, ``Wq`` + ``scale_w``: the options of wcc_forward_ex (see wcc.h);
     with pre-quantized weights ``Wt`` may be None."""
@@ -419,6 +420,8 @@ def forward(x: torch.Tensor, Wt: torch.Tensor | None, levels: int, k: int, bits:
                  Wq=torch.empty((Cout, kp), dtype=torch.int8, device=dev), scale_w=torch.empty((Cout,), dtype=torch.float32, device=dev))
     else:
         t.update(Xb=torch.empty((M, kp), dtype=torch.bfloat16, device=dev))
+    if taps is not True:
+        t = {name: v for name, v in t.items() if name in set(taps)}
     for name in ("Xq", "Xb", "acc"):          # every row is a kept position and gets written; start from zeros anyway
         if name in t:
             t[name].zero_()

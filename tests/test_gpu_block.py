@@ -72,6 +72,32 @@ def test_layer_with_many_channels(wcc, cfg):
         assert np.abs(y.float().cpu().numpy() - want).max() <= 2e-2 * np.abs(want).max()
 
 
+@pytest.mark.parametrize("cfg", LARGE + [(2, 288, 72, 32, 64, "bf16", 2, 0.25, 8), (1, 40, 520, 16, 32, "f32", 1, 0.3, 5)],
+                         ids=lambda c: "N%d_%dto%d_%dx%d_%s_L%d_g%s_b%d" % c)
+def test_wide_layer_without_coefficient_map(wcc, cfg):
+    """Without the coefficient tap these layers take two passes over x (the kept columns are transformed again and
+    quantized straight into the compressed matrix): every other intermediate is still identical to the oracle's."""
+    N, Cin, Cout, H, W, dtype, L, gamma, bits = cfg
+    w = inputs.custom("wide", 43, N, Cin, Cout, H, W, dtype, L, gamma, bits, n_sin=4, fmax=3.0)
+    x = torch.from_numpy(w.x.view(np.int16)).cuda().view(torch.bfloat16) if dtype == "bf16" else torch.from_numpy(w.x).cuda()
+    names = ("nrm2", "idx", "acc", "Xq", "scale_a", "Wq", "scale_w") if bits else ("nrm2", "idx", "Xb")
+    y, t = wcc.forward(x, torch.from_numpy(w.Wt).cuda(), L, w.k, bits, taps=names)
+    assert wcc.last_status() == 0
+    want, o = oracle.forward(w.x_f32(), w.Wt, L, w.k, bits, out_bf16=(dtype == "bf16"), taps=True)
+    assert np.array_equal(_bits(t["nrm2"].cpu().numpy()), _bits(o["nrm2"]))
+    assert np.array_equal(t["idx"].cpu().numpy(), o["idx"])
+    if bits:
+        kp = t["Xq"].shape[1]
+        assert np.array_equal(t["Xq"].cpu().numpy()[:, :Cin], o["Xq"].reshape(-1, o["Xq"].shape[-1])[:, :Cin])
+        assert not t["Xq"].cpu().numpy()[:, Cin:kp].any()
+        assert np.array_equal(t["acc"].cpu().numpy(), o["acc"].reshape(-1, Cout))
+        assert np.array_equal(_bits(y.float().cpu().numpy()), _bits(want))
+        y2 = wcc.forward(x, torch.from_numpy(w.Wt).cuda(), L, w.k, bits)        # plain call, same path
+        assert torch.equal(y, y2)
+    else:
+        assert np.abs(y.float().cpu().numpy() - want).max() <= 2e-2 * np.abs(want).max()
+
+
 BLOCKS = [  # N, C, E, H, W, dtype, levels, gamma
     (2, 8, 32, 16, 32, "f32", 2, 0.5),
     (1, 16, 96, 32, 64, "bf16", 3, 0.25),
