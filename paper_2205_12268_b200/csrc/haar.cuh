@@ -632,7 +632,9 @@ struct DwRaw {
     float k[9];
 };
 
-template <typename T, bool VEC>
+// ER / EC: the tile touches the top or bottom / the left or right border of the map (or hangs over it), so rows / columns
+// of the neighbourhood can fall outside; tiles in the interior load without any bounds test.
+template <typename T, bool VEC, bool ER = true, bool EC = true>
 __device__ __forceinline__ void dwconv_load(const T* __restrict__ plane, const float* __restrict__ w9, const LanePos& lp,
                                             int H, int W, DwRaw<T, VEC>& r)
 {
@@ -645,17 +647,17 @@ __device__ __forceinline__ void dwconv_load(const T* __restrict__ plane, const f
 #pragma unroll
     for (int a = 0; a < 4; ++a) {
         const int rr = lp.r0 + a - 1;
-        const bool row_in = rr >= 0 && rr < H;
+        const bool row_in = !ER || (rr >= 0 && rr < H);
         if constexpr (VEC) {
-            const uint32_t left = (row_in && lp.c0 > 0 && lp.c0 - 1 < W) ? load1(rr, lp.c0 - 1) : 0u;
-            const uint32_t right = (row_in && lp.c0 + 4 < W) ? load1(rr, lp.c0 + 4) : 0u;
+            const uint32_t left = (row_in && (!EC || (lp.c0 > 0 && lp.c0 - 1 < W))) ? load1(rr, lp.c0 - 1) : 0u;
+            const uint32_t right = (row_in && (!EC || lp.c0 + 4 < W)) ? load1(rr, lp.c0 + 4) : 0u;
             if constexpr (sizeof(T) == 4) {
                 uint4 m = make_uint4(0u, 0u, 0u, 0u);
-                if (row_in && lp.ok0) m = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint32_t*>(plane) + (size_t)rr * W + lp.c0));
+                if (row_in && (!EC || lp.ok0)) m = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint32_t*>(plane) + (size_t)rr * W + lp.c0));
                 r.v[a][0] = left; r.v[a][1] = m.x; r.v[a][2] = m.y; r.v[a][3] = m.z; r.v[a][4] = m.w; r.v[a][5] = right;
             } else {
                 uint2 m = make_uint2(0u, 0u);
-                if (row_in && lp.ok0) m = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const unsigned short*>(plane) + (size_t)rr * W + lp.c0));
+                if (row_in && (!EC || lp.ok0)) m = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const unsigned short*>(plane) + (size_t)rr * W + lp.c0));
                 r.v[a][0] = m.x; r.v[a][1] = m.y; r.v[a][2] = (left >> 16) | right;
             }
         } else {
@@ -698,8 +700,47 @@ __device__ __forceinline__ void dwconv_compute(const DwRaw<T, VEC>& r, float (&p
         }
 }
 
-// NORMS = false: a chunk of the channels (blockIdx.y), coefficients only.  The next channel's input is loaded while
-// the current one is convolved and transformed.
+// Channels [c_lo, c_hi) of one tile, two at a time: while one channel is convolved and transformed the next one's input
+// is in flight (two register buffers that swap roles).
+template <typename T, int L, bool VEC, bool NORMS, bool ER, bool EC>
+__device__ __forceinline__ void dwconv_channels(const T* __restrict__ uin, const float* __restrict__ w, float* __restrict__ cout,
+                                                int c_lo, int c_hi, const LanePos& lp, int lane, int n, int H, int W,
+                                                float* __restrict__ nrm2, float* __restrict__ amaxpos)
+{
+    const size_t P = (size_t)H * W;
+    float nacc[8], amax[8];
+#pragma unroll
+    for (int s = 0; s < 8; ++s) { nacc[s] = 0.0f; amax[s] = 0.0f; }
+    auto finish = [&](const DwRaw<T, VEC>& r, int c) {
+        float p[2][4], o[8];
+        dwconv_compute<T, VEC>(r, p);
+        haar_fwd_lane<L>(p, o, lane);
+        if (cout) store_slots<L, VEC>(cout + (size_t)c * P, lp, o);
+        if (NORMS) {
+#pragma unroll
+            for (int s = 0; s < 8; ++s) {
+                nacc[s] = __fmaf_rn(o[s], o[s], nacc[s]);
+                amax[s] = fmaxf(amax[s], fabsf(o[s]));
+            }
+        }
+    };
+    DwRaw<T, VEC> a, b;
+    if (c_lo < c_hi) dwconv_load<T, VEC, ER, EC>(uin + (size_t)c_lo * P, w + (size_t)c_lo * 9, lp, H, W, a);
+    for (int c = c_lo; c < c_hi; c += 2) {
+        if (c + 1 < c_hi) dwconv_load<T, VEC, ER, EC>(uin + (size_t)(c + 1) * P, w + (size_t)(c + 1) * 9, lp, H, W, b);
+        finish(a, c);
+        if (c + 1 < c_hi) {
+            if (c + 2 < c_hi) dwconv_load<T, VEC, ER, EC>(uin + (size_t)(c + 2) * P, w + (size_t)(c + 2) * 9, lp, H, W, a);
+            finish(b, c + 1);
+        }
+    }
+    if (NORMS) {
+        if (nrm2) store_slots<L, VEC>(nrm2 + (size_t)n * P, lp, nacc);
+        if (amaxpos) store_slots<L, VEC>(amaxpos + (size_t)n * P, lp, amax);
+    }
+}
+
+// NORMS = false: a chunk of the channels (blockIdx.y), coefficients only.
 template <typename T, int L, bool VEC, bool NORMS>
 __global__ void __launch_bounds__(128)
 dwconv_haar_fwd_kernel(const T* __restrict__ u, const float* __restrict__ w, int N, int C, int H, int W, int cpc,
@@ -718,31 +759,13 @@ dwconv_haar_fwd_kernel(const T* __restrict__ u, const float* __restrict__ w, int
     float* cout = coef ? coef + (size_t)n * C * P : nullptr;
     const int c_lo = (int)blockIdx.y * cpc, c_hi = min(C, c_lo + cpc);
 
-    float nacc[8], amax[8];
-#pragma unroll
-    for (int s = 0; s < 8; ++s) { nacc[s] = 0.0f; amax[s] = 0.0f; }
-    DwRaw<T, VEC> cur, nxt;
-    dwconv_load<T, VEC>(uin + (size_t)c_lo * P, w + (size_t)c_lo * 9, lp, H, W, cur);
-    nxt = cur;
-    for (int c = c_lo; c < c_hi; ++c) {
-        if (c + 1 < c_hi) dwconv_load<T, VEC>(uin + (size_t)(c + 1) * P, w + (size_t)(c + 1) * 9, lp, H, W, nxt);
-        float p[2][4], o[8];
-        dwconv_compute<T, VEC>(cur, p);
-        haar_fwd_lane<L>(p, o, lane);
-        if (cout) store_slots<L, VEC>(cout + (size_t)c * P, lp, o);
-        if (NORMS) {
-#pragma unroll
-            for (int s = 0; s < 8; ++s) {
-                nacc[s] = __fmaf_rn(o[s], o[s], nacc[s]);
-                amax[s] = fmaxf(amax[s], fabsf(o[s]));
-            }
-        }
-        cur = nxt;
-    }
-    if (NORMS) {
-        if (nrm2) store_slots<L, VEC>(nrm2 + (size_t)n * P, lp, nacc);
-        if (amaxpos) store_slots<L, VEC>(amaxpos + (size_t)n * P, lp, amax);
-    }
+    // border tests only where the tile needs them
+    const int ty0 = ty * TT::TH, tx0 = tx * TT::TW;
+    const bool er = !(ty0 >= 1 && ty0 + TT::TH < H), ec = !(tx0 >= 1 && tx0 + TT::TW < W);
+    if (!VEC || (er && ec)) dwconv_channels<T, L, VEC, NORMS, true, true>(uin, w, cout, c_lo, c_hi, lp, lane, n, H, W, nrm2, amaxpos);
+    else if (er) dwconv_channels<T, L, VEC, NORMS, true, false>(uin, w, cout, c_lo, c_hi, lp, lane, n, H, W, nrm2, amaxpos);
+    else if (ec) dwconv_channels<T, L, VEC, NORMS, false, true>(uin, w, cout, c_lo, c_hi, lp, lane, n, H, W, nrm2, amaxpos);
+    else dwconv_channels<T, L, VEC, NORMS, false, false>(uin, w, cout, c_lo, c_hi, lp, lane, n, H, W, nrm2, amaxpos);
 }
 
 // Channel norms of a stored coefficient map: one thread per position builds the chain of fused multiply-adds over the
@@ -777,10 +800,10 @@ coef_norms_kernel(const float* __restrict__ coef, int N, int C, long long P, flo
 }
 
 // Channels per chunk of the forward kernels: one chunk (norms in the same pass) when the tiles alone fill the GPU or no
-// coefficient map is stored; otherwise chunks of a multiple of `unit` channels, about 32 warps for each of the 148 SMs.
+// coefficient map is stored; otherwise chunks of a multiple of `unit` channels, about 64 warps for each of the 148 SMs.
 static int forward_chunk_channels(long long tile_warps, int C, int unit, bool has_coef)
 {
-    constexpr long long want = 148 * 32;
+    constexpr long long want = 148 * 64;              // measured on the block's shapes: 24 to 96 warps per SM tried
     if (!has_coef || tile_warps >= want || C <= 2 * unit) return C;
     const long long chunks = std::min<long long>((C + unit - 1) / unit, (want + tile_warps - 1) / tile_warps);
     int cpc = (int)((C + chunks - 1) / chunks);
