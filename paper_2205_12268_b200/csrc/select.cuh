@@ -584,6 +584,8 @@ __device__ __forceinline__ void block_find_bin_2048(const uint32_t* __restrict__
 // idx and rank are written only when asked for (want_rank) or when the threshold's ties are kept only in part
 // (then the order of positions matters); otherwise consumers compare keys with thr[n] = {threshold key, ties
 // kept, use_rank flag, number of candidate keys that were ranked (diagnostic)}.
+// MAXKPT: key registers per thread (16, or 4 for the launches that spread an image over enough threads).
+template <int MAXKPT>
 __global__ void __launch_bounds__(CL_THREADS, 1)
 select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int32_t* __restrict__ idx, float* __restrict__ tau,
                       int32_t* __restrict__ rank, const float* __restrict__ amaxpos, float* __restrict__ amax_kept,
@@ -598,10 +600,18 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
     const int base = (crank * (int)blockDim.x + (int)threadIdx.x) * kpt;  // kpt consecutive keys per thread
     const int lane = threadIdx.x & 31;
 
-    uint32_t key[CL_MAXKPT];
+    uint32_t key[MAXKPT];
 #pragma unroll
-    for (int i = 0; i < CL_MAXKPT; ++i) key[i] = (i < kpt && base + i < P) ? float_key(v[base + i]) : 0u;
+    for (int i = 0; i < MAXKPT; ++i) key[i] = (i < kpt && base + i < P) ? float_key(v[base + i]) : 0u;
     auto valid = [&](int i) { return i < kpt && base + i < P; };
+    // few keys per thread: the per-position maxima are fetched together with the keys, so that the pass over the kept
+    // positions at the end waits for no further load
+    constexpr bool PRE = MAXKPT <= 4;
+    float pre[PRE ? MAXKPT : 1];
+    if (PRE) {
+#pragma unroll
+        for (int i = 0; i < MAXKPT; ++i) pre[PRE ? i : 0] = (amaxpos && valid(i)) ? amaxpos[(size_t)n * P + base + i] : 0.0f;
+    }
 
     for (int i = threadIdx.x; i < SEL_BINS; i += blockDim.x) sm.hist[i] = 0u;
     if (threadIdx.x == 0) { sm.amax = 0u; sm.ncand = 0u; sm.thr[0] = 0xFFFFFFFFu; sm.thr[1] = 0u; sm.thr[2] = 0u; }   // thr: keep nothing
@@ -647,7 +657,7 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
         __syncthreads();
         // collect this CTA's candidates
 #pragma unroll
-        for (int i = 0; i < CL_MAXKPT; ++i) {
+        for (int i = 0; i < MAXKPT; ++i) {
             if (i >= kpt) break;
             const bool c = valid(i) && (key[i] >> 16) == prefix16;
             const unsigned m = __ballot_sync(0xFFFFFFFFu, c);
@@ -702,7 +712,7 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
             block_find_bin_2048(hist1 + (size_t)n * 3 * SEL_BINS, (uint32_t)k, sm, b1, above, nonzero);
         } else {
 #pragma unroll
-            for (int i = 0; i < CL_MAXKPT; ++i)
+            for (int i = 0; i < MAXKPT; ++i)
                 if (i < kpt) hist_add(sm.hist, key[i] >> 21, valid(i));
             cluster_find_bin(cluster, sm, cs, crank, SEL_BINS, (uint32_t)k, b1, above);
             for (int i = threadIdx.x; i < SEL_BINS; i += blockDim.x) sm.hist[i] = 0u;
@@ -711,7 +721,7 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
         const uint32_t k1 = (uint32_t)k - above;
         // round 2: next 11 bits of the keys that match
 #pragma unroll
-        for (int i = 0; i < CL_MAXKPT; ++i)     // plain atomics: these digits are mantissa bits, spread over the bins
+        for (int i = 0; i < MAXKPT; ++i)     // plain atomics: these digits are mantissa bits, spread over the bins
             if (valid(i) && (key[i] >> 21) == b1) atomicAdd(&sm.hist[(key[i] >> 10) & 0x7FFu], 1u);
         uint32_t b2;
         cluster_find_bin(cluster, sm, cs, crank, SEL_BINS, k1, b2, above);
@@ -721,7 +731,7 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
         for (int i = threadIdx.x; i < SEL_BINS; i += blockDim.x) sm.hist[i] = 0u;
         __syncthreads();
 #pragma unroll
-        for (int i = 0; i < CL_MAXKPT; ++i)
+        for (int i = 0; i < MAXKPT; ++i)
             if (valid(i) && (key[i] >> 10) == prefix) atomicAdd(&sm.hist[key[i] & 0x3FFu], 1u);
         uint32_t b3;
         cluster_find_bin(cluster, sm, cs, crank, 1024, k2, b3, above);
@@ -744,14 +754,14 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
         // every key >= threshold is kept; nobody needs the order
         if (amaxpos) {
 #pragma unroll
-            for (int i = 0; i < CL_MAXKPT; ++i)
-                if (valid(i) && key[i] >= tkey) amax = fmaxf(amax, amaxpos[(size_t)n * P + base + i]);
+            for (int i = 0; i < MAXKPT; ++i)
+                if (valid(i) && key[i] >= tkey) amax = fmaxf(amax, PRE ? pre[PRE ? i : 0] : amaxpos[(size_t)n * P + base + i]);
         }
     } else {
         // ordered compaction: ascending idx, rank map, ties to the lowest positions
         uint32_t gt = 0, eq = 0;
 #pragma unroll
-        for (int i = 0; i < CL_MAXKPT; ++i) {
+        for (int i = 0; i < MAXKPT; ++i) {
             if (!valid(i)) continue;
             gt += key[i] > tkey;
             eq += key[i] == tkey;
@@ -767,14 +777,14 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
             eq_before += c[1];
         }
 #pragma unroll
-        for (int i = 0; i < CL_MAXKPT; ++i) {
+        for (int i = 0; i < MAXKPT; ++i) {
             if (!valid(i)) continue;
             const bool is_gt = key[i] > tkey, is_eq = key[i] == tkey;
             const bool keep = is_gt || (is_eq && eq_before < need_eq);
             const uint32_t pos = gt_before + min(eq_before, need_eq);
             if (keep) {
                 if (idx) idx[(size_t)n * k + pos] = base + i;
-                if (amaxpos) amax = fmaxf(amax, amaxpos[(size_t)n * P + base + i]);
+                if (amaxpos) amax = fmaxf(amax, PRE ? pre[PRE ? i : 0] : amaxpos[(size_t)n * P + base + i]);
             }
             if (rank) rank[(size_t)n * P + base + i] = keep ? (int32_t)pos : -1;
             gt_before += is_gt;
@@ -826,7 +836,8 @@ wcc_status launch_select(const float* nrm2, int N, int P, int k, int32_t* idx, f
     WCC_CUDA_TRY(cudaGetDevice(&devc));
     if (devc >= 0 && devc < 64 && max_cs[devc] == 0) {
         max_cs[devc] = 8;
-        if (cudaFuncSetAttribute(select_cluster_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+        if (cudaFuncSetAttribute(select_cluster_kernel<CL_MAXKPT>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
+            cudaFuncSetAttribute(select_cluster_kernel<4>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
             cudaLaunchConfig_t q = {};
             q.gridDim = dim3(16, 1);
             q.blockDim = dim3(CL_THREADS);
@@ -835,7 +846,7 @@ wcc_status launch_select(const float* nrm2, int N, int P, int k, int32_t* idx, f
             qa[0].val.clusterDim.x = 16; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
             q.attrs = qa; q.numAttrs = 1;
             int nclusters = 0;
-            if (cudaOccupancyMaxActiveClusters(&nclusters, select_cluster_kernel, &q) == cudaSuccess && nclusters > 0) max_cs[devc] = 16;
+            if (cudaOccupancyMaxActiveClusters(&nclusters, select_cluster_kernel<CL_MAXKPT>, &q) == cudaSuccess && nclusters > 0) max_cs[devc] = 16;
         }
         (void)cudaGetLastError();
     }
@@ -864,8 +875,14 @@ wcc_status launch_select(const float* nrm2, int N, int P, int k, int32_t* idx, f
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        WCC_CUDA_TRY(cudaLaunchKernelEx(&cfg, select_cluster_kernel, nrm2, P, k, kpt, idx, tau, rank, amaxpos, amax_kept, hist1,
-                                        hist1_ready ? fine : (const uint32_t*)nullptr, thr, (want_rank || !thr) ? 1 : 0));
+        const uint32_t* fine_use = hist1_ready ? fine : (const uint32_t*)nullptr;
+        const int wr = (want_rank || !thr) ? 1 : 0;
+        if (kpt <= 4)                                  // few keys per thread: the instantiation with four key registers
+            WCC_CUDA_TRY(cudaLaunchKernelEx(&cfg, select_cluster_kernel<4>, nrm2, P, k, kpt, idx, tau, rank, amaxpos, amax_kept, hist1,
+                                            fine_use, thr, wr));
+        else
+            WCC_CUDA_TRY(cudaLaunchKernelEx(&cfg, select_cluster_kernel<CL_MAXKPT>, nrm2, P, k, kpt, idx, tau, rank, amaxpos, amax_kept,
+                                            hist1, fine_use, thr, wr));
         WCC_LAUNCH_CHECK();
         return WCC_OK;
     }
