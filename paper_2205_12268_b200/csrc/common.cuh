@@ -57,6 +57,12 @@ __device__ __forceinline__ float key_float(uint32_t k)
     return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
 }
 
+// Digits of a norm for the histograms that the producers of the norms hand to the selection.  A norm is a sum of squares,
+// never negative, so its sign bit carries nothing: the digits are the 11 and the 16 bits below it (digit16 >> 5 ==
+// digit11).  The masks keep a non-finite value with a sign bit inside the tables.
+__device__ __forceinline__ uint32_t norm_digit11(float v) { return (__float_as_uint(v) >> 20) & 0x7FFu; }
+__device__ __forceinline__ uint32_t norm_digit16(float v) { return (__float_as_uint(v) >> 15) & 0xFFFFu; }
+
 // Histogram increment with warp aggregation: lanes of a warp that hit the same bin elect one lane that adds their
 // count, so a bin that attracts most keys (typical for the leading digit of the norms) costs one shared-memory
 // atomic per warp instead of up to 32 serialized ones.  Must be reached by all 32 lanes (pred selects the ones that count).

@@ -479,12 +479,12 @@ fused_tiles_kernel(const __grid_constant__ CUtensorMap tmx, const Params pr)
                                 store_slots<L, true>(pr.nx.amaxpos + (size_t)n * P, lp, am);
                                 uint32_t* h = pr.nx.hist1 + (size_t)n * 3 * 2048;      // zero norms are not counted
 #pragma unroll
-                                for (int s = 0; s < 8; ++s) hist_add(h, float_key(nacc[s]) >> 21, lp.ok0 && nacc[s] != 0.0f);
+                                for (int s = 0; s < 8; ++s) hist_add(h, norm_digit11(nacc[s]), lp.ok0 && nacc[s] != 0.0f);
                                 if (lp.ok0) {
                                     uint32_t* f = pr.nx.fine + (size_t)n * 65536;
 #pragma unroll
                                     for (int s = 0; s < 8; ++s)
-                                        if (nacc[s] != 0.0f) atomicAdd(&f[float_key(nacc[s]) >> 16], 1u);
+                                        if (nacc[s] != 0.0f) atomicAdd(&f[norm_digit16(nacc[s])], 1u);
                                 }
                             }
                         }

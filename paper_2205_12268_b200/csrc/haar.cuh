@@ -879,12 +879,12 @@ struct PatchRing {
 // of every lane) over the round's channels in ascending order, so the sum is the same sequential chain a single
 // thread would build.  Inputs arrive through the per-warp cp.async ring (RING stages ahead).  Only the norms and
 // the per-position max |coef| are written, plus on request (NormsExtra): the coefficient map (tests), round 1 of
-// the select's histogram (top 11 bits of the order-preserving key of every norm), and, in extra CTAs appended to
+// the select's histogram (the 11 bits below the sign of every norm), and, in extra CTAs appended to
 // the grid, the quantized weights (one warp per output channel), which saves a launch of its own.
 struct NormsExtra {
     float* coef;          // fp32 [N][C][P] or NULL
     uint32_t* hist1;      // [N][3][2048] (round 1 first), zeroed by the caller, or NULL
-    uint32_t* fine;       // [N][65536]: histogram of the top 16 key bits, zeroed by the caller, or NULL
+    uint32_t* fine;       // [N][65536]: histogram of the 16 bits below the sign of every norm, zeroed by the caller, or NULL
     const float* Wt;      // weights to prepare in the extra CTAs, or NULL
     void* Wq;
     float* scale_w;
@@ -924,15 +924,15 @@ __device__ __forceinline__ void norms_finish(const LanePos& lp, int warp, int n,
             if (ok1) am[p1] = a1;
         }
     }
-    if (ex.hist1) {                                    // norms are >= +0: key = bits | sign bit, digit = top 11 bits
+    if (ex.hist1) {                                    // norms are >= +0: the digit is the 11 bits below the sign
         uint32_t* h = ex.hist1 + (size_t)n * 3 * 2048;
-        hist_add(h, float_key(n0) >> 21, ok0 && n0 != 0.0f);          // zero norms are not counted (see the token kernel)
-        hist_add(h, float_key(n1) >> 21, ok1 && n1 != 0.0f);
+        hist_add(h, norm_digit11(n0), ok0 && n0 != 0.0f);             // zero norms are not counted (see the token kernel)
+        hist_add(h, norm_digit11(n1), ok1 && n1 != 0.0f);
     }
     if (ex.fine) {                                     // 16-bit digits are spread out: plain atomics
         uint32_t* f = ex.fine + (size_t)n * 65536;
-        if (ok0 && n0 != 0.0f) atomicAdd(&f[float_key(n0) >> 16], 1u);
-        if (ok1 && n1 != 0.0f) atomicAdd(&f[float_key(n1) >> 16], 1u);
+        if (ok0 && n0 != 0.0f) atomicAdd(&f[norm_digit16(n0)], 1u);
+        if (ok1 && n1 != 0.0f) atomicAdd(&f[norm_digit16(n1)], 1u);
     }
 }
 
@@ -1274,16 +1274,16 @@ haar_norms_token_kernel(const __grid_constant__ CUtensorMap tmx, int N, int C, i
                 // Norms that are exactly zero are not counted: after a ReLU whole regions of a map are zero, and their
                 // positions would all hit one bin (thousands of atomics on one address).  The selection knows the number
                 // of positions, so the zeros are what the bins leave out; they rank below everything else.
-                if (ex.hist1) {                        // norms are >= +0: key = bits | sign bit, digit = top 11 bits
+                if (ex.hist1) {                        // norms are >= +0: the digit is the 11 bits below the sign
                     uint32_t* h = ex.hist1 + (size_t)n * 3 * 2048;
 #pragma unroll
-                    for (int s = 0; s < 8; ++s) hist_add(h, float_key(nacc[s]) >> 21, lp.ok0 && nacc[s] != 0.0f);
+                    for (int s = 0; s < 8; ++s) hist_add(h, norm_digit11(nacc[s]), lp.ok0 && nacc[s] != 0.0f);
                 }
                 if (ex.fine && lp.ok0) {               // 16-bit digits of non-zero norms are spread out: plain atomics
                     uint32_t* f = ex.fine + (size_t)n * 65536;
 #pragma unroll
                     for (int s = 0; s < 8; ++s)
-                        if (nacc[s] != 0.0f) atomicAdd(&f[float_key(nacc[s]) >> 16], 1u);
+                        if (nacc[s] != 0.0f) atomicAdd(&f[norm_digit16(nacc[s])], 1u);
                 }
             }
         }

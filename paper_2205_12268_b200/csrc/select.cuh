@@ -448,7 +448,7 @@ constexpr int CL_MAXKPT = 16;
 constexpr int CL_MAXCS = 16;          // 8 is the portable cluster size; 16 needs the non-portable opt-in
 constexpr int CL_CAND_CTA = 512;     // candidate slots per CTA
 constexpr int CL_CAND_MAX = 1024;    // most candidates ranked by brute force; beyond that: histogram rounds
-constexpr int FINE_BINS = 65536;     // histogram of the top 16 key bits, filled by the producer of the norms
+constexpr int FINE_BINS = 65536;     // histogram of the 16 bits below the sign of every norm, filled by the producer of the norms
 
 struct ClusterSmem {
     uint32_t hist[SEL_BINS];
@@ -459,7 +459,7 @@ struct ClusterSmem {
     uint32_t res[3];                // found bin, keys above it, keys in it
     uint32_t tot[CL_MAXCS];
     uint32_t amax;
-    uint32_t ncand;                 // candidates of this CTA (keys whose top 16 bits hold the threshold)
+    uint32_t ncand;                 // candidates of this CTA (keys in the 16-bit bin that holds the threshold)
     uint32_t cand[CL_CAND_CTA];
     __align__(16) uint32_t all[CL_CAND_MAX];      // candidates of the whole cluster
     uint32_t thr[3];                // threshold key, ties to keep, ties in total
@@ -578,8 +578,8 @@ __device__ __forceinline__ void block_find_bin_2048(const uint32_t* __restrict__
     __syncthreads();
 }
 
-// hist1 ([N][3][2048], round 1 first) and fine ([N][65536]) are optional histograms of the top 11 and top 16 key bits
-// that the producer of the norms filled; with both, the threshold is usually found without any histogram round:
+// hist1 ([N][3][2048], round 1 first) and fine ([N][65536]) are optional histograms of the 11 and 16 bits below the sign
+// of every norm (norm_digit11 / norm_digit16: norms are never negative) that the producer of the norms filled; with both, the threshold is usually found without any histogram round:
 // the 16-bit bin that holds the k-th key contains few keys, which the cluster gathers and ranks directly.
 // idx and rank are written only when asked for (want_rank) or when the threshold's ties are kept only in part
 // (then the order of positions matters); otherwise consumers compare keys with thr[n] = {threshold key, ties
@@ -659,7 +659,7 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
 #pragma unroll
         for (int i = 0; i < MAXKPT; ++i) {
             if (i >= kpt) break;
-            const bool c = valid(i) && (key[i] >> 16) == prefix16;
+            const bool c = valid(i) && ((key[i] >> 15) & 0xFFFFu) == prefix16;
             const unsigned m = __ballot_sync(0xFFFFFFFFu, c);
             if (m) {
                 uint32_t off = 0;
@@ -705,8 +705,15 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
         }
     }
     if (!found) {
-        // round 1: top 11 bits (only the bin search when the producer of the norms histogrammed them)
+        // round 1: top 11 bits (only the bin search when the producer of the norms histogrammed them).  The producer's
+        // digits start below the sign bit (norm_digit11), so with its histogram the rounds run on the keys shifted left
+        // by one: 11 + 11 + 9 bits and a zero; the threshold is shifted back at the end.
         uint32_t b1, above;
+        const bool shifted = hist1 != nullptr;
+        if (shifted) {
+#pragma unroll
+            for (int i = 0; i < MAXKPT; ++i) key[i] <<= 1;
+        }
         if (hist1) {
             uint32_t nonzero;
             block_find_bin_2048(hist1 + (size_t)n * 3 * SEL_BINS, (uint32_t)k, sm, b1, above, nonzero);
@@ -738,6 +745,11 @@ select_cluster_kernel(const float* __restrict__ nrm2, int P, int k, int kpt, int
         tkey = (prefix << 10) | b3;
         need_eq = k2 - above;
         total_eq = sm.res[2];
+        if (shifted) {                                 // back to whole keys (every norm has the sign bit of +0 and above)
+            tkey = (tkey >> 1) | 0x80000000u;
+#pragma unroll
+            for (int i = 0; i < MAXKPT; ++i) key[i] = (key[i] >> 1) | 0x80000000u;
+        }
     }
     if (tau && crank == 0 && threadIdx.x == 0) tau[n] = key_float(tkey);
 
@@ -818,7 +830,7 @@ __global__ void thr_use_rank_kernel(uint32_t* thr, int N)
 inline bool select_in_cluster(int P) { return P <= 8 * CL_THREADS * CL_MAXKPT; }
 
 // hist1_ready: the caller has already cleared the zero region of the workspace (carve_select_ws(...).hist,
-// zero_bytes) and filled round 1 of the histogram (top 11 key bits of every norm) before this call.
+// zero_bytes) and filled round 1 of the histogram (norm_digit11 of every non-zero norm) before this call.
 // fine / thr: see select_cluster_kernel; want_rank: idx (if non-NULL) and rank must be written even when the
 // threshold alone would do.  Without thr the rank map and idx are always written.
 wcc_status launch_select(const float* nrm2, int N, int P, int k, int32_t* idx, float* tau,
