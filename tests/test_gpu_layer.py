@@ -125,6 +125,24 @@ def test_layer_partial_ties_at_the_threshold(wcc):
         _run_and_compare(wcc, w)
 
 
+@pytest.mark.parametrize("distinct", [False, True], ids=["equal", "distinct"])
+def test_layer_threshold_bin_holds_more_keys_than_can_be_ranked(wcc, distinct):
+    """Thousands of norms fall into the histogram bin of the threshold (a 2x2 block tiled over a 128x128 map gives four
+    norm values, 4096 positions each; with `distinct` every position also gets a tiny relative perturbation, so the keys
+    of a bin differ in their low bits): the select cannot rank that many candidates directly and has to run its digit
+    rounds on top of the first pass's histogram.  k cuts through such a bin, through a run of equal keys, and lands on
+    its ends."""
+    w = inputs.custom("crowd", 4, 2, 3, 5, 128, 128, "f32", 1, 0.5, 8, n_sin=3, fmax=2.0)
+    blk = w.x[:, :, :2, :2].copy()
+    w.x[:] = np.tile(blk, (1, 1, 64, 64))
+    if distinct:
+        rng = np.random.default_rng(11)
+        w.x *= (1.0 + 1e-4 * rng.standard_normal(w.x.shape)).astype(np.float32)
+    for k in (1, 3000, 4096, 4097, 9000, 16383):
+        w.k = k
+        _run_and_compare(wcc, w)
+
+
 def test_layer_k_equals_one_and_all(wcc):
     for k in (1, 16 * 16):
         w = inputs.custom("edge", 5, 2, 5, 7, 16, 16, "f32", 2, 0.5, 8, k=k)
