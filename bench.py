@@ -36,10 +36,10 @@ NCU_TRAFFIC = {
     # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu captures summarised under profiles/.
     # C4 was captured with N=24 images (x = 189 MB > L2) and is divided by 2, C2 with N=16 and divided by 4: every stage
     # is per image, so traffic grows in proportion to the batch.
-    ("C4", "fused_pass2"): {"bytes": (191774208 + 135275264) / 2, "src": "2fcf053994b2"},
-    ("C4", "haar_norms"): {"bytes": (189054208 + 4007424) / 2, "src": "2fcf053994b2"},
-    ("C2", "fused_pass2"): {"bytes": (153169920 + 13190656) / 4, "src": "2fcf053994b2"},
-    ("C2", "haar_norms"): {"bytes": (151204608 + 4880128) / 4, "src": "2fcf053994b2"},
+    ("C4", "fused_pass2"): {"bytes": (191781376 + 134613504) / 2, "src": "cde0b5a6e295"},
+    ("C4", "haar_norms"): {"bytes": (189183744 + 3707392) / 2, "src": "cde0b5a6e295"},
+    ("C2", "fused_pass2"): {"bytes": (153168896 + 13833984) / 4, "src": "cde0b5a6e295"},
+    ("C2", "haar_norms"): {"bytes": (151312384 + 4362752) / 4, "src": "cde0b5a6e295"},
 }
 
 
