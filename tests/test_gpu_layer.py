@@ -170,6 +170,13 @@ def test_layer_named_workloads_full_size(wcc, name, staged):
     _run_and_compare(wcc, inputs.make(name), staged=staged)
 
 
+@pytest.mark.parametrize("name,batch", [("C4", 24), ("C2", 16)], ids=["C4x24", "C2x16"])
+def test_layer_profiled_batches_full_size(wcc, name, batch):
+    """The batches the DRAM counters are taken on (the named workload with more images, so that x exceeds the L2):
+    several waves of every kernel, the first pass walking more than one tile per CTA."""
+    _run_and_compare(wcc, inputs.make(name, N=batch))
+
+
 def _random_shapes(count, seed):
     rng = np.random.default_rng(seed)
     out = []
