@@ -137,7 +137,7 @@ wcc_status wcc_select_topk_static(const float* nrm2, int N, int P, int k, int32_
  *   y   out: [N][Cout][H][Wd] of dt; must not overlap x
  *   ws     : scratch of at least wcc_workspace_bytes(...) bytes, 256-byte aligned; contents undefined afterwards
  * Execution: three launches, two passes over x around the selection.  Pass 1 transforms x in registers and keeps
- * only the channel norms, the per-position max |coefficient| and two histograms of the norms' leading key bits (it
+ * only the channel norms, the per-position max |coefficient| and two histograms of the norms' leading bits below the sign (it
  * also quantizes the weights); the selection finds the threshold norm, max|kept| and, only if ties at the threshold
  * are kept in part, the rank of every position; pass 2 transforms x again, zeroes the dropped positions, quantizes
  * into shared memory, runs the contraction on tensor cores, dequantizes, applies the inverse transform and stores y.
