@@ -81,7 +81,7 @@ def stage_bytes(w, stage: str) -> float:
 class ClockSampler(threading.Thread):
     """Samples SM clock and clock-event reasons of one GPU through NVML while the timed region runs."""
 
-    def __init__(self, index: int, period: float = 0.005):
+    def __init__(self, index: int, period: float = 0.001):
         super().__init__(daemon=True)
         self.index, self.period = index, period
         self.samples, self.reasons, self.sm_max = [], set(), None
